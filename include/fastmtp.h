@@ -1,0 +1,216 @@
+/*
+ * fastmtp.h -- C ABI of the B200 (sm_100a) FastMTP draft / verify library.
+ *
+ * The library implements the inference hot path of FastMTP (arXiv 2509.18362): the
+ * recursive K-step draft of one position-shared Multi-Token-Prediction head with a
+ * compressed-vocabulary output head, the greedy verification that consumes the drafts,
+ * and a target-decoder step that reuses the same decoder-layer kernels.
+ *
+ * Conventions shared by every call
+ *   - All tensors are dense, row-major, caller-owned. "dev" = device (HBM) pointer,
+ *     "host" = host pointer. bf16 values are passed as raw 16-bit patterns (fmtp_bf16).
+ *   - Matrices are [out, in]. Token ids, lengths and indices are int32.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Device-pointer entry points only enqueue work on `stream`; they never synchronise
+ *     and never read device memory on the host. The *_host entry points copy their
+ *     per-step inputs host->device, run, copy results device->host and synchronise
+ *     `stream` before returning.
+ *   - Return value: FMTP_OK (0) or a negative fmtp_status. On a negative return nothing
+ *     was enqueued. Errors only a kernel can see (token id >= vocab, page index out of
+ *     range, position beyond the block table, a bounded wait that ran out) never fault:
+ *     the access is clamped or skipped, a bit is OR-ed into the caller's `dev_status`
+ *     word (FMTP_DEV_* flags) and the kernel runs to completion.
+ *   - The library allocates no device memory of its own except where stated: the caller
+ *     sizes a workspace with fmtp_workspace_bytes() and hands it over with
+ *     fmtp_set_workspace(). One context must not be used from two streams at once.
+ */
+#ifndef FASTMTP_H
+#define FASTMTP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef uint16_t fmtp_bf16;
+typedef struct fmtp_ctx fmtp_ctx;
+
+typedef enum {
+    FMTP_OK = 0,
+    FMTP_EINVAL = -1,       /* null pointer, non-positive size, misaligned pointer        */
+    FMTP_ESHAPE = -2,       /* shape outside what the kernels support (see fmtp_create)   */
+    FMTP_EUNSUPPORTED = -3, /* valid request that this build does not implement           */
+    FMTP_ENOMEM = -4,       /* workspace missing or too small                             */
+    FMTP_ECUDA = -5,        /* a CUDA runtime call failed (see fmtp_last_cuda_error)       */
+    FMTP_ETIMEOUT = -6,
+    FMTP_EBOUNDS = -7
+} fmtp_status;
+
+/* Bits OR-ed into *dev_status by kernels. */
+#define FMTP_DEV_BAD_TOKEN   0x1u  /* a token id or subset id outside [0, vocab) was clamped  */
+#define FMTP_DEV_BAD_PAGE    0x2u  /* a block-table entry outside [0, num_pages) was clamped  */
+#define FMTP_DEV_BAD_POS     0x4u  /* a position beyond max_pages_per_seq*page_size: KV write skipped */
+#define FMTP_DEV_TIMEOUT     0x8u  /* a bounded device-side wait gave up; outputs are invalid */
+#define FMTP_DEV_ALL_NAN     0x10u /* an argmax row held no comparable value; id 0 / lowest id returned */
+
+/* Model geometry and capacity limits (fixed for the life of a context).
+ * Supported: head_dim in {64, 128}; d, n_q_heads*head_dim and ffn multiples of 16 with
+ * d a multiple of 64; n_q_heads a multiple of n_kv_heads with at most 8 query heads per
+ * KV head; max_rows <= 8 (rows = batch x rows-per-sequence handled in one call). */
+typedef struct {
+    int32_t d, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
+    int32_t n_layers;      /* target decoder depth (fastmtp_target_step); the MTP head has 1 */
+    float rms_eps, rope_theta;
+    int32_t page_size;     /* tokens per KV page */
+    int32_t max_rows;      /* largest batch x rows-per-sequence of any call                 */
+    int32_t max_K;         /* largest number of draft steps                                  */
+    int32_t max_ctx;       /* largest position + 1 any sequence may reach                    */
+} fmtp_shape;
+
+/* One pre-norm decoder layer (Sec. 2.1 of the paper: the transformer block inside the MTP
+ * module; also each target layer). All dev, bf16. RMSNorm gains g_* are [d];
+ * wq [Hq*dh, d], wk/wv [Hkv*dh, d], wo [d, Hq*dh], w_gate/w_up [ffn, d], w_down [d, ffn]. */
+typedef struct {
+    const fmtp_bf16 *g_in, *wq, *wk, *wv, *wo, *g_post, *w_gate, *w_up, *w_down;
+} fmtp_layer_w;
+
+/* The MTP head (Sec. 2.1 "Architecture Design"): embed [vocab, d] and lm_head [vocab, d] are
+ * the main model's (shared, Sec. 2.2); g_hnorm / g_enorm [d] normalise the incoming hidden
+ * state and the token embedding; w_proj [d, 2d] projects their concatenation
+ * [norm(h) ; norm(emb)]; g_final [d] is the norm before the output head. */
+typedef struct {
+    const fmtp_bf16 *embed, *lm_head, *g_hnorm, *g_enorm, *w_proj, *g_final;
+    fmtp_layer_w layer;
+} fmtp_mtp_w;
+
+/* The target decoder: `layers` is a HOST array of n_layers entries holding dev pointers. */
+typedef struct {
+    const fmtp_bf16 *embed, *lm_head, *g_final;
+    const fmtp_layer_w *layers;
+} fmtp_target_w;
+
+/* Paged bf16 KV cache of one layer. k_pages / v_pages: dev [num_pages, Hkv, page_size, dh]
+ * (keys stored after the rotary embedding). block_table: dev [B, max_pages_per_seq] page
+ * indices; seq_lens: dev [B] committed tokens per sequence. Calls read seq_lens on the
+ * device (so a replayed launch sees current values) and never modify it. */
+typedef struct {
+    fmtp_bf16 *k_pages, *v_pages;
+    const int32_t *block_table;
+    const int32_t *seq_lens;
+    int32_t num_pages, max_pages_per_seq;
+} fmtp_kv;
+
+/* ---- context ------------------------------------------------------------------------ */
+
+/* Validates `shape` for the current device and creates a context (host memory only).
+ * FMTP_ESHAPE if the geometry is unsupported, FMTP_ECUDA if no sm_100 device is current. */
+int fmtp_create(const fmtp_shape *shape, fmtp_ctx **out);
+int fmtp_destroy(fmtp_ctx *ctx);
+
+/* Bytes of device scratch the context needs (activations between phases, attention
+ * partials, rotary table, control words). */
+size_t fmtp_workspace_bytes(const fmtp_ctx *ctx);
+
+/* Hands `bytes` of 256-byte-aligned device memory to the context; the context clears it,
+ * builds its rotary cos/sin table in it (computed on the host in double precision) and
+ * synchronises the device once. The caller keeps ownership and must keep it alive and
+ * untouched while the context is used. */
+int fmtp_set_workspace(fmtp_ctx *ctx, void *dev, size_t bytes);
+
+const char *fmtp_strerror(int status);
+/* cudaError_t of the most recent failing CUDA call made through this context (0 if none). */
+int fmtp_last_cuda_error(const fmtp_ctx *ctx);
+/* Number of kernel launches this context has enqueued so far. */
+long long fmtp_launch_count(const fmtp_ctx *ctx);
+
+/* ---- draft: Sec. 2.3 "Drafting phase", Sec. 2.1 steps k=1 / k>1, Sec. 2.2 Eq. 3 -------- */
+
+/* Recursive K-step draft for B sequences.
+ *
+ * Step 1 consumes, per sequence b, the pair (h_last[b], tok_last[b]): the target's last
+ * hidden state (the post-final-norm vector that feeds the target's output head) and the
+ * newest verified token. The pair occupies MTP-cache position L_b = mtp_kv->seq_lens[b].
+ * Each step embeds the token, RMS-normalises hidden state and embedding, projects their
+ * concatenation 2d -> d, runs one decoder layer (appending this position's K/V to the MTP
+ * cache and attending over positions 0..pos), applies the final norm, and takes the argmax
+ * of the output head restricted to rows `vocab_subset` (Eq. 3) -- ties go to the lowest
+ * token id; no logits are written. Step k >= 2 consumes the head's own previous output
+ * hidden state (kept in fp32) and the previous draft at position L_b + k - 1.
+ * All K steps run inside one kernel launch without returning to the host.
+ *
+ *   h_last        dev [B, d] bf16          tok_last     dev [B] int32
+ *   vocab_subset  dev [N] int32 distinct ids in [0, vocab), any order; NULL => full vocab (N ignored)
+ *   out_drafts    dev [B, K] int32         out_h        dev [B, K, d] bf16 or NULL (post-final-norm)
+ *   out_logits    dev [B, K, N] fp32 or NULL: debug copy of the subset logits (defeats the
+ *                 "no logits written" property; leave NULL in production)
+ *   dev_status    dev 1 word, OR-ed with FMTP_DEV_* flags; may be NULL
+ *
+ * The call writes MTP-cache slots L_b .. L_b+K-1 and does not change seq_lens; the caller
+ * commits by advancing seq_lens (normally by 1: slot L_b was computed from the target's
+ * hidden state, later slots are speculative and are overwritten by the next round).
+ * Requires B <= max_rows, K <= max_K, L_b + K <= max_ctx.
+ */
+int fastmtp_draft(fmtp_ctx *ctx, const fmtp_mtp_w *w,
+                  const fmtp_bf16 *h_last, const int32_t *tok_last,
+                  const fmtp_kv *mtp_kv, int B, int K,
+                  const int32_t *vocab_subset, int N,
+                  int32_t *out_drafts, fmtp_bf16 *out_h, float *out_logits,
+                  uint32_t *dev_status, void *stream);
+
+/* Same operation with the per-step inputs and the result in HOST memory: h_last host
+ * [B,d] bf16 and tok_last host [B] are copied to the device, the draft runs, out_drafts
+ * host [B,K] is copied back and `stream` is synchronised. Weights, subset and KV cache stay
+ * on the device. Returns FMTP_EBOUNDS / FMTP_ETIMEOUT if the kernels flagged a problem. */
+int fastmtp_draft_host(fmtp_ctx *ctx, const fmtp_mtp_w *w,
+                       const fmtp_bf16 *h_last_host, const int32_t *tok_last_host,
+                       const fmtp_kv *mtp_kv, int B, int K,
+                       const int32_t *vocab_subset, int N,
+                       int32_t *out_drafts_host, void *stream);
+
+/* ---- verification: Sec. 2.3 "Verification phase" (greedy, Sec. 3.1) --------------------- */
+
+/* g[b,j] = argmax over the full vocabulary of target_logits[b,j,:] (ties to the lowest id,
+ * NaN never wins); accept_len[b] = number of leading drafts with drafts[b,j] == g[b,j];
+ * bonus[b] = g[b, accept_len[b]]: the token the target emits after the accepted prefix, so
+ * a round emits accept_len + 1 tokens.
+ *
+ *   target_logits dev [B, K+1, V] bf16     drafts       dev [B, K] int32 (ignored if K == 0)
+ *   out_accept_len, out_bonus dev [B]      out_argmax   dev [B, K+1] or NULL
+ * Requires B*(K+1) <= 4096 rows. Uses the context workspace for per-row keys.
+ */
+int fastmtp_verify_accept(fmtp_ctx *ctx, const fmtp_bf16 *target_logits, const int32_t *drafts,
+                          int B, int K, int V,
+                          int32_t *out_accept_len, int32_t *out_bonus, int32_t *out_argmax,
+                          uint32_t *dev_status, void *stream);
+
+/* Host-buffer form: logits and drafts are copied in, accept_len / bonus copied out. */
+int fastmtp_verify_accept_host(fmtp_ctx *ctx, const fmtp_bf16 *target_logits_host,
+                               const int32_t *drafts_host, int B, int K, int V,
+                               int32_t *out_accept_len_host, int32_t *out_bonus_host, void *stream);
+
+/* ---- target decoder step (Sec. 2.1: embedding, transformer layers F, output head W) ----- */
+
+/* Runs M new tokens per sequence through the n_layers-deep target stack with the same
+ * decoder-layer kernels as the draft: rows are causal among themselves and sit at cache
+ * positions L_b .. L_b+M-1 (L_b = layer_kvs[0].seq_lens[b]); K/V of those positions are
+ * written to every layer's cache, seq_lens is not changed. M = 1 is plain decoding,
+ * M = K+1 scores [last token, drafts] for verification.
+ *
+ *   tokens      dev [B, M] int32           layer_kvs   HOST array [n_layers] of fmtp_kv
+ *   out_h       dev [B, M, d] bf16 (post-final-norm hidden states) or NULL
+ *   out_logits  dev [B, M, V] bf16 full-vocabulary logits or NULL
+ *   out_argmax  dev [B, M] int32 greedy token of every row (decided on the bf16-rounded
+ *               logits, ties to the lowest id) or NULL
+ * Requires B*M <= max_rows. A row's results do not depend on B or M.
+ */
+int fastmtp_target_step(fmtp_ctx *ctx, const fmtp_target_w *w, const int32_t *tokens,
+                        const fmtp_kv *layer_kvs, int B, int M,
+                        fmtp_bf16 *out_h, fmtp_bf16 *out_logits, int32_t *out_argmax,
+                        uint32_t *dev_status, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FASTMTP_H */

@@ -1,0 +1,443 @@
+// C ABI of the library: context, workspace layout, argument validation and the entry points
+// declared in include/fastmtp.h. Host code only marshals; every step of the path runs in the
+// kernels of megakernel.cu and verify.cu.
+#include "../../include/fastmtp.h"
+#include "mega.cuh"
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace fmtp;
+
+struct fmtp_ctx {
+    fmtp_shape shape;
+    int n_sm;
+    int smem_optin;
+    int KC;
+    int dp, qp, Fp;
+    int max_chunks;
+    int stage_F_pref;          // -1 auto, 0 never, 1 whenever it fits (env FMTP_STAGE_F)
+    int stages_cap;            // upper bound on ring stages (env FMTP_STAGES)
+    // workspace
+    unsigned char *ws;
+    size_t ws_bytes, ws_need;
+    Scratch s;
+    size_t ctrl_off, ctrl_bytes;
+    unsigned long long *vkeys;
+    uint32_t *vcounter;
+    // staging for the *_host entry points (device side inside the workspace, host side pinned)
+    bf16_t *st_h;
+    int32_t *st_tok, *st_out;
+    uint32_t *st_status;
+    void *pinned;
+    size_t pinned_bytes;
+    void *vstage;              // grow-only device staging of fastmtp_verify_accept_host
+    size_t vstage_bytes;
+    int last_cuda;
+    long long launches;
+};
+
+namespace {
+
+constexpr int kVerifyMaxRows = 4096;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Carver {
+    size_t off = 0;
+    unsigned char *base = nullptr;
+    template <typename T>
+    T *take(size_t n) {
+        off = align_up(off, 256);
+        T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += n * sizeof(T);
+        return p;
+    }
+};
+
+// Lays the scratch buffers out inside the workspace (base == nullptr: size query only).
+size_t layout(fmtp_ctx *c, unsigned char *base) {
+    const fmtp_shape &sh = c->shape;
+    const int R = sh.max_rows, d = sh.d;
+    const int qdim = sh.n_q_heads * sh.head_dim, kvdim = sh.n_kv_heads * sh.head_dim;
+    Carver cv;
+    cv.base = base;
+    Scratch &s = c->s;
+    s.x0 = cv.take<float>((size_t)R * d);
+    s.x1 = cv.take<float>((size_t)R * d);
+    s.qkv = cv.take<float>((size_t)R * (qdim + 2 * kvdim));
+    s.actD_hi = cv.take<bf16_t>((size_t)R * c->dp);  s.actD_lo = cv.take<bf16_t>((size_t)R * c->dp);
+    s.actP_hi = cv.take<bf16_t>((size_t)R * c->dp);  s.actP_lo = cv.take<bf16_t>((size_t)R * c->dp);
+    s.actH_hi = cv.take<bf16_t>((size_t)R * c->dp);  s.actH_lo = cv.take<bf16_t>((size_t)R * c->dp);
+    s.actR_hi = cv.take<bf16_t>((size_t)R * c->dp);  s.actR_lo = cv.take<bf16_t>((size_t)R * c->dp);
+    s.actO_hi = cv.take<bf16_t>((size_t)R * c->qp);  s.actO_lo = cv.take<bf16_t>((size_t)R * c->qp);
+    s.actF_hi = cv.take<bf16_t>((size_t)R * c->Fp);  s.actF_lo = cv.take<bf16_t>((size_t)R * c->Fp);
+    s.ssA = cv.take<float>((size_t)c->n_sm * kMaxRows);
+    s.ssB = cv.take<float>((size_t)c->n_sm * kMaxRows);
+    s.ssC = cv.take<float>((size_t)c->n_sm * kMaxRows);
+    s.ssD = cv.take<float>((size_t)c->n_sm * kMaxRows);
+    s.att_part = cv.take<float>((size_t)R * sh.n_q_heads * c->max_chunks * (sh.head_dim + 2));
+    // control block, cleared by one memset before every launch
+    cv.off = align_up(cv.off, 256);
+    c->ctrl_off = cv.off;
+    int nkeys = (sh.max_K > 1 ? sh.max_K : 1) * kMaxRows;
+    s.keys = cv.take<unsigned long long>((size_t)nkeys);
+    s.att_cnt = cv.take<uint32_t>((size_t)R * sh.n_kv_heads);
+    s.barrier = cv.take<uint32_t>(1);
+    s.abort_flag = cv.take<uint32_t>(1);
+    s.status = cv.take<uint32_t>(1);
+    cv.off = align_up(cv.off, 256);
+    c->ctrl_bytes = cv.off - c->ctrl_off;
+    float *cosb = cv.take<float>((size_t)sh.max_ctx * (sh.head_dim / 2));
+    float *sinb = cv.take<float>((size_t)sh.max_ctx * (sh.head_dim / 2));
+    s.rope_cos = cosb;
+    s.rope_sin = sinb;
+    c->vkeys = cv.take<unsigned long long>(kVerifyMaxRows);
+    c->vcounter = cv.take<uint32_t>(1);
+    c->st_h = cv.take<bf16_t>((size_t)R * d);
+    c->st_tok = cv.take<int32_t>((size_t)R);
+    c->st_out = cv.take<int32_t>((size_t)R * (sh.max_K > 1 ? sh.max_K : 1) + 2 * kVerifyMaxRows);
+    c->st_status = cv.take<uint32_t>(1);
+    return align_up(cv.off, 256);
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int cuda_fail(fmtp_ctx *c, cudaError_t e) {
+    c->last_cuda = (int)e;
+    return FMTP_ECUDA;
+}
+
+int act_stride(int len) { return ((len + 31) & ~31) + 32; }
+
+// Fills geometry / shared-memory configuration for a call with R rows (M rows per sequence).
+int configure(fmtp_ctx *c, MegaParams &p, int mode, int B, int M) {
+    const fmtp_shape &sh = c->shape;
+    std::memset(&p, 0, sizeof(p));
+    p.d = sh.d; p.Hq = sh.n_q_heads; p.Hkv = sh.n_kv_heads; p.dh = sh.head_dim; p.F = sh.ffn; p.V = sh.vocab;
+    p.qdim = p.Hq * p.dh; p.kvdim = p.Hkv * p.dh; p.page = sh.page_size;
+    p.dp = c->dp; p.qp = c->qp; p.Fp = c->Fp;
+    p.eps = sh.rms_eps;
+    p.KC = c->KC;
+    p.row_stride = p.KC * 2 + 64;
+    p.stage_bytes = kTileRows * p.row_stride;
+    p.max_chunks = c->max_chunks;
+    p.max_ctx = sh.max_ctx;
+    p.mode = mode; p.B = B; p.M = M; p.R = B * M;
+    const int R = p.R, Gq = p.Hq / p.Hkv;
+    size_t attn = ((size_t)M * Gq * p.dh + 2 * (size_t)M * p.dh + (size_t)kConsumerWarps * Gq * (p.dh + 2)) * 4;
+    size_t actd = (size_t)2 * R * act_stride(mode == 0 ? 2 * p.d : (p.d > p.qdim ? p.d : p.qdim)) * 2;
+    size_t actq = (size_t)2 * R * act_stride(p.qdim) * 2;
+    size_t base = attn > actd ? attn : actd;
+    if (actq > base) base = actq;
+    size_t actF = (size_t)2 * R * act_stride(p.F) * 2;
+    size_t withF = base > actF ? base : actF;
+    base = align_up(base, 128);
+    withF = align_up(withF, 128);
+    size_t fixed = mega_fixed_smem(R);
+    size_t avail = (size_t)c->smem_optin;
+    int st_noF = fixed + base < avail ? (int)((avail - fixed - base) / p.stage_bytes) : 0;
+    int st_F = fixed + withF < avail ? (int)((avail - fixed - withF) / p.stage_bytes) : 0;
+    bool useF;
+    if (c->stage_F_pref == 0) useF = false;
+    else if (c->stage_F_pref == 1) useF = st_F >= 2;
+    else useF = st_F >= 4 || st_F >= st_noF;
+    p.stage_F_in_smem = useF ? 1 : 0;
+    p.scratch_smem = (int)(useF ? withF : base);
+    int ns = useF ? st_F : st_noF;
+    if (ns > kMaxStages) ns = kMaxStages;
+    if (ns > c->stages_cap) ns = c->stages_cap;
+    if (ns < 2) return FMTP_ESHAPE;
+    p.n_stages = ns;
+    p.s = c->s;
+    return FMTP_OK;
+}
+
+void set_layer(LayerPtrs &dst, const fmtp_layer_w &w) {
+    dst.g_in = w.g_in; dst.wq = w.wq; dst.wk = w.wk; dst.wv = w.wv; dst.wo = w.wo;
+    dst.g_post = w.g_post; dst.w_gate = w.w_gate; dst.w_up = w.w_up; dst.w_down = w.w_down;
+}
+bool layer_ok(const fmtp_layer_w &w) {
+    const void *ps[] = {w.g_in, w.wq, w.wk, w.wv, w.wo, w.g_post, w.w_gate, w.w_up, w.w_down};
+    for (const void *q : ps) if (!q || !aligned16(q)) return false;
+    return true;
+}
+bool kv_ok(const fmtp_kv &kv) {
+    return kv.k_pages && kv.v_pages && kv.block_table && kv.seq_lens && kv.num_pages > 0 && kv.max_pages_per_seq > 0 &&
+           aligned16(kv.k_pages) && aligned16(kv.v_pages);
+}
+void set_kv(KvPtrs &dst, const fmtp_kv &kv) {
+    dst.k_pages = kv.k_pages; dst.v_pages = kv.v_pages; dst.block_table = kv.block_table;
+    dst.seq_lens = kv.seq_lens; dst.num_pages = kv.num_pages; dst.max_pages = kv.max_pages_per_seq;
+}
+
+int launch_mega(fmtp_ctx *c, MegaParams &p, cudaStream_t st) {
+    cudaError_t e = cudaMemsetAsync(c->ws + c->ctrl_off, 0, c->ctrl_bytes, st);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    int err = 0;
+    size_t smem = mega_smem_bytes(p);
+    int grid = mega_max_grid(smem, &err);
+    if (err) return cuda_fail(c, (cudaError_t)err);
+    if (grid < 1) return FMTP_ESHAPE;
+    if (grid > c->n_sm) grid = c->n_sm;
+    err = mega_launch(p, grid, st);
+    if (err) return cuda_fail(c, (cudaError_t)err);
+    c->launches++;
+    return FMTP_OK;
+}
+
+int status_to_code(uint32_t st) {
+    if (st & FMTP_DEV_TIMEOUT) return FMTP_ETIMEOUT;
+    if (st) return FMTP_EBOUNDS;
+    return FMTP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *fmtp_strerror(int status) {
+    switch (status) {
+        case FMTP_OK: return "ok";
+        case FMTP_EINVAL: return "invalid argument (null, misaligned or non-positive)";
+        case FMTP_ESHAPE: return "shape not supported by the kernels";
+        case FMTP_EUNSUPPORTED: return "not implemented in this build";
+        case FMTP_ENOMEM: return "workspace missing or too small";
+        case FMTP_ECUDA: return "CUDA runtime error (see fmtp_last_cuda_error)";
+        case FMTP_ETIMEOUT: return "a bounded device-side wait gave up";
+        case FMTP_EBOUNDS: return "a kernel clamped an out-of-range id, page or position";
+        default: return "unknown status";
+    }
+}
+
+int fmtp_create(const fmtp_shape *sh, fmtp_ctx **out) {
+    if (!sh || !out) return FMTP_EINVAL;
+    *out = nullptr;
+    if (sh->d <= 0 || sh->n_q_heads <= 0 || sh->n_kv_heads <= 0 || sh->ffn <= 0 || sh->vocab <= 0 ||
+        sh->page_size <= 0 || sh->max_rows <= 0 || sh->max_ctx <= 0 || sh->max_K < 0 || sh->n_layers < 0)
+        return FMTP_EINVAL;
+    if (sh->head_dim != 64 && sh->head_dim != 128) return FMTP_ESHAPE;
+    if (sh->d % 64 || sh->ffn % 16 || sh->n_q_heads % sh->n_kv_heads || sh->n_q_heads / sh->n_kv_heads > 8 ||
+        sh->max_rows > kMaxRows || sh->n_layers > kMaxLayers)
+        return FMTP_ESHAPE;
+    int dev = 0, major = 0, sms = 0, optin = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess || major < 10) return FMTP_ECUDA;
+    fmtp_ctx *c = new (std::nothrow) fmtp_ctx();
+    if (!c) return FMTP_ENOMEM;
+    std::memset(c, 0, sizeof(*c));
+    c->shape = *sh;
+    c->n_sm = sms;
+    c->smem_optin = optin;
+    c->KC = (sh->d % 512 == 0) ? 512 : (sh->d % 256 == 0) ? 256 : (sh->d % 128 == 0) ? 128 : 64;
+    if (const char *v = std::getenv("FMTP_KC")) {
+        int kc = std::atoi(v);
+        if ((kc == 64 || kc == 128 || kc == 256 || kc == 512 || kc == 1024) && sh->d % kc == 0) c->KC = kc;
+    }
+    c->dp = (sh->d + 31) & ~31;
+    c->qp = (sh->n_q_heads * sh->head_dim + 31) & ~31;
+    c->Fp = (sh->ffn + 31) & ~31;
+    c->max_chunks = (sh->max_ctx + kAttnChunk - 1) / kAttnChunk;
+    c->stage_F_pref = -1;
+    if (const char *v = std::getenv("FMTP_STAGE_F")) c->stage_F_pref = std::atoi(v);
+    c->stages_cap = kMaxStages;
+    if (const char *v = std::getenv("FMTP_STAGES")) { int n = std::atoi(v); if (n >= 2 && n <= kMaxStages) c->stages_cap = n; }
+    c->ws_need = layout(c, nullptr);
+    c->pinned_bytes = (size_t)sh->max_rows * sh->d * 2 + (size_t)sh->max_rows * 4 * (2 + (sh->max_K > 1 ? sh->max_K : 1)) +
+                      2 * kVerifyMaxRows * 4 + 256;
+    e = cudaMallocHost(&c->pinned, c->pinned_bytes);
+    if (e != cudaSuccess) { delete c; return FMTP_ECUDA; }
+    *out = c;
+    return FMTP_OK;
+}
+
+int fmtp_destroy(fmtp_ctx *c) {
+    if (!c) return FMTP_EINVAL;
+    if (c->pinned) cudaFreeHost(c->pinned);
+    if (c->vstage) cudaFree(c->vstage);
+    delete c;
+    return FMTP_OK;
+}
+
+size_t fmtp_workspace_bytes(const fmtp_ctx *c) { return c ? c->ws_need : 0; }
+int fmtp_last_cuda_error(const fmtp_ctx *c) { return c ? c->last_cuda : 0; }
+long long fmtp_launch_count(const fmtp_ctx *c) { return c ? c->launches : 0; }
+
+int fmtp_set_workspace(fmtp_ctx *c, void *dev, size_t bytes) {
+    if (!c || !dev) return FMTP_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(dev) & 255u) != 0) return FMTP_EINVAL;
+    if (bytes < c->ws_need) return FMTP_ENOMEM;
+    c->ws = static_cast<unsigned char *>(dev);
+    c->ws_bytes = bytes;
+    layout(c, c->ws);
+    cudaError_t e = cudaMemset(dev, 0, c->ws_need);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    // rotary table: angle(pos, i) = pos * theta^(-2i/dh), evaluated in double, stored as fp32
+    const fmtp_shape &sh = c->shape;
+    const int half = sh.head_dim / 2;
+    std::vector<float> cs((size_t)sh.max_ctx * half), sn((size_t)sh.max_ctx * half);
+    for (int i = 0; i < half; ++i) {
+        double inv = std::pow((double)sh.rope_theta, -2.0 * i / sh.head_dim);
+        for (int pos = 0; pos < sh.max_ctx; ++pos) {
+            double a = (double)pos * inv;
+            cs[(size_t)pos * half + i] = (float)std::cos(a);
+            sn[(size_t)pos * half + i] = (float)std::sin(a);
+        }
+    }
+    e = cudaMemcpy(const_cast<float *>(c->s.rope_cos), cs.data(), cs.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(const_cast<float *>(c->s.rope_sin), sn.data(), sn.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    return FMTP_OK;
+}
+
+int fastmtp_draft(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_last, const int32_t *tok_last,
+                  const fmtp_kv *kv, int B, int K, const int32_t *subset, int N, int32_t *out_drafts,
+                  fmtp_bf16 *out_h, float *out_logits, uint32_t *dev_status, void *stream) {
+    if (!c || !w || !h_last || !tok_last || !kv || !out_drafts) return FMTP_EINVAL;
+    if (!c->ws) return FMTP_ENOMEM;
+    if (B <= 0 || K <= 0) return FMTP_EINVAL;
+    if (B > c->shape.max_rows || K > c->shape.max_K) return FMTP_ESHAPE;
+    if (subset && (N <= 0 || N > c->shape.vocab)) return FMTP_EINVAL;
+    if (!w->embed || !w->lm_head || !w->g_hnorm || !w->g_enorm || !w->w_proj || !w->g_final) return FMTP_EINVAL;
+    if (!aligned16(w->embed) || !aligned16(w->lm_head) || !aligned16(w->g_hnorm) || !aligned16(w->g_enorm) ||
+        !aligned16(w->w_proj) || !aligned16(w->g_final) || !aligned16(h_last) || !layer_ok(w->layer) || !kv_ok(*kv))
+        return FMTP_EINVAL;
+    MegaParams p;
+    int rc = configure(c, p, 0, B, 1);
+    if (rc) return rc;
+    p.K = K;
+    p.N = subset ? N : c->shape.vocab;
+    p.ids = subset;
+    p.h_last = h_last;
+    p.tokens = tok_last;
+    p.out_tokens = out_drafts;
+    p.out_h = out_h;
+    p.out_logits_f32 = out_logits;
+    p.user_status = dev_status;
+    p.embed = w->embed; p.lm_head = w->lm_head; p.g_hnorm = w->g_hnorm; p.g_enorm = w->g_enorm;
+    p.w_proj = w->w_proj; p.g_final = w->g_final;
+    set_layer(p.layers[0], w->layer);
+    set_kv(p.kvs[0], *kv);
+    return launch_mega(c, p, static_cast<cudaStream_t>(stream));
+}
+
+int fastmtp_draft_host(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_host, const int32_t *tok_host,
+                       const fmtp_kv *kv, int B, int K, const int32_t *subset, int N, int32_t *out_host,
+                       void *stream) {
+    if (!c || !h_host || !tok_host || !out_host) return FMTP_EINVAL;
+    if (!c->ws) return FMTP_ENOMEM;
+    if (B <= 0 || K <= 0) return FMTP_EINVAL;
+    if (B > c->shape.max_rows || K > c->shape.max_K) return FMTP_ESHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t hb = (size_t)B * c->shape.d * 2, tb = (size_t)B * 4, ob = (size_t)B * K * 4;
+    unsigned char *pin = static_cast<unsigned char *>(c->pinned);
+    std::memcpy(pin, h_host, hb);
+    std::memcpy(pin + hb, tok_host, tb);
+    cudaError_t e = cudaMemcpyAsync(c->st_h, pin, hb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(c->st_tok, pin + hb, tb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->st_status, 0, 4, st);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    int rc = fastmtp_draft(c, w, c->st_h, c->st_tok, kv, B, K, subset, N, c->st_out, nullptr, nullptr, c->st_status, st);
+    if (rc) return rc;
+    unsigned char *po = pin + align_up(hb + tb, 16);
+    e = cudaMemcpyAsync(po, c->st_out, ob, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(po + ob, c->st_status, 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    std::memcpy(out_host, po, ob);
+    uint32_t stw;
+    std::memcpy(&stw, po + ob, 4);
+    return status_to_code(stw);
+}
+
+int fastmtp_verify_accept(fmtp_ctx *c, const fmtp_bf16 *logits, const int32_t *drafts, int B, int K, int V,
+                          int32_t *out_accept, int32_t *out_bonus, int32_t *out_argmax, uint32_t *dev_status,
+                          void *stream) {
+    if (!c || !logits || !out_accept || !out_bonus || (K > 0 && !drafts)) return FMTP_EINVAL;
+    if (!c->ws) return FMTP_ENOMEM;
+    if (B <= 0 || K < 0 || V <= 0) return FMTP_EINVAL;
+    if ((long long)B * (K + 1) > kVerifyMaxRows) return FMTP_ESHAPE;
+    int err = verify_launch(logits, drafts, B, K, V, out_accept, out_bonus, out_argmax, c->vkeys, c->vcounter,
+                            c->s.status, dev_status, c->n_sm, static_cast<cudaStream_t>(stream));
+    if (err) return cuda_fail(c, (cudaError_t)err);
+    c->launches++;
+    return FMTP_OK;
+}
+
+int fastmtp_verify_accept_host(fmtp_ctx *c, const fmtp_bf16 *logits_host, const int32_t *drafts_host, int B, int K,
+                               int V, int32_t *accept_host, int32_t *bonus_host, void *stream) {
+    if (!c || !logits_host || !accept_host || !bonus_host || (K > 0 && !drafts_host)) return FMTP_EINVAL;
+    if (!c->ws) return FMTP_ENOMEM;
+    if (B <= 0 || K < 0 || V <= 0) return FMTP_EINVAL;
+    if ((long long)B * (K + 1) > kVerifyMaxRows) return FMTP_ESHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    size_t lb = (size_t)B * (K + 1) * V * 2, db = (size_t)B * K * 4;
+    size_t need = align_up(lb, 256) + align_up(db + 16, 256);
+    cudaError_t e = cudaSuccess;
+    if (need > c->vstage_bytes) {   // the one device allocation this library makes (grow-only, freed in destroy)
+        if (c->vstage) cudaFree(c->vstage);
+        c->vstage = nullptr;
+        c->vstage_bytes = 0;
+        e = cudaMalloc(&c->vstage, need);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        c->vstage_bytes = need;
+    }
+    unsigned char *dv = static_cast<unsigned char *>(c->vstage);
+    int32_t *ddr = reinterpret_cast<int32_t *>(dv + align_up(lb, 256));
+    e = cudaMemcpyAsync(dv, logits_host, lb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && db) e = cudaMemcpyAsync(ddr, drafts_host, db, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->st_status, 0, 4, st);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    int32_t *dacc = c->st_out, *dbon = c->st_out + kVerifyMaxRows;
+    int rc = fastmtp_verify_accept(c, reinterpret_cast<const fmtp_bf16 *>(dv), ddr, B, K, V, dacc, dbon, nullptr,
+                                   c->st_status, st);
+    if (rc) return rc;
+    unsigned char *pin = static_cast<unsigned char *>(c->pinned);
+    e = cudaMemcpyAsync(pin, dacc, (size_t)B * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(pin + (size_t)B * 4, dbon, (size_t)B * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(pin + (size_t)B * 8, c->st_status, 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    std::memcpy(accept_host, pin, (size_t)B * 4);
+    std::memcpy(bonus_host, pin + (size_t)B * 4, (size_t)B * 4);
+    uint32_t stw;
+    std::memcpy(&stw, pin + (size_t)B * 8, 4);
+    return status_to_code(stw);
+}
+
+int fastmtp_target_step(fmtp_ctx *c, const fmtp_target_w *w, const int32_t *tokens, const fmtp_kv *kvs, int B, int M,
+                        fmtp_bf16 *out_h, fmtp_bf16 *out_logits, int32_t *out_argmax, uint32_t *dev_status,
+                        void *stream) {
+    if (!c || !w || !tokens || !kvs) return FMTP_EINVAL;
+    if (!c->ws) return FMTP_ENOMEM;
+    if (B <= 0 || M <= 0) return FMTP_EINVAL;
+    const int nl = c->shape.n_layers;
+    if (nl <= 0 || (long long)B * M > c->shape.max_rows) return FMTP_ESHAPE;
+    if (!w->embed || !w->lm_head || !w->g_final || !w->layers) return FMTP_EINVAL;
+    if (!aligned16(w->embed) || !aligned16(w->lm_head) || !aligned16(w->g_final)) return FMTP_EINVAL;
+    for (int l = 0; l < nl; ++l) if (!layer_ok(w->layers[l]) || !kv_ok(kvs[l])) return FMTP_EINVAL;
+    MegaParams p;
+    int rc = configure(c, p, 1, B, M);
+    if (rc) return rc;
+    p.K = 1;
+    p.n_layers = nl;
+    p.N = c->shape.vocab;
+    p.ids = nullptr;
+    p.tokens = tokens;
+    p.out_tokens = out_argmax;
+    p.out_h = out_h;
+    p.out_logits_bf16 = out_logits;
+    p.user_status = dev_status;
+    p.embed = w->embed; p.lm_head = w->lm_head; p.g_final = w->g_final;
+    for (int l = 0; l < nl; ++l) { set_layer(p.layers[l], w->layers[l]); set_kv(p.kvs[l], kvs[l]); }
+    return launch_mega(c, p, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,96 @@
+// Parameter block and launch interface of the persistent decoder kernel.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace fmtp {
+
+constexpr int kMaxLayers = 64;
+constexpr int kMaxRows = 8;          // activation rows (batch x rows-per-sequence) per launch
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kThreads = kConsumerThreads + 32;   // + one producer warp
+constexpr int kTileRows = 32;        // weight rows per pipeline stage (two 16-row MMA tiles)
+constexpr int kAttnChunk = 128;      // context tokens per attention work item
+constexpr int kMaxStages = 8;
+
+typedef uint16_t bf16_t;
+
+struct LayerPtrs {
+    const bf16_t *g_in, *wq, *wk, *wv, *wo, *g_post, *w_gate, *w_up, *w_down;
+};
+struct KvPtrs {
+    bf16_t *k_pages, *v_pages;
+    const int32_t *block_table, *seq_lens;
+    int32_t num_pages, max_pages;
+};
+
+// Global scratch carved out of the caller's workspace. "hi/lo" buffers hold an fp32 value as
+// two bf16 numbers (hi = bf16(x), lo = bf16(x - hi)) in two separate row-major arrays.
+struct Scratch {
+    float *x0, *x1;                   // [R][d] residual stream before / after attention
+    float *qkv;                       // [R][qdim + 2 kvdim]
+    bf16_t *actD_hi, *actD_lo;        // [R][dp]  input of QKV            (x * g_in, unnormalised)
+    bf16_t *actP_hi, *actP_lo;        // [R][dp]  input of gate/up        (x * g_post)
+    bf16_t *actH_hi, *actH_lo;        // [R][dp]  input of the head       (x * g_final)
+    bf16_t *actR_hi, *actR_lo;        // [R][dp]  recursed hidden state   (x * g_final * g_hnorm)
+    bf16_t *actO_hi, *actO_lo;        // [R][qp]  attention output
+    bf16_t *actF_hi, *actF_lo;        // [R][Fp]  SwiGLU activation
+    float *ssA, *ssB, *ssC, *ssD;     // [grid][8] per-CTA partial sums of squares
+    float *att_part;                  // [R][Hq][max_chunks][dh + 2] (o, m, l) per context chunk
+    uint32_t *att_cnt;                // [B_max][Hkv] arrival counters
+    unsigned long long *keys;         // [max_K or 1][8] argmax keys
+    const float *rope_cos, *rope_sin; // [max_ctx][dh/2]
+    uint32_t *barrier;                // grid barrier counter
+    uint32_t *abort_flag;             // set when a bounded wait gave up
+    uint32_t *status;                 // internal status word (OR of FMTP_DEV_*), merged to the caller's
+};
+
+struct MegaParams {
+    // geometry
+    int d, Hq, Hkv, dh, F, V, qdim, kvdim, page;
+    int dp, qp, Fp;                   // padded row lengths of the hi/lo buffers (multiples of 32)
+    float eps;
+    int KC;                           // k elements per pipeline stage
+    int n_stages, stage_bytes, row_stride;  // ring geometry (bytes)
+    int scratch_smem;                 // bytes of the per-phase shared scratch region
+    int stage_F_in_smem;              // 1: the ffn-length activation is staged in shared memory
+    int max_chunks;                   // capacity of att_part's chunk dimension
+    int max_ctx;                      // rows of the rotary table
+    // call
+    int mode;                         // 0: MTP draft, 1: target step
+    int B, M, R;                      // sequences, rows per sequence, R = B*M
+    int K;                            // draft steps (mode 0)
+    int n_layers;                     // mode 1
+    int N;                            // head rows (subset size or V)
+    const int32_t *ids;               // subset or NULL
+    const bf16_t *h_last;             // [B][d] (mode 0)
+    const int32_t *tokens;            // mode 0: tok_last [B]; mode 1: [B][M]
+    int32_t *out_tokens;              // mode 0: drafts [B][K]; mode 1: argmax [B][M] or NULL
+    bf16_t *out_h;                    // mode 0: [B][K][d]; mode 1: [B][M][d]; or NULL
+    float *out_logits_f32;            // mode 0 debug [B][K][N] or NULL
+    bf16_t *out_logits_bf16;          // mode 1 [R][V] or NULL
+    uint32_t *user_status;            // caller's status word or NULL
+    // weights
+    const bf16_t *embed, *lm_head, *g_hnorm, *g_enorm, *w_proj, *g_final;
+    LayerPtrs layers[kMaxLayers];
+    KvPtrs kvs[kMaxLayers];
+    Scratch s;
+};
+
+// Shared-memory bytes the kernel needs for these parameters.
+size_t mega_smem_bytes(const MegaParams &p);
+// Shared memory used besides the per-phase scratch and the ring, for R activation rows.
+size_t mega_fixed_smem(int R);
+// Cooperative launch on `stream` with `grid` CTAs (one per SM). Returns the cudaError_t.
+int mega_launch(const MegaParams &p, int grid, cudaStream_t stream);
+// Largest co-resident grid for this shared-memory footprint on the current device.
+int mega_max_grid(size_t smem_bytes, int *err);
+
+// Verification kernel (verify.cu).
+int verify_launch(const bf16_t *logits, const int32_t *drafts, int B, int K, int V,
+                  int32_t *accept_len, int32_t *bonus, int32_t *out_argmax,
+                  unsigned long long *keys, uint32_t *counter, uint32_t *status, uint32_t *user_status,
+                  int n_sm, cudaStream_t stream);
+
+}  // namespace fmtp

@@ -1,0 +1,130 @@
+// Greedy verification: full-vocabulary argmax of every target-logit row, then the longest
+// accepted draft prefix and the bonus token (Sec. 2.3 "Verification phase" of the paper).
+//
+// HBM-bound read-once scan. Each CTA scans a slice of one row with 128-bit streaming loads
+// (8 independent loads in flight per thread), reduces (value, id) to one 64-bit key -- highest
+// value first, then lowest token id, NaN never wins -- and publishes it with atomicMax (an
+// integer maximum: order independent, so the result is reproducible). The CTA that arrives last
+// turns the per-row winners into accept_len / bonus and clears the scratch for the next call.
+#include "mega.cuh"
+#include "ptx.cuh"
+
+namespace fmtp {
+
+namespace {
+
+constexpr int kVThreads = 256;
+constexpr int kVecPerThread = 8;                                  // 16-byte loads in flight per thread
+constexpr int kSlice = kVThreads * kVecPerThread * 8;             // bf16 elements per CTA (16384)
+constexpr int kNoIdx = 0x7fffffff;
+
+__device__ __forceinline__ void consider(float v, int i, float &best, int &idx) {
+    // strict '>' keeps the earliest (lowest) id among equal values; the second clause admits the
+    // first non-NaN value even if it is -inf
+    if (v > best || (idx == kNoIdx && v == v)) { best = v; idx = i; }
+}
+
+__global__ void __launch_bounds__(kVThreads) verify_kernel(const bf16_t *__restrict__ logits,
+                                                            const int32_t *__restrict__ drafts, int B, int K, int V,
+                                                            int slices_per_row, int32_t *accept_len, int32_t *bonus,
+                                                            int32_t *out_argmax, unsigned long long *keys,
+                                                            uint32_t *counter, uint32_t *status,
+                                                            uint32_t *user_status) {
+    const int row = blockIdx.x / slices_per_row;
+    const int slice = blockIdx.x - row * slices_per_row;
+    const bf16_t *src = logits + (size_t)row * V;
+    const int lo = slice * kSlice;
+    const int hi = min(V, lo + kSlice);
+    float best = -INFINITY;
+    int idx = kNoIdx;
+
+    const bool vec_ok = ((reinterpret_cast<uintptr_t>(src) & 15u) == 0);
+    if (vec_ok) {
+        const int nvec = (hi - lo) >> 3;
+        uint4 v[kVecPerThread];
+#pragma unroll
+        for (int j = 0; j < kVecPerThread; ++j) {
+            int vi = threadIdx.x + j * kVThreads;
+            v[j] = (vi < nvec) ? ldnc128(src + lo + (size_t)vi * 8) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int j = 0; j < kVecPerThread; ++j) {
+            int vi = threadIdx.x + j * kVThreads;
+            if (vi < nvec) {
+                int i0 = lo + vi * 8;
+                uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    consider(bf16lo_f32(w[q]), i0 + 2 * q, best, idx);
+                    consider(bf16hi_f32(w[q]), i0 + 2 * q + 1, best, idx);
+                }
+            }
+        }
+        for (int i = lo + (nvec << 3) + threadIdx.x; i < hi; i += kVThreads)   // ragged tail
+            consider(bf16bits_f32(src[i]), i, best, idx);
+    } else {
+        for (int i = lo + threadIdx.x; i < hi; i += kVThreads) consider(bf16bits_f32(src[i]), i, best, idx);
+    }
+
+    unsigned long long key = (idx == kNoIdx) ? 0ull : argmax_key(best, (uint32_t)idx);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+        key = other > key ? other : key;
+    }
+    __shared__ unsigned long long wkey[kVThreads / 32];
+    __shared__ int is_last;
+    if ((threadIdx.x & 31) == 0) wkey[threadIdx.x >> 5] = key;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long m = 0ull;
+        for (int w = 0; w < kVThreads / 32; ++w) m = wkey[w] > m ? wkey[w] : m;
+        if (m != 0ull) atomicMax(keys + row, m);
+        __threadfence();
+        uint32_t old = atomicAdd(counter, 1u);
+        is_last = (old == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+
+    // ---- last CTA: accept lengths
+    __threadfence();
+    const int M = K + 1;
+    for (int b = threadIdx.x; b < B; b += kVThreads) {
+        int a = 0;
+        bool open = true;
+        int bon = 0;
+        for (int j = 0; j < M; ++j) {
+            unsigned long long k = ldcg_u64(keys + (size_t)b * M + j);
+            int g = 0;
+            if ((k >> 32) == 0ull) { atomicOr(status, 0x10u); if (user_status) atomicOr(user_status, 0x10u); }
+            else g = (int)argmax_key_id(k);
+            if (out_argmax) out_argmax[(size_t)b * M + j] = g;
+            if (open) {
+                bon = g;
+                if (j < K && drafts[(size_t)b * K + j] == g) a = j + 1;
+                else open = false;
+            }
+        }
+        accept_len[b] = a;
+        bonus[b] = bon;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < B * M; i += kVThreads) keys[i] = 0ull;
+    if (threadIdx.x == 0) *counter = 0u;
+}
+
+}  // namespace
+
+int verify_launch(const bf16_t *logits, const int32_t *drafts, int B, int K, int V, int32_t *accept_len,
+                  int32_t *bonus, int32_t *out_argmax, unsigned long long *keys, uint32_t *counter,
+                  uint32_t *status, uint32_t *user_status, int n_sm, cudaStream_t stream) {
+    (void)n_sm;
+    int slices = (V + kSlice - 1) / kSlice;
+    int grid = B * (K + 1) * slices;
+    verify_kernel<<<grid, kVThreads, 0, stream>>>(logits, drafts, B, K, V, slices, accept_len, bonus, out_argmax,
+                                                  keys, counter, status, user_status);
+    return (int)cudaGetLastError();
+}
+
+}  // namespace fmtp
