@@ -33,7 +33,7 @@ namespace {
 
 constexpr uint32_t kDevBadToken = 0x1u, kDevBadPage = 0x2u, kDevBadPos = 0x4u, kDevTimeout = 0x8u,
                    kDevAllNan = 0x10u;
-constexpr uint32_t kPollLimit = 1u << 24;   // polls before a wait gives up (each >= ~100 ns)
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait gives up after 2 s
 
 enum Kind { PROJ = 0, QKV = 1, OPROJ = 2, GATEUP = 3, DOWN = 4, HEAD = 5 };
 
@@ -75,11 +75,17 @@ __device__ void do_abort(const Cta &c) {
 // Bounded wait on an mbarrier phase. Returns false (and raises the abort flag) on timeout.
 __device__ bool wait_bar(const Cta &c, uint64_t *bar, uint32_t parity) {
     if (aborted(c)) return false;
-    for (uint32_t n = 0; n < kPollLimit; ++n) {
+    unsigned long long t0 = 0;
+    for (uint32_t n = 0;; ++n) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((n & 1023u) == 1023u && ldcg_u32(c.p->s.abort_flag) != 0) {
-            c.misc->aborted = 1;
-            return false;
+        if ((n & 255u) == 255u) {
+            if (ldcg_u32(c.p->s.abort_flag) != 0) {
+                c.misc->aborted = 1;
+                return false;
+            }
+            unsigned long long now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) break;
         }
     }
     do_abort(c);
@@ -95,9 +101,14 @@ __device__ void grid_barrier(Cta &c) {
         atomicAdd(c.p->s.barrier, 1u);
         if (!aborted(c)) {
             uint32_t n = 0;
+            unsigned long long t0 = 0;
             while ((int32_t)(ld_acquire_u32(c.p->s.barrier) - c.bar_target) < 0) {
-                if (++n > kPollLimit) { do_abort(c); break; }
-                if ((n & 255u) == 255u && ldcg_u32(c.p->s.abort_flag) != 0) { c.misc->aborted = 1; break; }
+                if ((++n & 255u) == 255u) {
+                    if (ldcg_u32(c.p->s.abort_flag) != 0) { c.misc->aborted = 1; break; }
+                    unsigned long long now = global_timer_ns();
+                    if (t0 == 0) t0 = now;
+                    else if (now - t0 > kWaitLimitNs) { do_abort(c); break; }
+                }
                 __nanosleep(32);
             }
         }
@@ -653,7 +664,9 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
             for (uint32_t s = first; s < issued; ++s) {
                 uint64_t *bar = &c.misc->full[s % p.n_stages];
                 uint32_t parity = (s / p.n_stages) & 1u;
-                for (uint32_t n = 0; n < kPollLimit && !mbar_try_wait(bar, parity); ++n) {}
+                unsigned long long t0 = global_timer_ns();
+                for (uint32_t n = 0; !mbar_try_wait(bar, parity); ++n)
+                    if ((n & 255u) == 255u && global_timer_ns() - t0 > kWaitLimitNs) break;
             }
         }
         return;

@@ -1,0 +1,235 @@
+"""GPU parity of fastmtp_target_step and of the speculative loop built from the three calls."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fastmtp_oracle as O
+from paper_2509_18362_b200 import inputs as I
+from tests.gpu_util import GAP_TOL, close, copy_kv, ids_match
+
+pytestmark = pytest.mark.gpu
+
+
+def _binding():
+    from paper_2509_18362_b200 import binding
+    return binding
+
+
+class GpuTarget:
+    """Device copies of a target model and its per-layer caches, stepped through the C ABI."""
+
+    def __init__(self, shape, Wt, kvs, max_ctx):
+        Bd = _binding()
+        self.Bd, self.shape = Bd, shape
+        self.ctx = Bd.Context(shape, max_rows=8, max_K=8, max_ctx=max_ctx)
+        self.dW = Bd.to_device(Wt)
+        self.w, self._keep = Bd.target_w(self.dW)
+        self.dkvs = [Bd.to_device(copy_kv(kv)) for kv in kvs]
+
+    def step(self, tokens, want_logits=True):
+        Bd, s = self.Bd, self.shape
+        tokens = np.asarray(tokens, dtype=np.int32)
+        B, M = tokens.shape
+        out_h = torch.zeros((B, M, s.d), dtype=torch.bfloat16, device="cuda")
+        out_l = torch.zeros((B, M, s.vocab), dtype=torch.bfloat16, device="cuda") if want_logits else None
+        out_a = torch.full((B, M), -1, dtype=torch.int32, device="cuda")
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        self.ctx.fastmtp_target_step(self.w, torch.from_numpy(tokens).cuda(), [Bd.kv(k) for k in self.dkvs], B, M,
+                                     out_h, out_l, out_a, st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        return out_h, out_l, out_a.cpu().numpy()
+
+    def advance(self, n):
+        for k in self.dkvs:
+            k["seq_lens"] += torch.as_tensor(n, dtype=torch.int32, device="cuda")
+
+    def close(self):
+        self.ctx.close()
+
+
+def _bf16_gap(row):
+    """Top-2 gap of an oracle logit row, less one bf16 spacing at the winner's magnitude: the
+    greedy choice is made on bf16-rounded logits, so two candidates closer than the tolerance
+    plus one spacing can legitimately round to a tie (lowest id) on one side only."""
+    top2 = np.partition(row, row.shape[0] - 2)[-2:]
+    ulp = 2.0 ** (np.floor(np.log2(max(abs(top2[1]), 1e-30))) - 7)
+    return float(top2[1] - top2[0] - ulp)
+
+
+def _gaps(logits64):
+    """Top-2 gap of every row of oracle logits after bf16 rounding (the precision the greedy
+    choice is made in at the boundary)."""
+    flat = logits64.reshape(-1, logits64.shape[-1])
+    toks, gaps = [], []
+    for row in flat:
+        t, _ = O.argmax_token(O.round_bf16(row))
+        toks.append(t)
+        gaps.append(_bf16_gap(row))
+    return np.array(toks), np.array(gaps)
+
+
+@pytest.mark.parametrize("n_layers", [1, 3])
+def test_target_step_prefill_decode_verify(n_layers):
+    shape = I.TINY.with_layers(n_layers)
+    Wt = I.target_weights(shape, 300 + n_layers)
+    B = 2
+    kvs = [I.empty_paged_kv(shape, B, 48, 310 + l) for l in range(n_layers)]
+    okvs = [copy_kv(kv) for kv in kvs]
+    gpu = GpuTarget(shape, Wt, kvs, 64)
+    toks = I.token_ids(320, (B, 11), shape.vocab)
+    # rows per call: 4 + 4 + 3 (prefill chunks), then 1 (decode), then 4 (verify-shaped)
+    for lo, hi in [(0, 4), (4, 8), (8, 11)]:
+        h, l, a = gpu.step(toks[:, lo:hi])
+        rh, rl = O.target_forward(shape, Wt, toks[:, lo:hi], okvs)
+        close(h.float().cpu().numpy(), rh, f"target h rows {lo}:{hi}")
+        close(l.float().cpu().numpy(), rl, f"target logits rows {lo}:{hi}")
+        rt, gap = _gaps(rl)
+        ids_match(a, rt, gap, "target argmax")
+        gpu.advance(hi - lo)
+        for kv in okvs:
+            kv["seq_lens"] += hi - lo
+    for M in (1, 4):
+        t = I.token_ids(330 + M, (B, M), shape.vocab)
+        h, l, a = gpu.step(t)
+        rh, rl = O.target_forward(shape, Wt, t, okvs)
+        close(h.float().cpu().numpy(), rh, f"target h M={M}")
+        close(l.float().cpu().numpy(), rl, f"target logits M={M}")
+        # the kernel's own argmax equals the argmax of the logits it wrote (decided on bf16 values)
+        own = [O.argmax_token(O.bf16_to_f64(row))[0] for row in
+               _binding().bf16_bits(l).reshape(-1, shape.vocab)]
+        assert np.array_equal(a.ravel(), np.array(own))
+        gpu.advance(M)
+        for kv in okvs:
+            kv["seq_lens"] += M
+    for l in range(n_layers):
+        close(O.bf16_to_f64(_binding().bf16_bits(gpu.dkvs[l]["k_pages"])), O.bf16_to_f64(okvs[l]["k_pages"]),
+              f"layer {l} K cache")
+    gpu.close()
+
+
+def test_rows_do_not_depend_on_rows_per_call():
+    """A position's hidden state and logits are bit-identical whether it is scored alone (M=1)
+    or as one of several rows (M=4): the property that makes verification lossless."""
+    shape = I.TINY.with_layers(2)
+    Wt = I.target_weights(shape, 401)
+    kvs = [I.empty_paged_kv(shape, 1, 48, 410 + l) for l in range(2)]
+    toks = I.token_ids(420, (1, 8), shape.vocab)
+    a = GpuTarget(shape, Wt, kvs, 64)
+    hs, ls = [], []
+    for j in range(8):
+        h, l, _ = a.step(toks[:, j:j + 1])
+        a.advance(1)
+        hs.append(h)
+        ls.append(l)
+    a.close()
+    b = GpuTarget(shape, Wt, kvs, 64)
+    h4a, l4a, _ = b.step(toks[:, 0:4])
+    b.advance(4)
+    h4b, l4b, _ = b.step(toks[:, 4:8])
+    b.close()
+    one_h = torch.cat(hs, dim=1)
+    one_l = torch.cat(ls, dim=1)
+    assert torch.equal(one_h, torch.cat([h4a, h4b], dim=1))
+    assert torch.equal(one_l, torch.cat([l4a, l4b], dim=1))
+
+
+def _gpu_greedy(gpu, prompt, n_new):
+    P = len(prompt)
+    last = None
+    for lo in range(0, P, 8):
+        _, _, a = gpu.step(np.array([prompt[lo:lo + 8]]), want_logits=False)
+        gpu.advance(len(prompt[lo:lo + 8]))
+        last = int(a[0, -1])
+    out = [last]
+    while len(out) < n_new:
+        _, _, a = gpu.step(np.array([[out[-1]]]), want_logits=False)
+        gpu.advance(1)
+        out.append(int(a[0, 0]))
+    return out
+
+
+def test_speculative_loop_is_token_identical_to_greedy_on_gpu():
+    """Draft with the MTP head, score [last, drafts] with the target in one call, accept with
+    fastmtp_verify_accept: the emitted sequence equals plain greedy decoding by the same
+    library; and the first tokens agree with the oracle's greedy run up to near ties."""
+    Bd = _binding()
+    shape = I.TINY.with_layers(2)
+    K, n_new = 3, 40
+    Wt = I.target_weights(shape, 501)
+    Wm = I.mtp_weights(shape, 502, embed=Wt["embed"], lm_head=Wt["lm_head"])
+    prompt = [int(t) for t in I.token_ids(503, (19,), shape.vocab)]
+    ids = I.subset_uniform(shape.vocab, 1024, 504)
+    mk = lambda: [I.empty_paged_kv(shape, 1, 128, 510 + l) for l in range(2)]
+
+    g = GpuTarget(shape, Wt, mk(), 128)
+    ref = _gpu_greedy(g, prompt, n_new + K + 1)
+    g.close()
+
+    gpu = GpuTarget(shape, Wt, mk(), 128)
+    dWm = Bd.to_device(Wm)
+    wm = Bd.mtp_w(dWm)
+    mkv = Bd.to_device(I.empty_paged_kv(shape, 1, 128, 520))
+    dids = torch.from_numpy(ids).cuda()
+    # prefill the target; feed the MTP cache with pairs (h_j, t_{j+1}) one position per call
+    hs = []
+    last = None
+    for lo in range(0, len(prompt), 8):
+        h, _, a = gpu.step(np.array([prompt[lo:lo + 8]]), want_logits=False)
+        gpu.advance(len(prompt[lo:lo + 8]))
+        hs.append(h)
+        last = int(a[0, -1])
+    hP = torch.cat(hs, dim=1)[0]
+    out = [last]
+    pend_h = hP
+    pend_t = prompt[1:] + [last]
+    drafts_d = torch.zeros((1, K), dtype=torch.int32, device="cuda")
+    accepted = []
+    rnd = 0
+    while len(out) < n_new:
+        for m in range(len(pend_t)):
+            steps = K if m == len(pend_t) - 1 else 1
+            gpu.ctx.fastmtp_draft(wm, pend_h[m:m + 1].contiguous(),
+                                  torch.tensor([pend_t[m]], dtype=torch.int32, device="cuda"),
+                                  Bd.kv(mkv), 1, steps, dids, drafts_d)
+            mkv["seq_lens"] += 1
+        torch.cuda.synchronize()
+        drafts = [int(t) for t in drafts_d.cpu().numpy()[0]]
+        if rnd % 2 == 1:
+            # every other round: inject drafts that are right for a planted number of positions
+            e = len(out)
+            n_ok = (rnd // 2) % (K + 1)
+            good = ref[e:e + K]
+            drafts = list(good[:n_ok]) + [(t + 1) % shape.vocab for t in good[n_ok:]]
+        row = np.array([[out[-1]] + drafts], dtype=np.int32)
+        h, logits, _ = gpu.step(row)
+        acc = torch.zeros(1, dtype=torch.int32, device="cuda")
+        bon = torch.zeros(1, dtype=torch.int32, device="cuda")
+        gpu.ctx.fastmtp_verify_accept(logits, torch.tensor([drafts], dtype=torch.int32, device="cuda"), 1, K,
+                                      shape.vocab, acc, bon)
+        torch.cuda.synchronize()
+        a, bonus = int(acc.item()), int(bon.item())
+        gpu.advance(a + 1)
+        new = drafts[:a] + [bonus]
+        out.extend(new)
+        accepted.append(a)
+        pend_h = h[0, :a + 1]
+        pend_t = new
+        rnd += 1
+    gpu.close()
+    assert out[:n_new] == ref[:n_new]
+    assert {0, 1, 2, 3} <= set(accepted)
+
+    # oracle greedy on the first tokens, teacher-forced on near ties
+    okvs = mk()
+    _, lg = O.target_forward(shape, Wt, np.array([prompt]), okvs)
+    for kv in okvs:
+        kv["seq_lens"][0] = len(prompt)
+    row = lg[0, -1]
+    for i in range(12):
+        t, _ = O.argmax_token(O.round_bf16(row))
+        assert t == ref[i] or _bf16_gap(row) < GAP_TOL, f"token {i}: oracle {t}, gpu {ref[i]}"
+        _, lg = O.target_forward(shape, Wt, np.array([[ref[i]]]), okvs)
+        for kv in okvs:
+            kv["seq_lens"][0] += 1
+        row = lg[0, 0]
