@@ -1,0 +1,362 @@
+"""Benchmark of the FastMTP draft / verify hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--batch B] [--subset N] [--ctx L] [--draft-steps K] [--subset-kind uniform|zipf]
+
+One step = one pass of the hot path over one batch of synthetic input: fastmtp_draft (the K
+recursive MTP steps with the compressed-vocabulary head, one kernel launch) followed by
+fastmtp_verify_accept on target logits [B, K+1, V]. The default workload is the 7B-class head at
+batch 1 (d=3584, 28/4 heads of 128, ffn 18944, V=152064, subset 32768, 2048 cached tokens, K=3).
+
+Prints one JSON line (rank 0). `value` is draft tokens per second with every input resident in
+HBM; `e2e` is the same through the *_host entry points (pinned host buffers in, results out).
+With --gpus N > 1 (launched under torch.distributed.run) every rank runs an independent replica
+on its own sequences: sequences are the unit the path shards by, and no data crosses GPUs.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--subset", type=int, default=32768, help="compressed vocabulary size (0 = full vocabulary)")
+    ap.add_argument("--subset-kind", default="uniform", choices=["uniform", "zipf"])
+    ap.add_argument("--ctx", type=int, default=2048, help="cached context tokens per sequence")
+    ap.add_argument("--draft-steps", type=int, default=3)
+    ap.add_argument("--shape", default="7b", choices=["7b", "tiny"])
+    ap.add_argument("--seed", type=int, default=1234)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def algorithmic_bytes_per_draft_step(s, B, N, ctx_lens, k):
+    """Bytes one MTP draft step must move: every weight of the head once (projection, decoder
+    layer, the N gathered output-head rows), the cached K/V of every sequence up to the current
+    position, the embedding rows and the norm gains (bf16 = 2 bytes)."""
+    qd, kvd = s.n_q_heads * s.head_dim, s.n_kv_heads * s.head_dim
+    weights = 2 * s.d * s.d + s.d * (qd + 2 * kvd) + qd * s.d + 3 * s.d * s.ffn + N * s.d
+    kv = sum(2 * kvd * (int(L) + k) for L in ctx_lens)          # K and V entries
+    return 2 * weights + 2 * kv + B * 2 * s.d + 10 * s.d
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = [r for t, r in self.rows if t0 - 0.05 <= t <= t1 + 0.15] or [r for _, r in self.rows]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def make_inputs(a, rank):
+    from paper_2509_18362_b200 import inputs as I
+    s = I.QWEN7B if a.shape == "7b" else I.TINY
+    seed = a.seed + 1000 * rank
+    N = a.subset if 0 < a.subset < s.vocab else s.vocab
+    K = a.draft_steps
+    W = I.mtp_weights(s, a.seed)                     # same model on every replica
+    ctx_lens = [a.ctx] * a.batch
+    kv = I.paged_kv(s, ctx_lens, K + 1, seed + 1)
+    h = I.hidden_bf16(seed + 2, (a.batch, s.d))
+    tok = I.token_ids(seed + 3, (a.batch,), s.vocab)
+    if N >= s.vocab:
+        ids = None
+    elif a.subset_kind == "uniform":
+        ids = I.subset_uniform(s.vocab, N, a.seed + 4)
+    else:
+        ids = I.subset_zipf(s.vocab, N, a.seed + 4)
+    vcase = I.verify_case(a.batch, K, s.vocab, seed + 5)
+    return s, N, K, W, kv, h, tok, ids, vcase, ctx_lens
+
+
+def workload_name(a, s, N):
+    return (f"{a.shape} MTP head draft+verify: d={s.d} Hq/Hkv={s.n_q_heads}/{s.n_kv_heads} dh={s.head_dim} "
+            f"ffn={s.ffn} V={s.vocab} subset={N}({a.subset_kind}) ctx={a.ctx} page={s.page_size}")
+
+
+def cpu_oracle_sample(s, W, kv, h, tok, ids, vcase, K, seconds=12.0, max_calls=6):
+    """Times the oracle as it stands on sequence 0 of the workload: repeated K-step drafts plus
+    verification. Returns (draft tokens/s, cores, description)."""
+    from oracle import fastmtp_oracle as O
+    cores = os.cpu_count() or 1
+    try:
+        from threadpoolctl import threadpool_info
+        nt = [p.get("num_threads", 1) for p in threadpool_info()]
+        if nt:
+            cores = max(nt)
+    except Exception:
+        pass
+    kv1 = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in kv.items()}
+    kv1["block_table"] = kv1["block_table"][:1]
+    kv1["seq_lens"] = kv1["seq_lens"][:1]
+    times = []
+    t_begin = time.perf_counter()
+    for _ in range(max_calls):
+        t0 = time.perf_counter()
+        O.draft(s, W, h[:1], tok[:1], kv1, K, ids)
+        O.verify_accept(vcase["logits"][:1], vcase["drafts"][:1])
+        times.append(time.perf_counter() - t0)
+        if time.perf_counter() - t_begin > seconds:
+            break
+    best = min(times)
+    return K / best, cores, f"{len(times)} calls of draft(K={K})+verify on sequence 0 of the workload, best call {best:.3f} s"
+
+
+def run_reference(a):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    s, N, K, W, kv, h, tok, ids, vcase, _ = make_inputs(a, 0)
+    from oracle import fastmtp_oracle as O
+    kv1 = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in kv.items()}
+    kv1["block_table"], kv1["seq_lens"] = kv1["block_table"][:1], kv1["seq_lens"][:1]
+    cores = os.cpu_count() or 1
+
+    K = 1          # bounded sample: one recursive step per timed step keeps long runs to minutes
+
+    def step():
+        O.draft(s, W, h[:1], tok[:1], kv1, K, ids)
+        O.verify_accept(vcase["logits"][:1, :K + 1], vcase["drafts"][:1, :K])
+
+    for _ in range(a.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(a.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = K * a.steps / dt
+    sample = f"each step: oracle draft(K={K}) + verify of {K + 1} logit rows on sequence 0 (batch 1) of the workload"
+    print(json.dumps({
+        "impl": "reference", "metric": "draft_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": a.gpus,
+        "steps": a.steps, "warmup": a.warmup, "ms_per_step": dt / a.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(a, s, N), "batch": 1, "draft_steps": K},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(a):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    import __graft_entry__ as G
+    G.build()
+    from paper_2509_18362_b200 import binding as Bd
+
+    s, N, K, W, kv, h, tok, ids, vcase, ctx_lens = make_inputs(a, rank)
+    B = a.batch
+    ctx = Bd.Context(s, max_rows=max(8, B), max_K=max(8, K), max_ctx=a.ctx + K + 1)
+    dW = Bd.to_device(W)
+    w = Bd.mtp_w(dW)
+    dkv = Bd.to_device(kv)
+    ckv = Bd.kv(dkv)
+    dh, dtok = Bd.bf16_tensor(h), torch.from_numpy(tok).cuda()
+    dids = None if ids is None else torch.from_numpy(ids).cuda()
+    dlogits, ddrafts_v = Bd.bf16_tensor(vcase["logits"]), torch.from_numpy(vcase["drafts"]).cuda()
+    out_d = torch.zeros((B, K), dtype=torch.int32, device="cuda")
+    acc = torch.zeros(B, dtype=torch.int32, device="cuda")
+    bon = torch.zeros(B, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # host-side buffers of the end-to-end leg (pinned)
+    hh = Bd.bf16_tensor(h, "cpu").pin_memory()
+    htok = torch.from_numpy(tok).pin_memory()
+    hlog = Bd.bf16_tensor(vcase["logits"], "cpu").pin_memory()
+    hdv = torch.from_numpy(vcase["drafts"]).pin_memory()
+    hout = torch.zeros((B, K), dtype=torch.int32).pin_memory()
+    hacc = torch.zeros(B, dtype=torch.int32).pin_memory()
+    hbon = torch.zeros(B, dtype=torch.int32).pin_memory()
+
+    def step_dev():
+        ctx.fastmtp_draft(w, dh, dtok, ckv, B, K, dids, out_d, None, None, status)
+        ctx.fastmtp_verify_accept(dlogits, ddrafts_v, B, K, s.vocab, acc, bon, None, status)
+
+    def step_host():
+        ctx.fastmtp_draft_host(w, hh, htok, ckv, B, K, dids, hout)
+        ctx.fastmtp_verify_accept_host(hlog, hdv, B, K, s.vocab, hacc, hbon)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    sampler = ClockSampler(local)
+    for _ in range(max(a.warmup, 3)):
+        step_dev()
+    barrier()
+    sampler.start()
+    time.sleep(0.25)
+    # ---- timed region 1: inputs resident in HBM; one event pair around the whole region and one
+    # around every draft call (the dominant kernel), all on the launching stream
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(a.steps)]
+    launches0 = ctx.launch_count
+    barrier()
+    t_wall0 = time.time()
+    ev[0].record()
+    for i in range(a.steps):
+        kev[i][0].record()
+        ctx.fastmtp_draft(w, dh, dtok, ckv, B, K, dids, out_d, None, None, status)
+        kev[i][1].record()
+        ctx.fastmtp_verify_accept(dlogits, ddrafts_v, B, K, s.vocab, acc, bon, None, status)
+    ev[1].record()
+    barrier()
+    t_wall1 = time.time()
+    launches = ctx.launch_count - launches0
+    clocks = sampler.stop(t_wall0, t_wall1)
+    ms_total = max_over_ranks(ev[0].elapsed_time(ev[1]))
+    draft_ms = float(np.mean([e0.elapsed_time(e1) for e0, e1 in kev]))
+    assert int(status.item()) == 0, f"device status {int(status.item()):#x}"
+    assert np.array_equal(acc.cpu().numpy(), vcase["length"]), "verify_accept result changed"
+
+    # ---- timed region 2: end to end through the host-buffer entry points
+    for _ in range(3):
+        step_host()
+    barrier()
+    e2 = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    n_e2e = max(10, a.steps // 4)
+    e2[0].record()
+    for _ in range(n_e2e):
+        step_host()
+    e2[1].record()
+    barrier()
+    ms_e2e = max_over_ranks(e2[0].elapsed_time(e2[1]))
+    assert np.array_equal(hout.numpy(), out_d.cpu().numpy()), "host and device entry points disagree"
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = ms_total / a.steps
+    value = world * B * K * a.steps / (ms_total * 1e-3)
+    e2e_value = world * B * K * n_e2e / (ms_e2e * 1e-3)
+    bytes_launch = sum(algorithmic_bytes_per_draft_step(s, B, N, ctx_lens, k) for k in range(K))
+    peak, peak_kind = load_peaks()
+    achieved = bytes_launch / (draft_ms * 1e-3) / 1e9
+    out = {
+        "metric": "draft_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": a.steps,
+        "warmup": max(a.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate", "data": "synthetic",
+        "config": {"workload": workload_name(a, s, N), "batch": B, "draft_steps": K,
+                   "l2": "inputs larger than L2: every step re-streams %.0f MB of weights" % (bytes_launch / K / 1e6),
+                   "parallelism": "replicas" if world > 1 else "single GPU"},
+        "us_per_draft_step": draft_ms * 1e3 / K,
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "tokens/s",
+                "h2d_bytes_per_step": int(hh.numel() * 2 + htok.numel() * 4 + hlog.numel() * 2 + hdv.numel() * 4),
+                "d2h_bytes_per_step": int(hout.numel() * 4 + hacc.numel() * 4 + hbon.numel() * 4 + 8),
+                "steps": n_e2e},
+        "roofline": {"bound": "hbm", "kernel": "mega_kernel (fastmtp_draft, K steps per launch)",
+                     "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "algorithmic_bytes_per_launch": int(bytes_launch), "launch_ms": draft_ms, "traffic": None},
+    }
+    if world == 1 and not a.no_cpu_baseline:
+        v, cores, sample = cpu_oracle_sample(s, W, kv, h, tok, ids, vcase, K)
+        out["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample}
+    print(json.dumps(out))
+    ctx.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)
+
+
+if __name__ == "__main__":
+    main()
