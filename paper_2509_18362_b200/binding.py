@@ -14,7 +14,7 @@ import torch
 
 from . import build as _build
 
-_LIB_PATH = _build.LIB
+_LIB_PATH = os.environ.get("FASTMTP_LIB", _build.LIB)     # override: a library built elsewhere
 if not os.path.exists(_LIB_PATH):
     raise ImportError(f"{_LIB_PATH} not built: run `python -m paper_2509_18362_b200.build` "
                       "(there is no CPU fallback)")

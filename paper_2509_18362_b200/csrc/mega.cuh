@@ -9,7 +9,12 @@ constexpr int kMaxLayers = 64;
 constexpr int kMaxRows = 8;          // activation rows (batch x rows-per-sequence) per launch
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 32;   // + one producer warp
+constexpr int kProducerWarps = 4;       // one warpgroup
+constexpr int kThreads = kConsumerThreads + kProducerWarps * 32;
+// Registers per thread after the warpgroups split (setmaxnreg): the kernel launches with
+// 65536 / 384 = 168 per thread; the producer warpgroup hands 72 x 128 back to the two consumer ones.
+constexpr int kProducerRegs = 96;
+constexpr int kConsumerRegs = 200;
 constexpr int kTileRows = 32;        // weight rows per pipeline stage (two 16-row MMA tiles)
 constexpr int kAttnChunk = 128;      // context tokens per attention work item
 constexpr int kMaxStages = 8;

@@ -2,11 +2,12 @@
 // steps (or of one target-decoder step) with grid barriers in between, so a draft call never
 // returns to the host between steps.
 //
-// Structure of a CTA (one per SM): 8 consumer warps + 1 producer warp.
-//   * The producer streams bf16 weight rows from HBM into a ring of shared-memory stages with
-//     1-D bulk async copies (TMA engine) that complete on mbarriers. Weight addresses do not
-//     depend on activations, so the producer runs ahead of the grid barriers: while the
-//     consumers wait for the previous phase's vector, HBM keeps streaming the next phase's rows.
+// Structure of a CTA (one per SM): 8 consumer warps + 4 producer warps.
+//   * The producers stream bf16 weight rows from HBM into a ring of shared-memory stages with
+//     16-byte cp.async copies whose completion is counted on mbarriers (on B200 this path sustains
+//     ~65 GB/s per SM where 1 KB bulk copies reach ~25 GB/s and large ones ~47 GB/s). Weight addresses do not depend on activations, so the producers
+//     run ahead of the grid barriers: while the consumers wait for the previous phase's vector,
+//     HBM keeps streaming the next phase's rows.
 //   * A matrix-vector phase gives every CTA a contiguous range of output rows. A stage holds up
 //     to 32 rows x KC columns; the 8 consumer warps each take a fixed k-slice of the stage and
 //     multiply with mma.sync m16n8k16 (weights = A operand, activation rows = B operand columns),
@@ -50,7 +51,32 @@ struct Misc {   // small shared-memory block
     uint32_t aborted;
 };
 
+// Development aid, compiled only with -DFMTP_PROF: consumer thread 0 of every CTA stamps the
+// global timer at phase boundaries, and warp 0 of each role accumulates the cycles it spends
+// waiting / working, into device arrays the host reads with fmtp_prof_read() / fmtp_prof_wait().
+#ifdef FMTP_PROF
+constexpr int kProfMarks = 512;
+__device__ unsigned long long g_prof[160][kProfMarks];
+__device__ long long g_wait[160][8];   // consumer wait-full, consumer stage body, producer wait-empty, producer issue
+#define PROF(c) do { if ((c).tid == 0 && (c).nprof < kProfMarks) g_prof[(c).cta][(c).nprof++] = global_timer_ns(); } while (0)
+#define PROF_T0() long long prof_t0 = clock64()
+#define PROF_ACC(c, slot, cond) do { if (cond) { long long prof_t1 = clock64(); (c).pacc[slot] += prof_t1 - prof_t0; prof_t0 = prof_t1; } } while (0)
+#define PROF_FLUSH(c, lo, hi, cond) do { if (cond) for (int q_ = lo; q_ < hi; ++q_) atomicAdd((unsigned long long *)&g_wait[(c).cta][q_], (unsigned long long)(c).pacc[q_]); } while (0)
+#else
+#define PROF(c) do { } while (0)
+#define PROF_T0() do { } while (0)
+#define PROF_ACC(c, slot, cond) do { } while (0)
+#define PROF_FLUSH(c, lo, hi, cond) do { } while (0)
+#endif
+
+// Per-thread view of the CTA's state. Every function that takes it is force-inlined: if its address
+// escaped into a real call the whole struct would live in local memory and each field access
+// would queue behind the cp.async traffic in the load/store unit.
 struct Cta {
+#ifdef FMTP_PROF
+    int nprof;
+    long long pacc[5];
+#endif
     const MegaParams *p;
     Misc *misc;
     float *red;            // [2][8 warps][32 rows][R]
@@ -66,14 +92,14 @@ __device__ __forceinline__ void raise(const Cta &c, uint32_t bits) { atomicOr(c.
 
 __device__ __forceinline__ bool aborted(const Cta &c) { return *((volatile uint32_t *)&c.misc->aborted) != 0; }
 
-__device__ void do_abort(const Cta &c) {
+__device__ __forceinline__ void do_abort(const Cta &c) {
     c.misc->aborted = 1;
     atomicOr(c.p->s.status, kDevTimeout);
     atomicExch(c.p->s.abort_flag, 1u);
 }
 
 // Bounded wait on an mbarrier phase. Returns false (and raises the abort flag) on timeout.
-__device__ bool wait_bar(const Cta &c, uint64_t *bar, uint32_t parity) {
+__device__ __forceinline__ bool wait_bar(const Cta &c, uint64_t *bar, uint32_t parity) {
     if (aborted(c)) return false;
     unsigned long long t0 = 0;
     for (uint32_t n = 0;; ++n) {
@@ -93,7 +119,7 @@ __device__ bool wait_bar(const Cta &c, uint64_t *bar, uint32_t parity) {
 }
 
 // Grid-wide barrier among the consumer threads of all CTAs (the producer warp never joins).
-__device__ void grid_barrier(Cta &c) {
+__device__ __forceinline__ void grid_barrier(Cta &c) {
     bar_sync(1, kConsumerThreads);
     c.bar_target += (uint32_t)c.grid;
     if (c.tid == 0) {
@@ -109,7 +135,6 @@ __device__ void grid_barrier(Cta &c) {
                     if (t0 == 0) t0 = now;
                     else if (now - t0 > kWaitLimitNs) { do_abort(c); break; }
                 }
-                __nanosleep(32);
             }
         }
         __threadfence();
@@ -168,27 +193,82 @@ __device__ __forceinline__ const bf16_t *tile_row_ptr(const Cta &c, int kind, co
 }
 
 // ---- producer ------------------------------------------------------------------------------
-__device__ void produce_phase(Cta &c, int kind, const LayerPtrs &L) {
+// The producer warps copy a stage with 16-byte cp.async instructions: warp `pw` takes tile rows
+// pw, pw + 4, pw + 8, ...; its 32 lanes cover 512 contiguous bytes of a row per instruction.
+// Each thread then posts an asynchronous arrival on the stage's `full` barrier that fires when its
+// own copies have landed. The copies of a stage are issued from fully unrolled code with one
+// address register pair per instruction: a cp.async reads its address operands only when it
+// leaves the memory-instruction queue, so reusing an address register for the next copy would
+// stall the warp on every instruction (measured: 4.2 instead of 7.0 TB/s). Row pointers of the
+// next tile are computed one tile ahead so the subset-id lookup of the output head is off the
+// issue path.
+constexpr int kRowsPerProducer = kTileRows / kProducerWarps;   // 4
+
+__device__ __forceinline__ void tile_ptrs(const Cta &c, int kind, const LayerPtrs &L, int vr0, int nv, int pw,
+                                          const unsigned char *(&out)[kRowsPerProducer]) {
+#pragma unroll
+    for (int i = 0; i < kRowsPerProducer; ++i)
+        out[i] = reinterpret_cast<const unsigned char *>(tile_row_ptr(c, kind, L, vr0, nv, pw + i * kProducerWarps));
+}
+
+__device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs &L) {
     const MegaParams &p = *c.p;
     Geom g = geom(c, kind);
+    const int pw = c.warp - kConsumerWarps;
+    const unsigned char *cur[kRowsPerProducer], *nxt[kRowsPerProducer];
+#pragma unroll
+    for (int i = 0; i < kRowsPerProducer; ++i) nxt[i] = nullptr;
+    if (g.v0 < g.v1) tile_ptrs(c, kind, L, g.v0, min(g.cap, g.v1 - g.v0), pw, nxt);
+    const uint32_t lane16 = (uint32_t)c.lane * 16u;
     for (int vr0 = g.v0; vr0 < g.v1; vr0 += g.cap) {
-        int nv = min(g.cap, g.v1 - vr0);
-        const bf16_t *src = tile_row_ptr(c, kind, L, vr0, nv, c.lane);
-        int nrows = (kind == GATEUP) ? 2 * nv : nv;
+#pragma unroll
+        for (int i = 0; i < kRowsPerProducer; ++i) cur[i] = nxt[i];
+        if (vr0 + g.cap < g.v1) tile_ptrs(c, kind, L, vr0 + g.cap, min(g.cap, g.v1 - vr0 - g.cap), pw, nxt);
         for (int ks = 0; ks < g.nks; ++ks) {
             int slot = c.stage % p.n_stages;
             uint32_t parity = (c.stage / p.n_stages) & 1u;
             bool ok = true;
+            PROF_T0();
             if (c.lane == 0) ok = wait_bar(c, &c.misc->empty[slot], parity ^ 1u);
             ok = __shfl_sync(0xffffffffu, ok, 0);
+            PROF_ACC(c, 2, pw == 0 && c.lane == 0);
             if (!ok) return;   // abort: stop issuing copies
-            int klen = min(p.KC, g.K - ks * p.KC);
-            uint32_t bytes = (uint32_t)klen * 2u;
-            if (c.lane == 0) mbar_arrive_expect_tx(&c.misc->full[slot], bytes * (uint32_t)nrows);
-            __syncwarp();
-            if (src)
-                bulk_g2s(c.ring + (size_t)slot * p.stage_bytes + (size_t)c.lane * p.row_stride,
-                         src + (size_t)ks * p.KC, bytes, &c.misc->full[slot]);
+            const int klen = min(p.KC, g.K - ks * p.KC);
+            const uint32_t dst0 = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + (uint32_t)pw * (uint32_t)p.row_stride + lane16;
+            const size_t koff = (size_t)ks * p.KC * 2 + lane16;
+            if (klen == 512) {
+                // 1024 bytes per row: two instructions per row, eight per thread, all independent
+                uint32_t d[2 * kRowsPerProducer];
+                const unsigned char *q[2 * kRowsPerProducer];
+#pragma unroll
+                for (int i = 0; i < kRowsPerProducer; ++i) {
+                    d[2 * i] = dst0 + (uint32_t)(i * kProducerWarps) * (uint32_t)p.row_stride;
+                    d[2 * i + 1] = d[2 * i] + 512u;
+                    q[2 * i] = cur[i] + koff;
+                    q[2 * i + 1] = q[2 * i] + 512;
+                }
+#pragma unroll
+                for (int i = 0; i < kRowsPerProducer; ++i) {
+                    if (cur[i] != nullptr) {
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d[2 * i]), "l"(q[2 * i]) : "memory");
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d[2 * i + 1]), "l"(q[2 * i + 1]) : "memory");
+                    }
+                }
+            } else {
+                // other stage widths (small or odd geometries): generic loop
+                const int n16 = klen >> 3;
+#pragma unroll
+                for (int i = 0; i < kRowsPerProducer; ++i) {
+                    if (cur[i] != nullptr) {
+                        for (int u = c.lane; u < n16; u += 32) {
+                            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst0 + (uint32_t)(i * kProducerWarps) * (uint32_t)p.row_stride + (uint32_t)(u - c.lane) * 16u),
+                                         "l"(cur[i] + koff + (size_t)(u - c.lane) * 16) : "memory");
+                        }
+                    }
+                }
+            }
+            cp_async_arrive(&c.misc->full[slot]);
+            PROF_ACC(c, 3, pw == 0 && c.lane == 0);
             c.stage++;
         }
     }
@@ -204,74 +284,138 @@ struct ActSrc {          // where the B operand (activations) is read from
 template <int KIND>
 struct Epi;   // epilogue functors, specialised below
 
+// Moves the running sums of the first input segment aside (the projection scales its two input
+// segments with different RMSNorm factors).
+template <bool two_sets>
+__device__ __forceinline__ void park(float (&acc)[2][2][4], float (&acd)[2][2][4], float (&acc0)[2][4], float (&acd0)[2][4]) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            acc0[i][j] = acc[i][0][j] + acc[i][1][j];
+            acc[i][0][j] = acc[i][1][j] = 0.f;
+            if (two_sets) {
+                acd0[i][j] = acd[i][0][j] + acd[i][1][j];
+                acd[i][0][j] = acd[i][1][j] = 0.f;
+            }
+        }
+}
+
 // Runs all tiles of one phase for this CTA. `epi(vrow, col, v0, v1)` is called once per valid
 // (virtual row, activation row) by exactly one thread; v1 is the paired "up" value for GATEUP.
-template <int KIND, typename EpiF>
-__device__ void consume_phase(Cta &c, const ActSrc &act, int seg_stage, EpiF &&epi) {
+// One chunk (32 weight rows x 32 k) of a stage: four MMAs per activation set.
+struct Frag { uint4 u0, v0, u1, v1; };
+__device__ __forceinline__ Frag load_frag(const unsigned char *a, int g, int row_stride) {
+    Frag f;
+    f.u0 = lds128(a + (size_t)g * row_stride);
+    f.v0 = lds128(a + (size_t)(g + 8) * row_stride);
+    f.u1 = lds128(a + (size_t)(g + 16) * row_stride);
+    f.v1 = lds128(a + (size_t)(g + 24) * row_stride);
+    return f;
+}
+__device__ __forceinline__ void mma_chunk(float (&acc)[2][2][4], const Frag &f, const uint4 &b) {
+    mma_bf16(acc[0][0], f.u0.x, f.v0.x, f.u0.y, f.v0.y, b.x, b.y);
+    mma_bf16(acc[1][0], f.u1.x, f.v1.x, f.u1.y, f.v1.y, b.x, b.y);
+    mma_bf16(acc[0][1], f.u0.z, f.v0.z, f.u0.w, f.v0.w, b.z, b.w);
+    mma_bf16(acc[1][1], f.u1.z, f.v1.z, f.u1.w, f.v1.w, b.z, b.w);
+}
+__device__ __forceinline__ uint4 load_act(const bf16_t *base, size_t off, bool in_smem) {
+    return in_smem ? lds128(base + off) : ldcg128(base + off);
+}
+
+// Runs all tiles of one phase for this CTA. `epi(vrow, col, v0, v1)` is called once per valid
+// (virtual row, activation row) by exactly one thread; v1 is the paired "up" value for GATEUP.
+//
+// MMA mapping: A = 16 weight rows x 16 k, B column 2r holds the hi part and column 2r+1 the lo
+// part of activation row r, so one MMA covers four activation rows exactly (the two columns are
+// added at the end); rows 4..7 use a second set of accumulators. The two halves of the consumer
+// warps (warps 0-3 / 4-7) take alternate stages, so each warp does four chunks per barrier wait
+// and two stages are in work at once.
+template <int KIND, bool two_sets, typename EpiF>
+__device__ __forceinline__ void consume_tiles(Cta &c, const ActSrc &act, int seg_stage, EpiF &epi) {
     const MegaParams &p = *c.p;
     Geom geo = geom(c, KIND);
     const int R = p.R;
     const int g = c.lane >> 2, t = c.lane & 3;
-    const int nchunk_full = p.KC / 32;
+    const int grp = c.warp >> 2, wi = c.warp & 3;
+    const int arow = g >> 1;
+    const bf16_t *abase = (g & 1) ? act.lo : act.hi;
+    const bool has0 = arow < R, has1 = arow + 4 < R;
+    const size_t aoff0 = (size_t)arow * act.stride + t * 8, aoff1 = (size_t)(arow + 4) * act.stride + t * 8;
     for (int vr0 = geo.v0; vr0 < geo.v1; vr0 += geo.cap) {
         int nv = min(geo.cap, geo.v1 - vr0);
-        float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-        float acc0[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        float acc[2][2][4], acd[2][2][4], acc0[2][4], acd0[2][4];
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                acc[i][0][j] = acc[i][1][j] = acd[i][0][j] = acd[i][1][j] = 0.f;
+                acc0[i][j] = acd0[i][j] = 0.f;
+            }
+        bool moved = false;
         for (int ks = 0; ks < geo.nks; ++ks) {
-            int slot = c.stage % p.n_stages;
-            uint32_t parity = (c.stage / p.n_stages) & 1u;
-            wait_bar(c, &c.misc->full[slot], parity);
-            int klen = min(p.KC, geo.K - ks * p.KC);
-            int nchunk = (klen == p.KC) ? nchunk_full : (klen + 31) / 32;
-            const unsigned char *st = c.ring + (size_t)slot * p.stage_bytes;
-            for (int ch = c.warp; ch < nchunk; ch += kConsumerWarps) {
-                const unsigned char *a = st + ch * 64 + t * 16;
-                uint4 u0 = lds128(a + (size_t)g * p.row_stride);
-                uint4 v0 = lds128(a + (size_t)(g + 8) * p.row_stride);
-                uint4 u1 = lds128(a + (size_t)(g + 16) * p.row_stride);
-                uint4 v1 = lds128(a + (size_t)(g + 24) * p.row_stride);
-                uint4 bh = make_uint4(0, 0, 0, 0), bl = make_uint4(0, 0, 0, 0);
-                if (g < R) {
-                    size_t off = (size_t)g * act.stride + (size_t)ks * p.KC + ch * 32 + t * 8;
-                    if (act.in_smem) {
-                        bh = lds128(act.hi + off);
-                        bl = lds128(act.lo + off);
-                    } else {   // produced by other CTAs in the previous phase: read through L2
-                        bh = ldcg128(act.hi + off);
-                        bl = ldcg128(act.lo + off);
+            if ((int)(c.stage & 1u) == grp) {
+                int slot = c.stage % p.n_stages;
+                uint32_t parity = (c.stage / p.n_stages) & 1u;
+                PROF_T0();
+                wait_bar(c, &c.misc->full[slot], parity);
+                PROF_ACC(c, 0, c.tid == 0);
+                if (KIND == PROJ && !moved && ks >= seg_stage) {   // second input segment starts: park the first
+                    moved = true;
+                    park<two_sets>(acc, acd, acc0, acd0);
+                }
+                const int klen = min(p.KC, geo.K - ks * p.KC);
+                const int nchunk = (klen + 31) >> 5;
+                const unsigned char *st = c.ring + (size_t)slot * p.stage_bytes + t * 16;
+                const size_t kbase = (size_t)ks * p.KC;
+                const uint4 zero = make_uint4(0, 0, 0, 0);
+                // chunks wi, wi+4, wi+8, wi+12 in two batches of two: all loads of a batch are issued
+                // before its MMAs
+                for (int ch = wi; ch < nchunk; ch += 8) {
+                    const bool second = ch + 4 < nchunk;
+                    Frag f0 = load_frag(st + ch * 64, g, p.row_stride);
+                    uint4 b0 = has0 ? load_act(abase, aoff0 + kbase + ch * 32, act.in_smem) : zero;
+                    uint4 d0 = (two_sets && has1) ? load_act(abase, aoff1 + kbase + ch * 32, act.in_smem) : zero;
+                    Frag f1;
+                    uint4 b1 = zero, d1 = zero;
+                    if (second) {
+                        f1 = load_frag(st + (ch + 4) * 64, g, p.row_stride);
+                        if (has0) b1 = load_act(abase, aoff0 + kbase + (ch + 4) * 32, act.in_smem);
+                        if (two_sets && has1) d1 = load_act(abase, aoff1 + kbase + (ch + 4) * 32, act.in_smem);
+                    }
+                    mma_chunk(acc, f0, b0);
+                    if (two_sets) mma_chunk(acd, f0, d0);
+                    if (second) {
+                        mma_chunk(acc, f1, b1);
+                        if (two_sets) mma_chunk(acd, f1, d1);
                     }
                 }
-                mma_bf16(acc[0], u0.x, v0.x, u0.y, v0.y, bh.x, bh.y);
-                mma_bf16(acc[1], u1.x, v1.x, u1.y, v1.y, bh.x, bh.y);
-                mma_bf16(acc[0], u0.z, v0.z, u0.w, v0.w, bh.z, bh.w);
-                mma_bf16(acc[1], u1.z, v1.z, u1.w, v1.w, bh.z, bh.w);
-                mma_bf16(acc[0], u0.x, v0.x, u0.y, v0.y, bl.x, bl.y);
-                mma_bf16(acc[1], u1.x, v1.x, u1.y, v1.y, bl.x, bl.y);
-                mma_bf16(acc[0], u0.z, v0.z, u0.w, v0.w, bl.z, bl.w);
-                mma_bf16(acc[1], u1.z, v1.z, u1.w, v1.w, bl.z, bl.w);
+                __syncwarp();
+                if (c.lane == 0) mbar_arrive(&c.misc->empty[slot]);
+                PROF_ACC(c, 1, c.tid == 0);
             }
-            __syncwarp();
-            if (c.lane == 0) mbar_arrive(&c.misc->empty[slot]);
             c.stage++;
-            if (KIND == PROJ && ks + 1 == seg_stage) {
-#pragma unroll
-                for (int i = 0; i < 2; ++i)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) { acc0[i][j] = acc[i][j]; acc[i][j] = 0.f; }
-            }
         }
+        // a warp whose stages all lay in the first segment parks them now
+        if (KIND == PROJ && !moved) park<two_sets>(acc, acd, acc0, acd0);
         // cross-warp reduction in a fixed order
+        PROF_T0();
         float *red = c.red + (size_t)c.redbuf * kConsumerWarps * kTileRows * R + (size_t)c.warp * kTileRows * R;
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                int row = i * 16 + g + ((j >> 1) << 3);
-                int col = 2 * t + (j & 1);
-                if (col < R) {
-                    float v = acc[i][j];
-                    if (KIND == PROJ) v = acc0[i][j] * c.misc->scale0[col] + v * c.misc->scale1[col];
-                    red[row * R + col] = v;
+            for (int h = 0; h < 2; ++h) {
+                const int row = i * 16 + g + h * 8;
+                // activation row t (set 0) / t + 4 (set 1): hi column + lo column
+                if (t < R) {
+                    float v = (acc[i][0][2 * h] + acc[i][0][2 * h + 1]) + (acc[i][1][2 * h] + acc[i][1][2 * h + 1]);
+                    if (KIND == PROJ) v = (acc0[i][2 * h] + acc0[i][2 * h + 1]) * c.misc->scale0[t] + v * c.misc->scale1[t];
+                    red[row * R + t] = v;
+                }
+                if (two_sets && t + 4 < R) {
+                    float v = (acd[i][0][2 * h] + acd[i][0][2 * h + 1]) + (acd[i][1][2 * h] + acd[i][1][2 * h + 1]);
+                    if (KIND == PROJ) v = (acd0[i][2 * h] + acd0[i][2 * h + 1]) * c.misc->scale0[t + 4] + v * c.misc->scale1[t + 4];
+                    red[row * R + t + 4] = v;
                 }
             }
         }
@@ -297,12 +441,19 @@ __device__ void consume_phase(Cta &c, const ActSrc &act, int seg_stage, EpiF &&e
             }
         }
         c.redbuf ^= 1;
+        PROF_ACC(c, 4, c.tid == 0);
     }
+}
+
+template <int KIND, typename EpiF>
+__device__ __forceinline__ void consume_phase(Cta &c, const ActSrc &act, int seg_stage, EpiF &&epi) {
+    if (c.p->R > 4) consume_tiles<KIND, true>(c, act, seg_stage, epi);
+    else consume_tiles<KIND, false>(c, act, seg_stage, epi);
 }
 
 // Sum over CTAs of a per-CTA partial-sums-of-squares table [grid][8], for activation row `col`.
 // Called by one full warp; fixed reduction tree => reproducible.
-__device__ float sum_partials(const Cta &c, const float *tbl, int col) {
+__device__ __forceinline__ float sum_partials(const Cta &c, const float *tbl, int col) {
     float s = 0.f;
     for (int i = c.lane; i < c.grid; i += 32) s += ldcg_f32(tbl + (size_t)i * kMaxRows + col);
 #pragma unroll
@@ -313,7 +464,7 @@ __device__ float sum_partials(const Cta &c, const float *tbl, int col) {
 // Copies R rows of a hi/lo activation pair from global scratch into the shared staging area.
 // `len` elements per row (multiple of 8), rows `stride_s` apart in shared memory, starting at
 // element offset `dst_off`.
-__device__ void stage_hilo(const Cta &c, const bf16_t *ghi, const bf16_t *glo, int gstride, int len, bf16_t *shi,
+__device__ __forceinline__ void stage_hilo(const Cta &c, const bf16_t *ghi, const bf16_t *glo, int gstride, int len, bf16_t *shi,
                            bf16_t *slo, int sstride, int dst_off) {
     int per_row = len / 8;
     int total = c.p->R * per_row;
@@ -328,7 +479,7 @@ __device__ void stage_hilo(const Cta &c, const bf16_t *ghi, const bf16_t *glo, i
 
 // Block-wide sum of up to 2 values per activation row, all consumer threads participate.
 // Result for (col, which) is left in misc->ssred[0][col][which].
-__device__ void block_sum2(const Cta &c, float (&v)[kMaxRows][2], int R) {
+__device__ __forceinline__ void block_sum2(const Cta &c, float (&v)[kMaxRows][2], int R) {
     for (int r = 0; r < R; ++r)
 #pragma unroll
         for (int w = 0; w < 2; ++w) {
@@ -353,7 +504,7 @@ struct SqAcc {
     float a, b;
     __device__ SqAcc() : a(0.f), b(0.f) {}
 };
-__device__ void flush_sq(const Cta &c, const SqAcc &q, float *tblA, float *tblB) {
+__device__ __forceinline__ void flush_sq(const Cta &c, const SqAcc &q, float *tblA, float *tblB) {
     // thread (row = tid>>3, col = tid&7)
     int row = c.tid >> 3, col = c.tid & 7;
     for (int which = 0; which < 2; ++which) {
@@ -382,7 +533,7 @@ __device__ __forceinline__ void store_split(bf16_t *hi, bf16_t *lo, size_t idx, 
 //   qs[M*Gq][dh]  rotated, pre-scaled queries of one KV head
 //   kn[M][dh], vn[M][dh]  this call's new keys / values (after bf16 rounding)
 //   wp[8 warps][Gq][dh + 2] per-warp partial (o, m, l) for the row being processed
-__device__ void attention_phase(Cta &c, const KvPtrs &kv, int posoff) {
+__device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int posoff) {
     const MegaParams &p = *c.p;
     const int dh = p.dh, half = dh >> 1, Gq = p.Hq / p.Hkv, M = p.M;
     const int epl = dh >> 5;   // elements per lane (2 or 4)
@@ -625,11 +776,15 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
     c.stage = 0;
     c.bar_target = 0;
     c.redbuf = 0;
+#ifdef FMTP_PROF
+    c.nprof = 0;
+    for (int i = 0; i < 5; ++i) c.pacc[i] = 0;
+#endif
 
     if (c.tid == 0) {
         for (int i = 0; i < p.n_stages; ++i) {
-            mbar_init(&c.misc->full[i], 1);
-            mbar_init(&c.misc->empty[i], kConsumerWarps);
+            mbar_init(&c.misc->full[i], kProducerWarps * 32);
+            mbar_init(&c.misc->empty[i], kConsumerWarps / 2);   // the four warps that own the stage
         }
         c.misc->aborted = 0;
         mbar_fence_init();
@@ -637,15 +792,19 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
     // the ring starts zeroed so that never-written tails multiply as finite numbers
     for (size_t i = (size_t)c.tid * 16; i < (size_t)p.n_stages * p.stage_bytes; i += (size_t)kThreads * 16)
         *reinterpret_cast<uint4 *>(c.ring + i) = make_uint4(0, 0, 0, 0);
-    fence_proxy_async();
     __syncthreads();
 
-    const bool is_producer = (c.warp == kConsumerWarps);
+#ifdef FMTP_PROF
+    const long long prof_c0 = clock64();
+    const unsigned long long prof_n0 = global_timer_ns();
+#endif
+    const bool is_producer = (c.warp >= kConsumerWarps);
     const int R = p.R;
     const int n_steps = (p.mode == 0) ? p.K : 1;
     const int n_layers = (p.mode == 0) ? 1 : p.n_layers;
 
     if (is_producer) {
+        setmaxnreg_dec<kProducerRegs>();
         // ---------------- producer: the weight stream of every phase, in program order
         for (int step = 0; step < n_steps; ++step) {
             if (p.mode == 0) produce_phase(c, PROJ, p.layers[0]);
@@ -657,27 +816,19 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
             }
             produce_phase(c, HEAD, p.layers[0]);
         }
-        // drain: every copy this warp issued must have landed before the CTA may exit
-        if (c.lane == 0) {
-            uint32_t issued = c.stage;
-            uint32_t first = issued > (uint32_t)p.n_stages ? issued - p.n_stages : 0;
-            for (uint32_t s = first; s < issued; ++s) {
-                uint64_t *bar = &c.misc->full[s % p.n_stages];
-                uint32_t parity = (s / p.n_stages) & 1u;
-                unsigned long long t0 = global_timer_ns();
-                for (uint32_t n = 0; !mbar_try_wait(bar, parity); ++n)
-                    if ((n & 255u) == 255u && global_timer_ns() - t0 > kWaitLimitNs) break;
-            }
-        }
+        cp_async_wait_all();   // every copy this thread issued has landed before the CTA may exit
+        PROF_FLUSH(c, 2, 4, c.warp == kConsumerWarps && c.lane == 0);
         return;
     }
 
     // ---------------- consumers
+    setmaxnreg_inc<kConsumerRegs>();
     bf16_t *s_hi = reinterpret_cast<bf16_t *>(c.scr);
     const int KCd = p.KC;
     auto act_stride = [&](int len) { return ((len + 31) & ~31) + 32; };   // +64 B: rows land in different banks
 
     for (int step = 0; step < n_steps; ++step) {
+        PROF(c);
         // ============ front end
         if (p.mode == 0) {
             // ---- PROJ: x0 = W_p [ rms(h) ; rms(Emb(tok)) ]
@@ -741,13 +892,16 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
             SqAcc sqa;
             ActSrc act{a_hi, a_lo, st, true};
             const LayerPtrs &L0 = p.layers[0];
+            PROF(c);
             consume_phase<PROJ>(c, act, p.d / KCd, [&](int row, int col, float v, float) {
                 p.s.x0[(size_t)col * p.d + row] = v;
                 store_split(p.s.actD_hi, p.s.actD_lo, (size_t)col * p.dp + row, v * bf16bits_f32(L0.g_in[row]));
                 sqa.a += v * v;
             });
             flush_sq(c, sqa, p.s.ssA, nullptr);
+            PROF(c);
             grid_barrier(c);
+            PROF(c);
         } else {
             // ---- EMBED (target): x0 = Emb(tok), CTA-sliced over d
             int r0 = (int)(((long long)c.cta * p.d) / c.grid), r1 = (int)(((long long)(c.cta + 1) * p.d) / c.grid);
@@ -785,14 +939,19 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                 bar_sync(1, kConsumerThreads);
                 ActSrc act{a_hi, a_lo, st, true};
                 const int nq = p.qdim + 2 * p.kvdim;
+                PROF(c);
                 consume_phase<QKV>(c, act, 0, [&](int row, int col, float v, float) {
                     p.s.qkv[(size_t)col * nq + row] = v * c.misc->scale0[col];
                 });
+                PROF(c);
                 grid_barrier(c);
+                PROF(c);
             }
             // ---- attention
             attention_phase(c, p.kvs[l], (p.mode == 0) ? step : 0);
+            PROF(c);
             grid_barrier(c);
+            PROF(c);
             // ---- O projection + residual
             {
                 const int st = act_stride(p.qdim);
@@ -801,6 +960,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                 bar_sync(1, kConsumerThreads);
                 ActSrc act{a_hi, a_lo, st, true};
                 SqAcc sqa;
+                PROF(c);
                 consume_phase<OPROJ>(c, act, 0, [&](int row, int col, float v, float) {
                     float x = ldcg_f32(p.s.x0 + (size_t)col * p.d + row) + v;
                     p.s.x1[(size_t)col * p.d + row] = x;
@@ -808,7 +968,9 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                     sqa.a += x * x;
                 });
                 flush_sq(c, sqa, p.s.ssB, nullptr);
+                PROF(c);
                 grid_barrier(c);
+                PROF(c);
             }
             // ---- gate / up + SwiGLU
             {
@@ -821,6 +983,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                 }
                 bar_sync(1, kConsumerThreads);
                 ActSrc act{a_hi, a_lo, st, true};
+                PROF(c);
                 consume_phase<GATEUP>(c, act, 0, [&](int row, int col, float gt, float up) {
                     float s = c.misc->scale0[col];
                     gt *= s;
@@ -828,7 +991,9 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                     float a = gt / (1.f + expf(-gt)) * up;
                     store_split(p.s.actF_hi, p.s.actF_lo, (size_t)col * p.Fp + row, a);
                 });
+                PROF(c);
                 grid_barrier(c);
+                PROF(c);
             }
             // ---- down projection + residual
             {
@@ -844,6 +1009,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                     act = ActSrc{p.s.actF_hi, p.s.actF_lo, p.Fp, false};
                 }
                 SqAcc sqa;
+                PROF(c);
                 const bf16_t *gnext = (p.mode == 1 && !last_layer) ? p.layers[l + 1].g_in : p.g_final;
                 consume_phase<DOWN>(c, act, 0, [&](int row, int col, float v, float) {
                     float x = ldcg_f32(p.s.x1 + (size_t)col * p.d + row) + v;
@@ -863,7 +1029,9 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                 });
                 bool to_head = !(p.mode == 1 && !last_layer);
                 flush_sq(c, sqa, to_head ? p.s.ssC : p.s.ssA, (p.mode == 0) ? p.s.ssD : nullptr);
+                PROF(c);
                 grid_barrier(c);
+                PROF(c);
             }
         }
 
@@ -888,6 +1056,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
             }
             ActSrc act{a_hi, a_lo, st, true};
             unsigned long long best = 0ull;
+            PROF(c);
             consume_phase<HEAD>(c, act, 0, [&](int row, int col, float v, float) {
                 int id = p.ids ? p.ids[row] : row;
                 if ((unsigned)id >= (unsigned)p.V) id = 0;
@@ -918,10 +1087,20 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                     if (m != 0ull) atomicMax(p.s.keys + (size_t)step * kMaxRows + c.tid, m);
                 }
             }
+            PROF(c);
             grid_barrier(c);
+            PROF(c);
         }
     }
 
+    PROF_FLUSH(c, 0, 2, c.tid == 0);
+    PROF_FLUSH(c, 4, 5, c.tid == 0);
+#ifdef FMTP_PROF
+    if (c.tid == 0) {
+        atomicAdd((unsigned long long *)&g_wait[c.cta][5], (unsigned long long)(clock64() - prof_c0));
+        atomicAdd((unsigned long long *)&g_wait[c.cta][6], global_timer_ns() - prof_n0);
+    }
+#endif
     // ============ publish the last step's tokens and the status word
     if (c.cta == 0 && c.tid < R) {
         int last = n_steps - 1;
@@ -941,6 +1120,17 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
 }
 
 }  // namespace
+
+#ifdef FMTP_PROF
+extern "C" int fmtp_prof_wait(long long *host, int reset) {
+    int e = (int)cudaMemcpyFromSymbol(host, g_wait, sizeof(g_wait));
+    if (reset) { static long long z[160][8]; cudaMemcpyToSymbol(g_wait, z, sizeof(z)); }
+    return e;
+}
+extern "C" int fmtp_prof_read(unsigned long long *host, size_t bytes) {
+    return (int)cudaMemcpyFromSymbol(host, g_prof, bytes < sizeof(g_prof) ? bytes : sizeof(g_prof));
+}
+#endif
 
 size_t mega_smem_bytes(const MegaParams &p) {
     size_t off = (sizeof(Misc) + 127) & ~size_t(127);
