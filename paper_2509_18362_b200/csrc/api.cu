@@ -124,11 +124,16 @@ int configure(fmtp_ctx *c, MegaParams &p, int mode, int B, int M) {
     p.KC = c->KC;
     p.row_stride = p.KC * 2 + 64;
     p.stage_bytes = kTileRows * p.row_stride;
+    {   // a stage also has to hold one 64-token K/V chunk of a KV head
+        int kvb = 2 * kAttnChunk * p.dh * 2;
+        if (kvb > p.stage_bytes) p.stage_bytes = kvb;
+        p.stage_bytes = (p.stage_bytes + 127) & ~127;
+    }
     p.max_chunks = c->max_chunks;
     p.max_ctx = sh.max_ctx;
     p.mode = mode; p.B = B; p.M = M; p.R = B * M;
     const int R = p.R, Gq = p.Hq / p.Hkv;
-    size_t attn = ((size_t)M * Gq * p.dh + 2 * (size_t)M * p.dh + (size_t)kConsumerWarps * Gq * (p.dh + 2)) * 4;
+    size_t attn = ((size_t)M * Gq * p.dh + (size_t)kConsumerWarps * Gq * (p.dh + 2)) * 4;
     size_t actd = (size_t)2 * R * act_stride(mode == 0 ? 2 * p.d : (p.d > p.qdim ? p.d : p.qdim)) * 2;
     size_t actq = (size_t)2 * R * act_stride(p.qdim) * 2;
     size_t base = attn > actd ? attn : actd;

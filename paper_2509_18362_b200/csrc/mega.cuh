@@ -16,7 +16,7 @@ constexpr int kThreads = kConsumerThreads + kProducerWarps * 32;
 constexpr int kProducerRegs = 96;
 constexpr int kConsumerRegs = 200;
 constexpr int kTileRows = 32;        // weight rows per pipeline stage (two 16-row MMA tiles)
-constexpr int kAttnChunk = 128;      // context tokens per attention work item
+constexpr int kAttnChunk = 64;       // context tokens per attention work item
 constexpr int kMaxStages = 8;
 
 typedef uint16_t bf16_t;

@@ -9,17 +9,21 @@
 //     run ahead of the grid barriers: while the consumers wait for the previous phase's vector,
 //     HBM keeps streaming the next phase's rows.
 //   * A matrix-vector phase gives every CTA a contiguous range of output rows. A stage holds up
-//     to 32 rows x KC columns; the 8 consumer warps each take a fixed k-slice of the stage and
-//     multiply with mma.sync m16n8k16 (weights = A operand, activation rows = B operand columns),
-//     then reduce across warps in a fixed order. The activation vector is fp32 carried as two
-//     bf16 numbers (hi + lo), so products are exact and the sum is fp32-accurate; each of the up
-//     to 8 activation rows occupies its own MMA column, so a row's result does not depend on how
-//     many other rows the call carries.
+//     to 32 rows x KC columns; the two halves of the consumer warps take alternate stages, each
+//     warp a fixed k-slice, and multiply with mma.sync m16n8k16 (weights = A operand, activation
+//     rows = B operand columns), then reduce across warps in a fixed order. The activation vector
+//     is fp32 carried as two bf16 numbers (hi + lo, two adjacent MMA columns), so products are
+//     exact and the sum is fp32-accurate; every activation row has its own column pair, so a
+//     row's result does not depend on how many other rows the call carries.
 //   * RMSNorm is folded: the producing phase stores x*g (split hi/lo) plus per-CTA partial sums of
 //     x^2; the consuming phase multiplies its accumulators by rsqrt(mean(x^2)+eps).
-//   * Attention splits the context into fixed 128-token chunks (work items over sequence x KV head
-//     x chunk), fp32 online softmax, and the CTA that finishes a (sequence, KV head) group last
-//     merges its chunks in a fixed order -- no float atomics anywhere, results are reproducible.
+//   * Attention splits the context into fixed 64-token chunks (work items over sequence x KV head
+//     x chunk) whose committed K/V the producers stream through the same ring, fp32 softmax per
+//     chunk, and the CTA that finishes a (sequence, KV head) group last merges its chunks in a
+//     fixed order -- no float atomics anywhere, results are reproducible.
+//   * Producers and consumers each walk the phase program from ONE loop with a runtime phase
+//     kind: the code is much larger than the instruction cache, and straight-line code that runs
+//     once per step is fetched from L2 (measured: 3-10x slower than the same code in a loop).
 //   * The output head gathers rows W[ids[j]] (Eq. 3 of the paper), keeps a running (value, id)
 //     maximum per activation row and publishes it with one 64-bit atomicMax per CTA; logits are
 //     never written unless a debug buffer is passed.
@@ -36,7 +40,12 @@ constexpr uint32_t kDevBadToken = 0x1u, kDevBadPage = 0x2u, kDevBadPos = 0x4u, k
                    kDevAllNan = 0x10u;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait gives up after 2 s
 
-enum Kind { PROJ = 0, QKV = 1, OPROJ = 2, GATEUP = 3, DOWN = 4, HEAD = 5 };
+enum Kind { PROJ = 0, QKV = 1, OPROJ = 2, GATEUP = 3, DOWN = 4, HEAD = 5, ATTN = 6, EMBED = 7, DONE = 8 };
+
+// The phase program of a launch. Draft: K x (PROJ, QKV, ATTN, OPROJ, GATEUP, DOWN, HEAD).
+// Target step: EMBED, n_layers x (QKV, ATTN, OPROJ, GATEUP, DOWN), HEAD. Producers and consumers
+// walk it independently with this iterator, each from a single loop.
+struct Prog { int step, layer, kind; };
 
 struct Misc {   // small shared-memory block
     uint64_t full[kMaxStages];
@@ -140,6 +149,27 @@ __device__ __forceinline__ void grid_barrier(Cta &c) {
         __threadfence();
     }
     bar_sync(1, kConsumerThreads);
+}
+
+__device__ __forceinline__ void prog_begin(const MegaParams &p, Prog &g) {
+    g.step = 0; g.layer = 0; g.kind = (p.mode == 0) ? PROJ : EMBED;
+}
+__device__ __forceinline__ void prog_next(const MegaParams &p, Prog &g) {
+    switch (g.kind) {
+        case PROJ: case EMBED: g.kind = QKV; break;
+        case QKV: g.kind = ATTN; break;
+        case ATTN: g.kind = OPROJ; break;
+        case OPROJ: g.kind = GATEUP; break;
+        case GATEUP: g.kind = DOWN; break;
+        case DOWN:
+            if (p.mode == 1 && g.layer + 1 < p.n_layers) { g.layer++; g.kind = QKV; }
+            else g.kind = HEAD;
+            break;
+        default:   // HEAD
+            g.step++; g.layer = 0;
+            g.kind = (p.mode == 0 && g.step < p.K) ? PROJ : DONE;
+            break;
+    }
 }
 
 // ---- phase geometry ----------------------------------------------------------------------
@@ -281,8 +311,107 @@ struct ActSrc {          // where the B operand (activations) is read from
     bool in_smem;
 };
 
-template <int KIND>
-struct Epi;   // epilogue functors, specialised below
+// Per-thread accumulation of v^2 per activation row across the tiles of a phase, reduced over
+// the CTA's rows at phase end and written to this CTA's line of a partial table.
+struct SqAcc {
+    float a, b;
+};
+
+// What the per-row epilogue of a matrix phase needs besides the value.
+struct EpiCtx {
+    SqAcc sq;
+    unsigned long long best;     // running (logit, id) maximum of this thread (output head)
+    const LayerPtrs *L;
+    const bf16_t *gnext;         // gain applied after the down projection (next layer's or the final norm's)
+    int step;
+    bool to_next_layer;          // target mode, not the last layer: the result feeds the next layer
+};
+
+__device__ __forceinline__ void store_split(bf16_t *hi, bf16_t *lo, size_t idx, float v) {
+    uint16_t h, l;
+    split_bf16(v, h, l);
+    hi[idx] = h;
+    lo[idx] = l;
+}
+
+// Epilogue of one (virtual row, activation row): what the phase does with the finished dot product.
+__device__ __forceinline__ void epilogue(const Cta &c, int kind, EpiCtx &x, int row, int col, float v, float up) {
+    const MegaParams &p = *c.p;
+    const Scratch &s = p.s;
+    switch (kind) {
+        case PROJ: {
+            s.x0[(size_t)col * p.d + row] = v;
+            store_split(s.actD_hi, s.actD_lo, (size_t)col * p.dp + row, v * bf16bits_f32(x.L->g_in[row]));
+            x.sq.a += v * v;
+            break;
+        }
+        case QKV:
+            s.qkv[(size_t)col * (p.qdim + 2 * p.kvdim) + row] = v * c.misc->scale0[col];
+            break;
+        case OPROJ: {
+            float r = ldcg_f32(s.x0 + (size_t)col * p.d + row) + v;
+            s.x1[(size_t)col * p.d + row] = r;
+            store_split(s.actP_hi, s.actP_lo, (size_t)col * p.dp + row, r * bf16bits_f32(x.L->g_post[row]));
+            x.sq.a += r * r;
+            break;
+        }
+        case GATEUP: {
+            float sc = c.misc->scale0[col];
+            float gt = v * sc, u = up * sc;
+            store_split(s.actF_hi, s.actF_lo, (size_t)col * p.Fp + row, gt / (1.f + expf(-gt)) * u);
+            break;
+        }
+        case DOWN: {
+            float r = ldcg_f32(s.x1 + (size_t)col * p.d + row) + v;
+            float y = r * bf16bits_f32(x.gnext[row]);
+            x.sq.a += r * r;
+            if (x.to_next_layer) {
+                s.x0[(size_t)col * p.d + row] = r;
+                store_split(s.actD_hi, s.actD_lo, (size_t)col * p.dp + row, y);
+            } else {
+                store_split(s.actH_hi, s.actH_lo, (size_t)col * p.dp + row, y);
+                if (p.mode == 0) {
+                    store_split(s.actR_hi, s.actR_lo, (size_t)col * p.dp + row, y * bf16bits_f32(p.g_hnorm[row]));
+                    x.sq.b += y * y;
+                }
+            }
+            break;
+        }
+        default: {   // HEAD
+            int id = p.ids ? p.ids[row] : row;
+            if ((unsigned)id >= (unsigned)p.V) id = 0;
+            float lv = v;
+            if (p.mode == 1) {
+                // target: the decision is taken on the bf16 logits that cross the boundary
+                uint16_t lb = f32_bf16bits(v * c.misc->scale0[col]);
+                if (p.out_logits_bf16) p.out_logits_bf16[(size_t)col * p.V + row] = lb;
+                lv = bf16bits_f32(lb);
+            } else if (p.out_logits_f32) {
+                p.out_logits_f32[((size_t)col * p.K + x.step) * p.N + row] = v * c.misc->scale0[col];
+            }
+            unsigned long long key = argmax_key(lv, (uint32_t)id);
+            x.best = key > x.best ? key : x.best;
+            break;
+        }
+    }
+}
+
+// One chunk (32 weight rows x 32 k) of a stage: four MMAs per activation set.
+struct Frag { uint4 u0, v0, u1, v1; };
+__device__ __forceinline__ void mma_chunk(float (&acc)[2][2][4], const Frag &f, const uint4 &b) {
+    mma_bf16(acc[0][0], f.u0.x, f.v0.x, f.u0.y, f.v0.y, b.x, b.y);
+    mma_bf16(acc[1][0], f.u1.x, f.v1.x, f.u1.y, f.v1.y, b.x, b.y);
+    mma_bf16(acc[0][1], f.u0.z, f.v0.z, f.u0.w, f.v0.w, b.z, b.w);
+    mma_bf16(acc[1][1], f.u1.z, f.v1.z, f.u1.w, f.v1.w, b.z, b.w);
+}
+__device__ __forceinline__ Frag load_frag(uint32_t a, uint32_t rs) {
+    Frag f;
+    f.u0 = lds128_u32(a);
+    f.v0 = lds128_u32(a + 8 * rs);
+    f.u1 = lds128_u32(a + 16 * rs);
+    f.v1 = lds128_u32(a + 24 * rs);
+    return f;
+}
 
 // Moves the running sums of the first input segment aside (the projection scales its two input
 // segments with different RMSNorm factors).
@@ -301,49 +430,31 @@ __device__ __forceinline__ void park(float (&acc)[2][2][4], float (&acd)[2][2][4
         }
 }
 
-// Runs all tiles of one phase for this CTA. `epi(vrow, col, v0, v1)` is called once per valid
-// (virtual row, activation row) by exactly one thread; v1 is the paired "up" value for GATEUP.
-// One chunk (32 weight rows x 32 k) of a stage: four MMAs per activation set.
-struct Frag { uint4 u0, v0, u1, v1; };
-__device__ __forceinline__ Frag load_frag(const unsigned char *a, int g, int row_stride) {
-    Frag f;
-    f.u0 = lds128(a + (size_t)g * row_stride);
-    f.v0 = lds128(a + (size_t)(g + 8) * row_stride);
-    f.u1 = lds128(a + (size_t)(g + 16) * row_stride);
-    f.v1 = lds128(a + (size_t)(g + 24) * row_stride);
-    return f;
-}
-__device__ __forceinline__ void mma_chunk(float (&acc)[2][2][4], const Frag &f, const uint4 &b) {
-    mma_bf16(acc[0][0], f.u0.x, f.v0.x, f.u0.y, f.v0.y, b.x, b.y);
-    mma_bf16(acc[1][0], f.u1.x, f.v1.x, f.u1.y, f.v1.y, b.x, b.y);
-    mma_bf16(acc[0][1], f.u0.z, f.v0.z, f.u0.w, f.v0.w, b.z, b.w);
-    mma_bf16(acc[1][1], f.u1.z, f.v1.z, f.u1.w, f.v1.w, b.z, b.w);
-}
-__device__ __forceinline__ uint4 load_act(const bf16_t *base, size_t off, bool in_smem) {
-    return in_smem ? lds128(base + off) : ldcg128(base + off);
-}
-
-// Runs all tiles of one phase for this CTA. `epi(vrow, col, v0, v1)` is called once per valid
-// (virtual row, activation row) by exactly one thread; v1 is the paired "up" value for GATEUP.
+// Runs all tiles of one matrix phase for this CTA and calls epilogue() once per valid (virtual
+// row, activation row), by exactly one thread. The kernel has a single call site per template
+// argument, so the streaming loop exists once in the instruction stream: this kernel is far
+// larger than the instruction cache and anything not in a loop is fetched from L2.
 //
 // MMA mapping: A = 16 weight rows x 16 k, B column 2r holds the hi part and column 2r+1 the lo
 // part of activation row r, so one MMA covers four activation rows exactly (the two columns are
 // added at the end); rows 4..7 use a second set of accumulators. The two halves of the consumer
 // warps (warps 0-3 / 4-7) take alternate stages, so each warp does four chunks per barrier wait
 // and two stages are in work at once.
-template <int KIND, bool two_sets, typename EpiF>
-__device__ __forceinline__ void consume_tiles(Cta &c, const ActSrc &act, int seg_stage, EpiF &epi) {
+template <bool two_sets>
+__device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActSrc &act, const int seg_stage, EpiCtx &ex) {
     const MegaParams &p = *c.p;
-    Geom geo = geom(c, KIND);
+    const Geom geo = geom(c, kind);
     const int R = p.R;
     const int g = c.lane >> 2, t = c.lane & 3;
     const int grp = c.warp >> 2, wi = c.warp & 3;
     const int arow = g >> 1;
     const bf16_t *abase = (g & 1) ? act.lo : act.hi;
-    const bool has0 = arow < R, has1 = arow + 4 < R;
+    const bool has0 = arow < R, has1 = two_sets && (arow + 4 < R);
     const size_t aoff0 = (size_t)arow * act.stride + t * 8, aoff1 = (size_t)(arow + 4) * act.stride + t * 8;
+    const uint32_t rs = (uint32_t)p.row_stride;
+    const uint4 zero = make_uint4(0, 0, 0, 0);
     for (int vr0 = geo.v0; vr0 < geo.v1; vr0 += geo.cap) {
-        int nv = min(geo.cap, geo.v1 - vr0);
+        const int nv = min(geo.cap, geo.v1 - vr0);
         float acc[2][2][4], acd[2][2][4], acc0[2][4], acd0[2][4];
 #pragma unroll
         for (int i = 0; i < 2; ++i)
@@ -353,41 +464,50 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const ActSrc &act, int seg
                 acc0[i][j] = acd0[i][j] = 0.f;
             }
         bool moved = false;
+        // which half of the warps takes a stage depends only on the stage's index within the phase,
+        // never on how many stages the CTA has seen before: the summation order of a row must not
+        // depend on the batch or on earlier calls
+        const int stage0 = ((vr0 - geo.v0) / geo.cap) * geo.nks;
+#pragma unroll 1
         for (int ks = 0; ks < geo.nks; ++ks) {
-            if ((int)(c.stage & 1u) == grp) {
-                int slot = c.stage % p.n_stages;
-                uint32_t parity = (c.stage / p.n_stages) & 1u;
+            if (((stage0 + ks) & 1) == grp) {
+                const int slot = c.stage % p.n_stages;
+                const uint32_t parity = (c.stage / p.n_stages) & 1u;
                 PROF_T0();
                 wait_bar(c, &c.misc->full[slot], parity);
                 PROF_ACC(c, 0, c.tid == 0);
-                if (KIND == PROJ && !moved && ks >= seg_stage) {   // second input segment starts: park the first
+                if (kind == PROJ && !moved && ks >= seg_stage) {   // second input segment starts: park the first
                     moved = true;
                     park<two_sets>(acc, acd, acc0, acd0);
                 }
                 const int klen = min(p.KC, geo.K - ks * p.KC);
                 const int nchunk = (klen + 31) >> 5;
-                const unsigned char *st = c.ring + (size_t)slot * p.stage_bytes + t * 16;
+                const uint32_t sb = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + t * 16 + g * rs;
                 const size_t kbase = (size_t)ks * p.KC;
-                const uint4 zero = make_uint4(0, 0, 0, 0);
-                // chunks wi, wi+4, wi+8, wi+12 in two batches of two: all loads of a batch are issued
-                // before its MMAs
-                for (int ch = wi; ch < nchunk; ch += 8) {
-                    const bool second = ch + 4 < nchunk;
-                    Frag f0 = load_frag(st + ch * 64, g, p.row_stride);
-                    uint4 b0 = has0 ? load_act(abase, aoff0 + kbase + ch * 32, act.in_smem) : zero;
-                    uint4 d0 = (two_sets && has1) ? load_act(abase, aoff1 + kbase + ch * 32, act.in_smem) : zero;
-                    Frag f1;
-                    uint4 b1 = zero, d1 = zero;
-                    if (second) {
-                        f1 = load_frag(st + (ch + 4) * 64, g, p.row_stride);
-                        if (has0) b1 = load_act(abase, aoff0 + kbase + (ch + 4) * 32, act.in_smem);
-                        if (two_sets && has1) d1 = load_act(abase, aoff1 + kbase + (ch + 4) * 32, act.in_smem);
-                    }
-                    mma_chunk(acc, f0, b0);
-                    if (two_sets) mma_chunk(acd, f0, d0);
-                    if (second) {
+                // chunks wi, wi+4, wi+8, wi+12
+                if (!two_sets && nchunk == 16 && act.in_smem) {
+                    // common case (full 512-wide stage, at most four activation rows staged in shared
+                    // memory): two batches of two chunks, all loads of a batch issued before its MMAs
+                    const uint32_t ab = smem_u32(abase + aoff0 + kbase);
+#pragma unroll
+                    for (int ch = wi; ch < 16; ch += 8) {
+                        uint4 b0 = zero, b1 = zero;
+                        Frag f0 = load_frag(sb + ch * 64, rs);
+                        if (has0) b0 = lds128_u32(ab + ch * 64);
+                        Frag f1 = load_frag(sb + (ch + 4) * 64, rs);
+                        if (has0) b1 = lds128_u32(ab + (ch + 4) * 64);
+                        mma_chunk(acc, f0, b0);
                         mma_chunk(acc, f1, b1);
-                        if (two_sets) mma_chunk(acd, f1, d1);
+                    }
+                } else {
+#pragma unroll 1
+                    for (int ch = wi; ch < nchunk; ch += 4) {
+                        Frag f0 = load_frag(sb + ch * 64, rs);
+                        uint4 b0 = zero, d0 = zero;
+                        if (has0) b0 = act.in_smem ? lds128(abase + aoff0 + kbase + ch * 32) : ldcg128(abase + aoff0 + kbase + ch * 32);
+                        if (has1) d0 = act.in_smem ? lds128(abase + aoff1 + kbase + ch * 32) : ldcg128(abase + aoff1 + kbase + ch * 32);
+                        mma_chunk(acc, f0, b0);
+                        if (two_sets) mma_chunk(acd, f0, d0);
                     }
                 }
                 __syncwarp();
@@ -397,7 +517,7 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const ActSrc &act, int seg
             c.stage++;
         }
         // a warp whose stages all lay in the first segment parks them now
-        if (KIND == PROJ && !moved) park<two_sets>(acc, acd, acc0, acd0);
+        if (kind == PROJ && !moved) park<two_sets>(acc, acd, acc0, acd0);
         // cross-warp reduction in a fixed order
         PROF_T0();
         float *red = c.red + (size_t)c.redbuf * kConsumerWarps * kTileRows * R + (size_t)c.warp * kTileRows * R;
@@ -409,12 +529,12 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const ActSrc &act, int seg
                 // activation row t (set 0) / t + 4 (set 1): hi column + lo column
                 if (t < R) {
                     float v = (acc[i][0][2 * h] + acc[i][0][2 * h + 1]) + (acc[i][1][2 * h] + acc[i][1][2 * h + 1]);
-                    if (KIND == PROJ) v = (acc0[i][2 * h] + acc0[i][2 * h + 1]) * c.misc->scale0[t] + v * c.misc->scale1[t];
+                    if (kind == PROJ) v = (acc0[i][2 * h] + acc0[i][2 * h + 1]) * c.misc->scale0[t] + v * c.misc->scale1[t];
                     red[row * R + t] = v;
                 }
                 if (two_sets && t + 4 < R) {
                     float v = (acd[i][0][2 * h] + acd[i][0][2 * h + 1]) + (acd[i][1][2 * h] + acd[i][1][2 * h + 1]);
-                    if (KIND == PROJ) v = (acd0[i][2 * h] + acd0[i][2 * h + 1]) * c.misc->scale0[t + 4] + v * c.misc->scale1[t + 4];
+                    if (kind == PROJ) v = (acd0[i][2 * h] + acd0[i][2 * h + 1]) * c.misc->scale0[t + 4] + v * c.misc->scale1[t + 4];
                     red[row * R + t + 4] = v;
                 }
             }
@@ -422,33 +542,22 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const ActSrc &act, int seg
         bar_sync(1, kConsumerThreads);
         {
             const float *rb = c.red + (size_t)c.redbuf * kConsumerWarps * kTileRows * R;
-            int row = c.tid >> 3, col = c.tid & 7;
-            if (KIND == GATEUP) {
-                if (row < 16 && row < nv && col < R) {
-                    float a = 0.f, b = 0.f;
-#pragma unroll
-                    for (int w = 0; w < kConsumerWarps; ++w) {
-                        a += rb[(size_t)w * kTileRows * R + row * R + col];
-                        b += rb[(size_t)w * kTileRows * R + (row + 16) * R + col];
-                    }
-                    epi(vr0 + row, col, a, b);
-                }
-            } else if (row < nv && col < R) {
-                float a = 0.f;
+            const int row = c.tid >> 3, col = c.tid & 7;
+            const int rlim = (kind == GATEUP) ? min(nv, 16) : nv;
+            if (row < rlim && col < R) {
+                float a = 0.f, b = 0.f;
 #pragma unroll
                 for (int w = 0; w < kConsumerWarps; ++w) a += rb[(size_t)w * kTileRows * R + row * R + col];
-                epi(vr0 + row, col, a, 0.f);
+                if (kind == GATEUP) {
+#pragma unroll
+                    for (int w = 0; w < kConsumerWarps; ++w) b += rb[(size_t)w * kTileRows * R + (row + 16) * R + col];
+                }
+                epilogue(c, kind, ex, vr0 + row, col, a, b);
             }
         }
         c.redbuf ^= 1;
         PROF_ACC(c, 4, c.tid == 0);
     }
-}
-
-template <int KIND, typename EpiF>
-__device__ __forceinline__ void consume_phase(Cta &c, const ActSrc &act, int seg_stage, EpiF &&epi) {
-    if (c.p->R > 4) consume_tiles<KIND, true>(c, act, seg_stage, epi);
-    else consume_tiles<KIND, false>(c, act, seg_stage, epi);
 }
 
 // Sum over CTAs of a per-CTA partial-sums-of-squares table [grid][8], for activation row `col`.
@@ -477,33 +586,6 @@ __device__ __forceinline__ void stage_hilo(const Cta &c, const bf16_t *ghi, cons
     }
 }
 
-// Block-wide sum of up to 2 values per activation row, all consumer threads participate.
-// Result for (col, which) is left in misc->ssred[0][col][which].
-__device__ __forceinline__ void block_sum2(const Cta &c, float (&v)[kMaxRows][2], int R) {
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-        for (int w = 0; w < 2; ++w) {
-            float s = v[r][w];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            if (c.lane == 0) c.misc->ssred[c.warp][r][w] = s;
-        }
-    bar_sync(1, kConsumerThreads);
-    if (c.tid < R * 2) {
-        int r = c.tid >> 1, w = c.tid & 1;
-        float s = 0.f;
-        for (int i = 0; i < kConsumerWarps; ++i) s += c.misc->ssred[i][r][w];
-        c.misc->ssred[0][r][w] = s;
-    }
-    bar_sync(1, kConsumerThreads);
-}
-
-// Per-thread accumulation of v^2 per activation row across the tiles of a phase, reduced over
-// the CTA's rows at phase end and written to this CTA's line of a partial table.
-struct SqAcc {
-    float a, b;
-    __device__ SqAcc() : a(0.f), b(0.f) {}
-};
 __device__ __forceinline__ void flush_sq(const Cta &c, const SqAcc &q, float *tblA, float *tblB) {
     // thread (row = tid>>3, col = tid&7)
     int row = c.tid >> 3, col = c.tid & 7;
@@ -521,49 +603,217 @@ __device__ __forceinline__ void flush_sq(const Cta &c, const SqAcc &q, float *tb
     }
 }
 
-__device__ __forceinline__ void store_split(bf16_t *hi, bf16_t *lo, size_t idx, float v) {
-    uint16_t h, l;
-    split_bf16(v, h, l);
-    hi[idx] = h;
-    lo[idx] = l;
+// ---- attention phase -------------------------------------------------------------------------
+// Rows r = b*M + m sit at position seq_lens[b] + posoff + m. The context of a sequence is cut
+// into fixed 64-token chunks from position 0; a work item is (sequence, KV head, chunk) and items
+// are dealt round-robin over the CTAs. A row's result therefore depends on its own position only.
+//
+// The producers stream the committed part of a chunk (positions below seq_lens[b], which nothing
+// in this launch writes) through the same ring as the weights: K rows at token*dh, V rows after
+// the 64 K rows. The consumers add the positions this launch produced (earlier draft steps from
+// the pages, this call's rows from the QKV scratch, rotated and rounded to bf16 exactly as they
+// are stored) into the same stage buffer and then work from shared memory only.
+// Scratch layout (floats): qs[M*Gq][dh] rotated, pre-scaled queries of one KV head;
+// wp[8 warps][Gq][dh + 2] per-warp partial (o, m, l) of the row being processed.
+
+// One chunk of one KV head from shared memory, for every row of the call: each warp takes 8 tokens.
+// Scores: lane = (token, quarter of the head dimension); the four quarters are added with two
+// shuffles. Softmax statistics are per warp (merged across warps, then across chunks, in fixed
+// order). P*V: lane owns DH/32 output elements, probabilities are broadcast by shuffle.
+// The loop over query heads is a real loop (not unrolled) to keep this once-per-step code small.
+template <int DH>
+__device__ __forceinline__ void attn_rows(Cta &c, const bf16_t *sk, const bf16_t *sv, const float *qs, float *wp,
+                                          int b, int kvh, int chunk, int base, int max_tokens) {
+    const MegaParams &p = *c.p;
+    constexpr int SEG = DH / 4, EPL = DH / 32, wstride = DH + 2;
+    const int Gq = p.Hq / p.Hkv, M = p.M;
+    const int c0 = chunk * kAttnChunk;
+    const int tl = c.warp * 8;                       // first token (within the chunk) of this warp
+    const int tkk = c.lane >> 2, part = c.lane & 3;
+    const int e0 = c.lane * EPL;
+    // this warp's K slice (token tkk, quarter `part`) and V rows (8 tokens x EPL elements) in registers
+    float kf[SEG], vf[8][EPL];
+    {
+        const uint4 *kr = reinterpret_cast<const uint4 *>(sk + (size_t)(tl + tkk) * DH + part * SEG);
+#pragma unroll
+        for (int i = 0; i < SEG / 8; ++i) {
+            uint4 w = kr[i];
+            kf[8 * i + 0] = bf16lo_f32(w.x); kf[8 * i + 1] = bf16hi_f32(w.x);
+            kf[8 * i + 2] = bf16lo_f32(w.y); kf[8 * i + 3] = bf16hi_f32(w.y);
+            kf[8 * i + 4] = bf16lo_f32(w.z); kf[8 * i + 5] = bf16hi_f32(w.z);
+            kf[8 * i + 6] = bf16lo_f32(w.w); kf[8 * i + 7] = bf16hi_f32(w.w);
+        }
+#pragma unroll
+        for (int tk = 0; tk < 8; ++tk) {
+            const bf16_t *vr = sv + (size_t)(tl + tk) * DH + e0;
+            if (EPL == 4) {
+                uint2 w = *reinterpret_cast<const uint2 *>(vr);
+                vf[tk][0] = bf16lo_f32(w.x); vf[tk][1] = bf16hi_f32(w.x); vf[tk][EPL - 2] = bf16lo_f32(w.y); vf[tk][EPL - 1] = bf16hi_f32(w.y);
+            } else {
+                uint32_t w = *reinterpret_cast<const uint32_t *>(vr);
+                vf[tk][0] = bf16lo_f32(w); vf[tk][1] = bf16hi_f32(w);
+            }
+        }
+    }
+#pragma unroll 1
+    for (int m = 0; m < M; ++m) {
+        const int npos = min(base + m, max_tokens - 1);   // last visible position of this row
+        const int nvis = min(8, npos - (c0 + tl) + 1);    // visible tokens of this warp (may be <= 0)
+#pragma unroll 1
+        for (int h = 0; h < Gq; ++h) {
+            float s = 0.f;
+            const float4 *qv = reinterpret_cast<const float4 *>(qs + (size_t)(m * Gq + h) * DH + part * SEG);
+#pragma unroll
+            for (int i = 0; i < SEG / 4; ++i) {
+                float4 q4 = qv[i];
+                s += q4.x * kf[4 * i] + q4.y * kf[4 * i + 1];
+                s += q4.z * kf[4 * i + 2] + q4.w * kf[4 * i + 3];
+            }
+            s += __shfl_xor_sync(0xffffffffu, s, 1);
+            s += __shfl_xor_sync(0xffffffffu, s, 2);
+            if (tkk >= nvis) s = -INFINITY;
+            float mx = s;
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+            const float pe = (s == -INFINITY) ? 0.f : expf(s - mx);
+            float sm = pe;
+            sm += __shfl_xor_sync(0xffffffffu, sm, 4);
+            sm += __shfl_xor_sync(0xffffffffu, sm, 8);
+            sm += __shfl_xor_sync(0xffffffffu, sm, 16);
+            // o[e] = sum over the warp's tokens (ascending) of p * V
+            float o[EPL];
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) o[e] = 0.f;
+#pragma unroll
+            for (int tk = 0; tk < 8; ++tk) {
+                const float pr = __shfl_sync(0xffffffffu, pe, tk * 4);
+                if (tk < nvis) {
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) o[e] += pr * vf[tk][e];
+                }
+            }
+            float *w = wp + ((size_t)c.warp * Gq + h) * wstride;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) w[e0 + e] = o[e];
+            if (c.lane == 0) { w[DH] = mx; w[DH + 1] = sm; }
+        }
+        bar_sync(1, kConsumerThreads);
+        // ---- merge the 8 warps (fixed order) -> chunk partial in global memory
+        for (int i = c.tid; i < Gq * DH; i += kConsumerThreads) {
+            int h = i / DH, e = i - h * DH;
+            float mx = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w) mx = fmaxf(mx, wp[((size_t)w * Gq + h) * wstride + DH]);
+            float ov = 0.f, l = 0.f;
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w) {
+                const float *pw = wp + ((size_t)w * Gq + h) * wstride;
+                float f = (pw[DH] == -INFINITY) ? 0.f : expf(pw[DH] - mx);
+                ov += f * pw[e];
+                l += f * pw[DH + 1];
+            }
+            int r = b * M + m, hq = kvh * Gq + h;
+            float *dst = p.s.att_part + (((size_t)r * p.Hq + hq) * p.max_chunks + chunk) * wstride;
+            dst[e] = ov;
+            if (e == 0) { dst[DH] = mx; dst[DH + 1] = l; }
+        }
+        bar_sync(1, kConsumerThreads);
+    }
 }
 
-// ---- attention phase -------------------------------------------------------------------------
-// Rows r = b*M + m sit at position seq_lens[b] + posoff + m. Scratch layout (floats):
-//   qs[M*Gq][dh]  rotated, pre-scaled queries of one KV head
-//   kn[M][dh], vn[M][dh]  this call's new keys / values (after bf16 rounding)
-//   wp[8 warps][Gq][dh + 2] per-warp partial (o, m, l) for the row being processed
+struct AttnItem { int b, kvh, chunk, Lb, nch; };
+
+__device__ __forceinline__ int attn_total(const MegaParams &p, const KvPtrs &kv, int posoff) {
+    int total = 0;
+    for (int b = 0; b < p.B; ++b) total += p.Hkv * ((kv.seq_lens[b] + posoff + p.M - 1) / kAttnChunk + 1);
+    return total;
+}
+__device__ __forceinline__ AttnItem attn_item(const MegaParams &p, const KvPtrs &kv, int posoff, int item) {
+    AttnItem it;
+    int b = 0, rem = item, Lb = 0, nch = 1;
+    for (; b < p.B; ++b) {
+        Lb = kv.seq_lens[b];
+        nch = (Lb + posoff + p.M - 1) / kAttnChunk + 1;
+        if (rem < p.Hkv * nch) break;
+        rem -= p.Hkv * nch;
+    }
+    it.b = b; it.Lb = Lb; it.nch = nch;
+    it.kvh = rem / nch;
+    it.chunk = rem - it.kvh * nch;
+    return it;
+}
+
+__device__ __forceinline__ void produce_attention(Cta &c, const KvPtrs &kv, int posoff) {
+    const MegaParams &p = *c.p;
+    const int ptid = c.tid - kConsumerThreads;               // 0 .. 127
+    const int upt = p.dh >> 3;                                // 16-byte units per token row
+    const int total = attn_total(p, kv, posoff);
+    for (int item = c.cta; item < total; item += c.grid) {
+        const AttnItem it = attn_item(p, kv, posoff, item);
+        const int c0 = it.chunk * kAttnChunk;
+        const int n_old = max(0, min(kAttnChunk, it.Lb - c0));   // committed tokens of this chunk
+        const int32_t *bt = kv.block_table + (size_t)it.b * kv.max_pages;
+        int slot = c.stage % p.n_stages;
+        uint32_t parity = (c.stage / p.n_stages) & 1u;
+        bool ok = true;
+        if (c.lane == 0) ok = wait_bar(c, &c.misc->empty[slot], parity ^ 1u);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) return;
+        const uint32_t dst0 = smem_u32(c.ring + (size_t)slot * p.stage_bytes);
+        const int nunits = n_old * upt;
+        // four units per round so that the copies in flight use distinct address registers
+        for (int u0 = ptid; u0 < nunits; u0 += 4 * kProducerWarps * 32) {
+            uint32_t d[4];
+            const unsigned char *qk[4], *qv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                int u = u0 + i * kProducerWarps * 32;
+                int tok = min(u / upt, n_old - 1), w = u % upt;
+                int j = c0 + tok;
+                int page = bt[j / p.page];
+                if ((unsigned)page >= (unsigned)kv.num_pages) { raise(c, kDevBadPage); page = 0; }
+                size_t off = ((((size_t)page * p.Hkv + it.kvh) * p.page + (j % p.page)) * p.dh) * 2 + (size_t)w * 16;
+                d[i] = dst0 + (uint32_t)(tok * p.dh * 2 + w * 16);
+                qk[i] = reinterpret_cast<const unsigned char *>(kv.k_pages) + off;
+                qv[i] = reinterpret_cast<const unsigned char *>(kv.v_pages) + off;
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (u0 + i * kProducerWarps * 32 < nunits) {
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d[i]), "l"(qk[i]) : "memory");
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d[i] + (uint32_t)(kAttnChunk * p.dh * 2)), "l"(qv[i]) : "memory");
+                }
+            }
+        }
+        cp_async_arrive(&c.misc->full[slot]);
+        c.stage++;
+    }
+}
+
 __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int posoff) {
     const MegaParams &p = *c.p;
     const int dh = p.dh, half = dh >> 1, Gq = p.Hq / p.Hkv, M = p.M;
-    const int epl = dh >> 5;   // elements per lane (2 or 4)
     float *qs = reinterpret_cast<float *>(c.scr);
-    float *kn = qs + (size_t)M * Gq * dh;
-    float *vn = kn + (size_t)M * dh;
-    float *wp = vn + (size_t)M * dh;
+    float *wp = qs + (size_t)M * Gq * dh;
     const int wstride = dh + 2;
     const float qscale = rsqrtf((float)dh);
     const int max_tokens = min(kv.max_pages * p.page, p.max_ctx);   // positions beyond are flagged, not touched
+    const int upt = dh >> 3;
 
-    // work list: per sequence Hkv * nch items
-    int total = 0;
-    for (int b = 0; b < p.B; ++b) {
-        int last = kv.seq_lens[b] + posoff + M - 1;
-        total += p.Hkv * (last / kAttnChunk + 1);
-    }
+    const int total = attn_total(p, kv, posoff);
     for (int item = c.cta; item < total; item += c.grid) {
-        int b = 0, rem = item, Lb = 0, nch = 1;
-        for (; b < p.B; ++b) {
-            Lb = kv.seq_lens[b];
-            nch = (Lb + posoff + M - 1) / kAttnChunk + 1;
-            if (rem < p.Hkv * nch) break;
-            rem -= p.Hkv * nch;
-        }
-        const int kvh = rem / nch, chunk = rem - kvh * nch;
+        const AttnItem it = attn_item(p, kv, posoff, item);
+        const int b = it.b, kvh = it.kvh, chunk = it.chunk, Lb = it.Lb, nch = it.nch;
         const int base = Lb + posoff;              // position of row m = 0
+        const int c0 = chunk * kAttnChunk;
         const int32_t *bt = kv.block_table + (size_t)b * kv.max_pages;
+        const int slot = c.stage % p.n_stages;
+        const uint32_t parity = (c.stage / p.n_stages) & 1u;
+        bf16_t *sk = reinterpret_cast<bf16_t *>(c.ring + (size_t)slot * p.stage_bytes);
+        bf16_t *sv = sk + (size_t)kAttnChunk * dh;
 
-        // -- stage rotated queries and the new K/V of this KV head
+        // -- rotated, pre-scaled queries of this KV head (independent of the stage)
         for (int i = c.tid; i < M * Gq * half; i += kConsumerThreads) {
             int qi = i / half, e = i - qi * half;
             int m = qi / Gq, hq = kvh * Gq + (qi - m * Gq);
@@ -575,154 +825,52 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
             qs[qi * dh + e] = (x * cs - y * sn) * qscale;
             qs[qi * dh + e + half] = (y * cs + x * sn) * qscale;
         }
+        PROF(c);
+        wait_bar(c, &c.misc->full[slot], parity);
+        PROF(c);
+        // -- positions written earlier in this launch (previous draft steps): from the pages
+        {
+            const int lo = max(Lb, c0), hi = min(min(base, c0 + kAttnChunk), max_tokens);
+            for (int i = c.tid; i < (hi - lo) * upt; i += kConsumerThreads) {
+                int tk = i / upt, w = i - tk * upt, j = lo + tk;
+                int page = bt[j / p.page];
+                if ((unsigned)page >= (unsigned)kv.num_pages) { raise(c, kDevBadPage); page = 0; }
+                size_t off = (((size_t)page * p.Hkv + kvh) * p.page + (j % p.page)) * dh + (size_t)w * 8;
+                *reinterpret_cast<uint4 *>(sk + (size_t)(j - c0) * dh + w * 8) = ldcg128(kv.k_pages + off);
+                *reinterpret_cast<uint4 *>(sv + (size_t)(j - c0) * dh + w * 8) = ldcg128(kv.v_pages + off);
+            }
+        }
+        // -- this call's rows: rotate, round to bf16, put into the stage and append to the cache
         for (int i = c.tid; i < M * half; i += kConsumerThreads) {
             int m = i / half, e = i - m * half;
             int r = b * M + m, pos = base + m;
-            bool pos_ok = pos < max_tokens;
-            if (!pos_ok) { raise(c, kDevBadPos); pos = max_tokens - 1; }
+            if (pos >= max_tokens) { if (chunk == 0) raise(c, kDevBadPos); continue; }
+            if (pos < c0 || pos >= c0 + kAttnChunk) continue;     // another chunk's item owns it
             const float *kk = p.s.qkv + (size_t)r * (p.qdim + 2 * p.kvdim) + p.qdim + kvh * dh;
             const float *vv = kk + p.kvdim;
             float x = ldcg_f32(kk + e), y = ldcg_f32(kk + e + half);
             float cs = p.s.rope_cos[(size_t)pos * half + e], sn = p.s.rope_sin[(size_t)pos * half + e];
             uint16_t k0 = f32_bf16bits(x * cs - y * sn), k1 = f32_bf16bits(y * cs + x * sn);
             uint16_t v0 = f32_bf16bits(ldcg_f32(vv + e)), v1 = f32_bf16bits(ldcg_f32(vv + e + half));
-            kn[m * dh + e] = bf16bits_f32(k0);
-            kn[m * dh + e + half] = bf16bits_f32(k1);
-            vn[m * dh + e] = bf16bits_f32(v0);
-            vn[m * dh + e + half] = bf16bits_f32(v1);
-            if (pos_ok && pos / kAttnChunk == chunk) {   // the item that owns this position appends it
-                int page = bt[pos / p.page];
-                if ((unsigned)page >= (unsigned)kv.num_pages) { raise(c, kDevBadPage); page = 0; }
-                size_t o = (((size_t)page * p.Hkv + kvh) * p.page + (pos % p.page)) * dh;
-                kv.k_pages[o + e] = k0;
-                kv.k_pages[o + e + half] = k1;
-                kv.v_pages[o + e] = v0;
-                kv.v_pages[o + e + half] = v1;
-            }
+            bf16_t *dk = sk + (size_t)(pos - c0) * dh, *dv = sv + (size_t)(pos - c0) * dh;
+            dk[e] = k0; dk[e + half] = k1; dv[e] = v0; dv[e + half] = v1;
+            int page = bt[pos / p.page];
+            if ((unsigned)page >= (unsigned)kv.num_pages) { raise(c, kDevBadPage); page = 0; }
+            size_t o = (((size_t)page * p.Hkv + kvh) * p.page + (pos % p.page)) * dh;
+            kv.k_pages[o + e] = k0;
+            kv.k_pages[o + e + half] = k1;
+            kv.v_pages[o + e] = v0;
+            kv.v_pages[o + e + half] = v1;
         }
         bar_sync(1, kConsumerThreads);
+        PROF(c);
 
-        const int j0 = chunk * kAttnChunk + c.warp * 16;     // this warp's 16 tokens
-        const int e0 = c.lane * epl;
-        for (int m = 0; m < M; ++m) {
-            const int npos = min(base + m, max_tokens - 1);  // last visible position of this row
-            float q[8][4];
-#pragma unroll
-            for (int h = 0; h < 8; ++h)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) q[h][e] = (h < Gq && e < epl) ? qs[(m * Gq + h) * dh + e0 + e] : 0.f;
-            float sc[8];
-#pragma unroll
-            for (int h = 0; h < 8; ++h) sc[h] = -INFINITY;
-            // pass 1: scores; lane `tk` keeps the score of token j0 + tk
-            for (int tk = 0; tk < 16; ++tk) {
-                int j = j0 + tk;
-                if (j > npos) break;
-                float kf[4] = {0.f, 0.f, 0.f, 0.f};
-                if (j >= base) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) if (e < epl) kf[e] = kn[(j - base) * dh + e0 + e];
-                } else {
-                    int page = bt[j / p.page];
-                    if ((unsigned)page >= (unsigned)kv.num_pages) { raise(c, kDevBadPage); page = 0; }
-                    const bf16_t *kr = kv.k_pages + (((size_t)page * p.Hkv + kvh) * p.page + (j % p.page)) * dh + e0;
-                    if (epl == 4) {
-                        uint2 w = ldcg64(kr);
-                        kf[0] = bf16lo_f32(w.x); kf[1] = bf16hi_f32(w.x); kf[2] = bf16lo_f32(w.y); kf[3] = bf16hi_f32(w.y);
-                    } else {
-                        uint32_t w = ldcg_u32(kr);
-                        kf[0] = bf16lo_f32(w); kf[1] = bf16hi_f32(w);
-                    }
-                }
-#pragma unroll
-                for (int h = 0; h < 8; ++h) {
-                    if (h < Gq) {
-                        float s = q[h][0] * kf[0] + q[h][1] * kf[1];
-                        s += q[h][2] * kf[2] + q[h][3] * kf[3];
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-                        if (c.lane == tk) sc[h] = s;
-                    }
-                }
-            }
-            // softmax statistics over the warp's tokens
-            float mw[8], lw[8], pj[8];
-#pragma unroll
-            for (int h = 0; h < 8; ++h) {
-                float mx = sc[h];
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                mw[h] = mx;
-                pj[h] = (sc[h] == -INFINITY) ? 0.f : expf(sc[h] - mx);
-                float sm = pj[h];
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, o);
-                lw[h] = sm;
-            }
-            // pass 2: o[h][e] = sum_j p_j V[j][e]
-            float o[8][4];
-#pragma unroll
-            for (int h = 0; h < 8; ++h)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) o[h][e] = 0.f;
-            for (int tk = 0; tk < 16; ++tk) {
-                int j = j0 + tk;
-                if (j > npos) break;
-                float vf[4] = {0.f, 0.f, 0.f, 0.f};
-                if (j >= base) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) if (e < epl) vf[e] = vn[(j - base) * dh + e0 + e];
-                } else {
-                    int page = bt[j / p.page];
-                    if ((unsigned)page >= (unsigned)kv.num_pages) page = 0;
-                    const bf16_t *vr = kv.v_pages + (((size_t)page * p.Hkv + kvh) * p.page + (j % p.page)) * dh + e0;
-                    if (epl == 4) {
-                        uint2 w = ldcg64(vr);
-                        vf[0] = bf16lo_f32(w.x); vf[1] = bf16hi_f32(w.x); vf[2] = bf16lo_f32(w.y); vf[3] = bf16hi_f32(w.y);
-                    } else {
-                        uint32_t w = ldcg_u32(vr);
-                        vf[0] = bf16lo_f32(w); vf[1] = bf16hi_f32(w);
-                    }
-                }
-#pragma unroll
-                for (int h = 0; h < 8; ++h) {
-                    if (h < Gq) {
-                        float pr = __shfl_sync(0xffffffffu, pj[h], tk);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) o[h][e] += pr * vf[e];
-                    }
-                }
-            }
-            // per-warp partial -> shared
-#pragma unroll
-            for (int h = 0; h < 8; ++h) {
-                if (h < Gq) {
-                    float *w = wp + ((size_t)c.warp * Gq + h) * wstride;
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) if (e < epl) w[e0 + e] = o[h][e];
-                    if (c.lane == 0) { w[dh] = mw[h]; w[dh + 1] = lw[h]; }
-                }
-            }
-            bar_sync(1, kConsumerThreads);
-            // merge the 8 warps (fixed order) -> chunk partial in global memory
-            for (int i = c.tid; i < Gq * dh; i += kConsumerThreads) {
-                int h = i / dh, e = i - h * dh;
-                float mx = -INFINITY;
-                for (int w = 0; w < kConsumerWarps; ++w) mx = fmaxf(mx, wp[((size_t)w * Gq + h) * wstride + dh]);
-                float ov = 0.f, l = 0.f;
-                for (int w = 0; w < kConsumerWarps; ++w) {
-                    const float *pw = wp + ((size_t)w * Gq + h) * wstride;
-                    float f = (pw[dh] == -INFINITY) ? 0.f : expf(pw[dh] - mx);
-                    ov += f * pw[e];
-                    l += f * pw[dh + 1];
-                }
-                int r = b * M + m, hq = kvh * Gq + h;
-                float *dst = p.s.att_part + (((size_t)r * p.Hq + hq) * p.max_chunks + chunk) * wstride;
-                dst[e] = ov;
-                if (e == 0) { dst[dh] = mx; dst[dh + 1] = l; }
-            }
-            bar_sync(1, kConsumerThreads);
-        }
+        if (dh == 128) attn_rows<128>(c, sk, sv, qs, wp, b, kvh, chunk, base, max_tokens);
+        else attn_rows<64>(c, sk, sv, qs, wp, b, kvh, chunk, base, max_tokens);
+        PROF(c);
+        // the stage is free again (all consumer warps passed the barrier at the end of attn_rows)
+        if (c.warp < kConsumerWarps / 2 && c.lane == 0) mbar_arrive(&c.misc->empty[slot]);
+        c.stage++;
         // -- last CTA of this (sequence, KV head) merges the chunks
         __threadfence();
         bar_sync(1, kConsumerThreads);
@@ -740,8 +888,10 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
                 const float *src = p.s.att_part + ((size_t)r * p.Hq + hq) * p.max_chunks * wstride;
                 int ncm = min(base + m, max_tokens - 1) / kAttnChunk + 1;   // chunks visible to this row
                 float mx = -INFINITY;
+#pragma unroll 8
                 for (int ch = 0; ch < ncm; ++ch) mx = fmaxf(mx, ldcg_f32(src + (size_t)ch * wstride + dh));
                 float ov = 0.f, l = 0.f;
+#pragma unroll 4
                 for (int ch = 0; ch < ncm; ++ch) {
                     float mc = ldcg_f32(src + (size_t)ch * wstride + dh);
                     float f = (mc == -INFINITY) ? 0.f : expf(mc - mx);
@@ -801,39 +951,72 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
     const bool is_producer = (c.warp >= kConsumerWarps);
     const int R = p.R;
     const int n_steps = (p.mode == 0) ? p.K : 1;
-    const int n_layers = (p.mode == 0) ? 1 : p.n_layers;
 
     if (is_producer) {
         setmaxnreg_dec<kProducerRegs>();
-        // ---------------- producer: the weight stream of every phase, in program order
-        for (int step = 0; step < n_steps; ++step) {
-            if (p.mode == 0) produce_phase(c, PROJ, p.layers[0]);
-            for (int l = 0; l < n_layers; ++l) {
-                produce_phase(c, QKV, p.layers[l]);
-                produce_phase(c, OPROJ, p.layers[l]);
-                produce_phase(c, GATEUP, p.layers[l]);
-                produce_phase(c, DOWN, p.layers[l]);
-            }
-            produce_phase(c, HEAD, p.layers[0]);
+        // ---------------- producers: the weight / KV stream of every phase, in program order
+        Prog g;
+        for (prog_begin(p, g); g.kind != DONE; prog_next(p, g)) {
+            if (g.kind == ATTN) produce_attention(c, p.kvs[g.layer], (p.mode == 0) ? g.step : 0);
+            else if (g.kind != EMBED) produce_phase(c, g.kind, p.layers[g.layer]);
         }
         cp_async_wait_all();   // every copy this thread issued has landed before the CTA may exit
         PROF_FLUSH(c, 2, 4, c.warp == kConsumerWarps && c.lane == 0);
         return;
     }
 
-    // ---------------- consumers
+    // ---------------- consumers: one loop over the phase program; every phase ends in a grid barrier
     setmaxnreg_inc<kConsumerRegs>();
     bf16_t *s_hi = reinterpret_cast<bf16_t *>(c.scr);
-    const int KCd = p.KC;
-    auto act_stride = [&](int len) { return ((len + 31) & ~31) + 32; };   // +64 B: rows land in different banks
-
-    for (int step = 0; step < n_steps; ++step) {
+    EpiCtx ex;
+    ex.best = 0ull;
+    Prog g;
+#pragma unroll 1
+    for (prog_begin(p, g); g.kind != DONE; prog_next(p, g)) {
+        const int kind = g.kind, step = g.step;
+        const LayerPtrs &L = p.layers[g.layer];
+        const bool last_layer = (p.mode == 0) || (g.layer + 1 == p.n_layers);
+        ex.sq.a = 0.f; ex.sq.b = 0.f;
+        ex.L = &L;
+        ex.step = step;
+        ex.to_next_layer = (p.mode == 1) && !last_layer;
+        ex.gnext = ex.to_next_layer ? p.layers[g.layer + 1].g_in : p.g_final;
         PROF(c);
-        // ============ front end
-        if (p.mode == 0) {
-            // ---- PROJ: x0 = W_p [ rms(h) ; rms(Emb(tok)) ]
-            const int st = act_stride(2 * p.d);
-            bf16_t *a_hi = s_hi, *a_lo = s_hi + (size_t)R * st;
+        if (kind == ATTN) {
+            attention_phase(c, p.kvs[g.layer], (p.mode == 0) ? step : 0);
+            PROF(c);
+            grid_barrier(c);
+            continue;
+        }
+        if (kind == EMBED) {
+            // ---- target: x0 = Emb(tok), CTA-sliced over d; thread = (row slot tid>>3, activation row tid&7)
+            int r0 = (int)(((long long)c.cta * p.d) / c.grid), r1 = (int)(((long long)(c.cta + 1) * p.d) / c.grid);
+            for (int row = r0 + (c.tid >> 3); row < r1; row += kTileRows) {
+                int col = c.tid & 7;
+                if (col < R) {
+                    int tok = p.tokens[col];
+                    if ((unsigned)tok >= (unsigned)p.V) { raise(c, kDevBadToken); tok = 0; }
+                    float v = bf16bits_f32(p.embed[(size_t)tok * p.d + row]);
+                    p.s.x0[(size_t)col * p.d + row] = v;
+                    store_split(p.s.actD_hi, p.s.actD_lo, (size_t)col * p.dp + row, v * bf16bits_f32(L.g_in[row]));
+                    ex.sq.a += v * v;
+                }
+            }
+            flush_sq(c, ex.sq, p.s.ssA, nullptr);
+            PROF(c);
+            grid_barrier(c);
+            continue;
+        }
+
+        // ============ matrix phases: stage the input vector(s) in shared memory ...
+        const int klen = (kind == PROJ) ? 2 * p.d : (kind == OPROJ) ? p.qdim : (kind == DOWN) ? p.F : p.d;
+        const int st = ((klen + 31) & ~31) + 32;      // +64 B: rows land in different banks
+        bf16_t *a_hi = s_hi, *a_lo = s_hi + (size_t)R * st;
+        ActSrc act{a_hi, a_lo, st, true};
+        int seg = 0;
+        if (kind == PROJ) {
+            // ---- x0 = W_p [ rms(h) ; rms(Emb(tok)) ]
+            seg = p.d / p.KC;
             if (c.tid < R) {
                 int tok;
                 if (step == 0) tok = p.tokens[c.tid];
@@ -847,9 +1030,10 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                 c.misc->tok[c.tid] = tok;
             }
             bar_sync(1, kConsumerThreads);
-            float sq[kMaxRows][2];
-            for (int r = 0; r < R; ++r) { sq[r][0] = 0.f; sq[r][1] = 0.f; }
+            if (step > 0) stage_hilo(c, p.s.actR_hi, p.s.actR_lo, p.dp, p.d, a_hi, a_lo, st, 0);
+#pragma unroll 1
             for (int r = 0; r < R; ++r) {
+                float sqh = 0.f, sqe = 0.f;
                 const bf16_t *erow = p.embed + (size_t)c.misc->tok[r] * p.d;
                 for (int k = c.tid * 8; k < p.d; k += kConsumerThreads * 8) {
                     uint4 ev = ldnc128(erow + k);
@@ -858,7 +1042,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         float e0 = bf16lo_f32(ew[i]), e1 = bf16hi_f32(ew[i]);
-                        sq[r][1] += e0 * e0 + e1 * e1;
+                        sqe += e0 * e0 + e1 * e1;
                         store_split(a_hi, a_lo, (size_t)r * st + p.d + k + 2 * i, e0 * bf16lo_f32(gw[i]));
                         store_split(a_hi, a_lo, (size_t)r * st + p.d + k + 2 * i + 1, e1 * bf16hi_f32(gw[i]));
                     }
@@ -869,15 +1053,21 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             float h0 = bf16lo_f32(hw[i]), h1 = bf16hi_f32(hw[i]);
-                            sq[r][0] += h0 * h0 + h1 * h1;
+                            sqh += h0 * h0 + h1 * h1;
                             store_split(a_hi, a_lo, (size_t)r * st + k + 2 * i, h0 * bf16lo_f32(hgw[i]));
                             store_split(a_hi, a_lo, (size_t)r * st + k + 2 * i + 1, h1 * bf16hi_f32(hgw[i]));
                         }
                     }
                 }
+                // block sums of the two squared norms of row r
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    sqh += __shfl_xor_sync(0xffffffffu, sqh, o);
+                    sqe += __shfl_xor_sync(0xffffffffu, sqe, o);
+                }
+                if (c.lane == 0) { c.misc->ssred[c.warp][r][0] = sqh; c.misc->ssred[c.warp][r][1] = sqe; }
             }
-            if (step > 0) stage_hilo(c, p.s.actR_hi, p.s.actR_lo, p.dp, p.d, a_hi, a_lo, st, 0);
-            block_sum2(c, sq, R);
+            bar_sync(1, kConsumerThreads);
             if (step > 0 && c.warp < R) {
                 // recursed state: h = (x2*g_final) * s_x; rms(h) adds s_h = rsqrt(s_x^2 * mean((x2 g)^2) + eps)
                 float sx = rsqrtf(sum_partials(c, p.s.ssC, c.warp) / (float)p.d + p.eps);
@@ -885,213 +1075,70 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                 if (c.lane == 0) c.misc->scale0[c.warp] = sx * rsqrtf(sx * sx * sy + p.eps);
             }
             if (c.tid < R) {
-                if (step == 0) c.misc->scale0[c.tid] = rsqrtf(c.misc->ssred[0][c.tid][0] / (float)p.d + p.eps);
-                c.misc->scale1[c.tid] = rsqrtf(c.misc->ssred[0][c.tid][1] / (float)p.d + p.eps);
+                float sh = 0.f, se = 0.f;
+                for (int i = 0; i < kConsumerWarps; ++i) { sh += c.misc->ssred[i][c.tid][0]; se += c.misc->ssred[i][c.tid][1]; }
+                if (step == 0) c.misc->scale0[c.tid] = rsqrtf(sh / (float)p.d + p.eps);
+                c.misc->scale1[c.tid] = rsqrtf(se / (float)p.d + p.eps);
             }
-            bar_sync(1, kConsumerThreads);
-            SqAcc sqa;
-            ActSrc act{a_hi, a_lo, st, true};
-            const LayerPtrs &L0 = p.layers[0];
-            PROF(c);
-            consume_phase<PROJ>(c, act, p.d / KCd, [&](int row, int col, float v, float) {
-                p.s.x0[(size_t)col * p.d + row] = v;
-                store_split(p.s.actD_hi, p.s.actD_lo, (size_t)col * p.dp + row, v * bf16bits_f32(L0.g_in[row]));
-                sqa.a += v * v;
-            });
-            flush_sq(c, sqa, p.s.ssA, nullptr);
-            PROF(c);
-            grid_barrier(c);
-            PROF(c);
         } else {
-            // ---- EMBED (target): x0 = Emb(tok), CTA-sliced over d
+            // ---- the previous phase's output vector (hi/lo) and the sum of squares that normalises it
+            const bf16_t *ghi, *glo;
+            const float *sstab = nullptr;
+            int gstride = p.dp, glen = p.d;
+            switch (kind) {
+                case QKV:    ghi = p.s.actD_hi; glo = p.s.actD_lo; sstab = p.s.ssA; break;
+                case OPROJ:  ghi = p.s.actO_hi; glo = p.s.actO_lo; gstride = p.qp; glen = p.qdim; break;
+                case GATEUP: ghi = p.s.actP_hi; glo = p.s.actP_lo; sstab = p.s.ssB; break;
+                case DOWN:   ghi = p.s.actF_hi; glo = p.s.actF_lo; gstride = p.Fp; glen = p.Fp; break;   // pad beyond F is zero
+                default:     ghi = p.s.actH_hi; glo = p.s.actH_lo; sstab = p.s.ssC; break;               // HEAD
+            }
+            if (kind == DOWN && !p.stage_F_in_smem) act = ActSrc{ghi, glo, gstride, false};
+            else stage_hilo(c, ghi, glo, gstride, glen, a_hi, a_lo, st, 0);
+            if (sstab && c.warp < R) {
+                float sc = rsqrtf(sum_partials(c, sstab, c.warp) / (float)p.d + p.eps);
+                if (c.lane == 0) c.misc->scale0[c.warp] = sc;
+            }
+        }
+        bar_sync(1, kConsumerThreads);
+        if (kind == HEAD && p.out_h) {   // every CTA writes its slice of the post-final-norm hidden state
             int r0 = (int)(((long long)c.cta * p.d) / c.grid), r1 = (int)(((long long)(c.cta + 1) * p.d) / c.grid);
-            // thread = (row slot tid>>3, activation row tid&7)
-            SqAcc sqa;
-            for (int row = r0 + (c.tid >> 3); row < r1; row += kTileRows) {
-                int col = c.tid & 7;
-                if (col < R) {
-                    int tok = p.tokens[col];
-                    if ((unsigned)tok >= (unsigned)p.V) { raise(c, kDevBadToken); tok = 0; }
-                    float v = bf16bits_f32(p.embed[(size_t)tok * p.d + row]);
-                    p.s.x0[(size_t)col * p.d + row] = v;
-                    store_split(p.s.actD_hi, p.s.actD_lo, (size_t)col * p.dp + row,
-                                v * bf16bits_f32(p.layers[0].g_in[row]));
-                    sqa.a += v * v;
-                }
-            }
-            flush_sq(c, sqa, p.s.ssA, nullptr);
-            grid_barrier(c);
-        }
-
-        // ============ decoder layers
-        for (int l = 0; l < n_layers; ++l) {
-            const LayerPtrs &L = p.layers[l];
-            const bool last_layer = (l + 1 == n_layers);
-            // ---- QKV
-            {
-                const int st = act_stride(p.d);
-                bf16_t *a_hi = s_hi, *a_lo = s_hi + (size_t)R * st;
-                stage_hilo(c, p.s.actD_hi, p.s.actD_lo, p.dp, p.d, a_hi, a_lo, st, 0);
-                if (c.warp < R) {
-                    float s = rsqrtf(sum_partials(c, p.s.ssA, c.warp) / (float)p.d + p.eps);
-                    if (c.lane == 0) c.misc->scale0[c.warp] = s;
-                }
-                bar_sync(1, kConsumerThreads);
-                ActSrc act{a_hi, a_lo, st, true};
-                const int nq = p.qdim + 2 * p.kvdim;
-                PROF(c);
-                consume_phase<QKV>(c, act, 0, [&](int row, int col, float v, float) {
-                    p.s.qkv[(size_t)col * nq + row] = v * c.misc->scale0[col];
-                });
-                PROF(c);
-                grid_barrier(c);
-                PROF(c);
-            }
-            // ---- attention
-            attention_phase(c, p.kvs[l], (p.mode == 0) ? step : 0);
-            PROF(c);
-            grid_barrier(c);
-            PROF(c);
-            // ---- O projection + residual
-            {
-                const int st = act_stride(p.qdim);
-                bf16_t *a_hi = s_hi, *a_lo = s_hi + (size_t)R * st;
-                stage_hilo(c, p.s.actO_hi, p.s.actO_lo, p.qp, p.qdim, a_hi, a_lo, st, 0);
-                bar_sync(1, kConsumerThreads);
-                ActSrc act{a_hi, a_lo, st, true};
-                SqAcc sqa;
-                PROF(c);
-                consume_phase<OPROJ>(c, act, 0, [&](int row, int col, float v, float) {
-                    float x = ldcg_f32(p.s.x0 + (size_t)col * p.d + row) + v;
-                    p.s.x1[(size_t)col * p.d + row] = x;
-                    store_split(p.s.actP_hi, p.s.actP_lo, (size_t)col * p.dp + row, x * bf16bits_f32(L.g_post[row]));
-                    sqa.a += x * x;
-                });
-                flush_sq(c, sqa, p.s.ssB, nullptr);
-                PROF(c);
-                grid_barrier(c);
-                PROF(c);
-            }
-            // ---- gate / up + SwiGLU
-            {
-                const int st = act_stride(p.d);
-                bf16_t *a_hi = s_hi, *a_lo = s_hi + (size_t)R * st;
-                stage_hilo(c, p.s.actP_hi, p.s.actP_lo, p.dp, p.d, a_hi, a_lo, st, 0);
-                if (c.warp < R) {
-                    float s = rsqrtf(sum_partials(c, p.s.ssB, c.warp) / (float)p.d + p.eps);
-                    if (c.lane == 0) c.misc->scale0[c.warp] = s;
-                }
-                bar_sync(1, kConsumerThreads);
-                ActSrc act{a_hi, a_lo, st, true};
-                PROF(c);
-                consume_phase<GATEUP>(c, act, 0, [&](int row, int col, float gt, float up) {
-                    float s = c.misc->scale0[col];
-                    gt *= s;
-                    up *= s;
-                    float a = gt / (1.f + expf(-gt)) * up;
-                    store_split(p.s.actF_hi, p.s.actF_lo, (size_t)col * p.Fp + row, a);
-                });
-                PROF(c);
-                grid_barrier(c);
-                PROF(c);
-            }
-            // ---- down projection + residual
-            {
-                ActSrc act;
-                if (p.stage_F_in_smem) {
-                    const int st = act_stride(p.F);
-                    bf16_t *a_hi = s_hi, *a_lo = s_hi + (size_t)R * st;
-                    // Fp is a multiple of 32 and the pad beyond F is zero in global scratch
-                    stage_hilo(c, p.s.actF_hi, p.s.actF_lo, p.Fp, p.Fp, a_hi, a_lo, st, 0);
-                    bar_sync(1, kConsumerThreads);
-                    act = ActSrc{a_hi, a_lo, st, true};
-                } else {
-                    act = ActSrc{p.s.actF_hi, p.s.actF_lo, p.Fp, false};
-                }
-                SqAcc sqa;
-                PROF(c);
-                const bf16_t *gnext = (p.mode == 1 && !last_layer) ? p.layers[l + 1].g_in : p.g_final;
-                consume_phase<DOWN>(c, act, 0, [&](int row, int col, float v, float) {
-                    float x = ldcg_f32(p.s.x1 + (size_t)col * p.d + row) + v;
-                    float y = x * bf16bits_f32(gnext[row]);
-                    sqa.a += x * x;
-                    if (p.mode == 1 && !last_layer) {
-                        p.s.x0[(size_t)col * p.d + row] = x;
-                        store_split(p.s.actD_hi, p.s.actD_lo, (size_t)col * p.dp + row, y);
-                    } else {
-                        store_split(p.s.actH_hi, p.s.actH_lo, (size_t)col * p.dp + row, y);
-                        if (p.mode == 0) {
-                            store_split(p.s.actR_hi, p.s.actR_lo, (size_t)col * p.dp + row,
-                                        y * bf16bits_f32(p.g_hnorm[row]));
-                            sqa.b += y * y;
-                        }
-                    }
-                });
-                bool to_head = !(p.mode == 1 && !last_layer);
-                flush_sq(c, sqa, to_head ? p.s.ssC : p.s.ssA, (p.mode == 0) ? p.s.ssD : nullptr);
-                PROF(c);
-                grid_barrier(c);
-                PROF(c);
+            for (int i = c.tid; i < R * (r1 - r0); i += kConsumerThreads) {
+                int r = i / (r1 - r0), k = r0 + (i - r * (r1 - r0));
+                float y = bf16bits_f32(a_hi[(size_t)r * st + k]) + bf16bits_f32(a_lo[(size_t)r * st + k]);
+                size_t o = (p.mode == 0) ? ((size_t)r * p.K + step) * p.d + k : (size_t)r * p.d + k;
+                p.out_h[o] = f32_bf16bits(y * c.misc->scale0[r]);
             }
         }
+        PROF(c);
 
-        // ============ output head
-        {
-            const int st = act_stride(p.d);
-            bf16_t *a_hi = s_hi, *a_lo = s_hi + (size_t)R * st;
-            stage_hilo(c, p.s.actH_hi, p.s.actH_lo, p.dp, p.d, a_hi, a_lo, st, 0);
-            if (c.warp < R) {
-                float s = rsqrtf(sum_partials(c, p.s.ssC, c.warp) / (float)p.d + p.eps);
-                if (c.lane == 0) c.misc->scale0[c.warp] = s;
-            }
-            bar_sync(1, kConsumerThreads);
-            if (p.out_h) {   // every CTA writes its slice of the post-final-norm hidden state
-                int r0 = (int)(((long long)c.cta * p.d) / c.grid), r1 = (int)(((long long)(c.cta + 1) * p.d) / c.grid);
-                for (int i = c.tid; i < R * (r1 - r0); i += kConsumerThreads) {
-                    int r = i / (r1 - r0), k = r0 + (i - r * (r1 - r0));
-                    float y = bf16bits_f32(a_hi[(size_t)r * st + k]) + bf16bits_f32(a_lo[(size_t)r * st + k]);
-                    size_t o = (p.mode == 0) ? ((size_t)r * p.K + step) * p.d + k : (size_t)r * p.d + k;
-                    p.out_h[o] = f32_bf16bits(y * c.misc->scale0[r]);
-                }
-            }
-            ActSrc act{a_hi, a_lo, st, true};
-            unsigned long long best = 0ull;
-            PROF(c);
-            consume_phase<HEAD>(c, act, 0, [&](int row, int col, float v, float) {
-                int id = p.ids ? p.ids[row] : row;
-                if ((unsigned)id >= (unsigned)p.V) id = 0;
-                float lv = v;
-                if (p.mode == 1) {
-                    // target: the decision is taken on the bf16 logits that cross the boundary
-                    uint16_t lb = f32_bf16bits(v * c.misc->scale0[col]);
-                    if (p.out_logits_bf16) p.out_logits_bf16[(size_t)col * p.V + row] = lb;
-                    lv = bf16bits_f32(lb);
-                } else if (p.out_logits_f32) {
-                    p.out_logits_f32[((size_t)col * p.K + step) * p.N + row] = v * c.misc->scale0[col];
-                }
-                unsigned long long key = argmax_key(lv, (uint32_t)id);
-                best = key > best ? key : best;
-            });
+        // ============ ... stream the weights ...
+        if (R > 4) consume_tiles<true>(c, kind, act, seg, ex);
+        else consume_tiles<false>(c, kind, act, seg, ex);
+
+        // ============ ... and publish what the next phase needs besides the vector
+        if (kind == PROJ) flush_sq(c, ex.sq, p.s.ssA, nullptr);
+        else if (kind == OPROJ) flush_sq(c, ex.sq, p.s.ssB, nullptr);
+        else if (kind == DOWN) flush_sq(c, ex.sq, ex.to_next_layer ? p.s.ssA : p.s.ssC, (p.mode == 0) ? p.s.ssD : nullptr);
+        else if (kind == HEAD) {
             // reduce the per-thread maxima (thread = (row slot, col)) over the 32 row slots
-            {
-                unsigned long long k = best;
-                unsigned long long o8 = __shfl_xor_sync(0xffffffffu, k, 8);
-                k = o8 > k ? o8 : k;
-                unsigned long long o16 = __shfl_xor_sync(0xffffffffu, k, 16);
-                k = o16 > k ? o16 : k;
-                if (c.lane < 8) c.misc->keyred[c.warp][c.lane] = k;
-                bar_sync(1, kConsumerThreads);
-                if (c.tid < R) {
-                    unsigned long long m = 0ull;
-                    for (int w = 0; w < kConsumerWarps; ++w) m = c.misc->keyred[w][c.tid] > m ? c.misc->keyred[w][c.tid] : m;
-                    if (m != 0ull) atomicMax(p.s.keys + (size_t)step * kMaxRows + c.tid, m);
-                }
+            unsigned long long k = ex.best;
+            unsigned long long o8 = __shfl_xor_sync(0xffffffffu, k, 8);
+            k = o8 > k ? o8 : k;
+            unsigned long long o16 = __shfl_xor_sync(0xffffffffu, k, 16);
+            k = o16 > k ? o16 : k;
+            if (c.lane < 8) c.misc->keyred[c.warp][c.lane] = k;
+            bar_sync(1, kConsumerThreads);
+            if (c.tid < R) {
+                unsigned long long m = 0ull;
+                for (int w = 0; w < kConsumerWarps; ++w) m = c.misc->keyred[w][c.tid] > m ? c.misc->keyred[w][c.tid] : m;
+                if (m != 0ull) atomicMax(p.s.keys + (size_t)step * kMaxRows + c.tid, m);
             }
-            PROF(c);
-            grid_barrier(c);
-            PROF(c);
+            ex.best = 0ull;
         }
+        PROF(c);
+        grid_barrier(c);
     }
+    PROF(c);
 
     PROF_FLUSH(c, 0, 2, c.tid == 0);
     PROF_FLUSH(c, 4, 5, c.tid == 0);

@@ -96,6 +96,11 @@ __device__ __forceinline__ uint4 lds128(const void *p) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_u32(p)));
     return v;
 }
+__device__ __forceinline__ uint4 lds128_u32(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
 // L2-coherent loads for data other CTAs wrote earlier in the same kernel (bypass L1).
 __device__ __forceinline__ uint4 ldcg128(const void *p) {
     uint4 v;
