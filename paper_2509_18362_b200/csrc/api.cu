@@ -134,6 +134,8 @@ int configure(fmtp_ctx *c, MegaParams &p, int mode, int B, int M) {
     p.mode = mode; p.B = B; p.M = M; p.R = B * M;
     const int R = p.R, Gq = p.Hq / p.Hkv;
     size_t attn = ((size_t)M * Gq * p.dh + (size_t)kConsumerWarps * Gq * (p.dh + 2)) * 4;
+    size_t mrg = ((size_t)2 * c->max_chunks + (size_t)kConsumerThreads + 64) * 4;      // chunk-merge scratch
+    if (mrg > attn) attn = mrg;
     size_t actd = (size_t)2 * R * act_stride(mode == 0 ? 2 * p.d : (p.d > p.qdim ? p.d : p.qdim)) * 2;
     size_t actq = (size_t)2 * R * act_stride(p.qdim) * 2;
     size_t base = attn > actd ? attn : actd;

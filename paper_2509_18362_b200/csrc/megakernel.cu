@@ -40,10 +40,10 @@ constexpr uint32_t kDevBadToken = 0x1u, kDevBadPage = 0x2u, kDevBadPos = 0x4u, k
                    kDevAllNan = 0x10u;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait gives up after 2 s
 
-enum Kind { PROJ = 0, QKV = 1, OPROJ = 2, GATEUP = 3, DOWN = 4, HEAD = 5, ATTN = 6, EMBED = 7, DONE = 8 };
+enum Kind { PROJ = 0, QKV = 1, OPROJ = 2, GATEUP = 3, DOWN = 4, HEAD = 5, ATTN = 6, EMBED = 7, MERGE = 8, DONE = 9 };
 
-// The phase program of a launch. Draft: K x (PROJ, QKV, ATTN, OPROJ, GATEUP, DOWN, HEAD).
-// Target step: EMBED, n_layers x (QKV, ATTN, OPROJ, GATEUP, DOWN), HEAD. Producers and consumers
+// The phase program of a launch. Draft: K x (PROJ, QKV, ATTN, MERGE, OPROJ, GATEUP, DOWN, HEAD).
+// Target step: EMBED, n_layers x (QKV, ATTN, MERGE, OPROJ, GATEUP, DOWN), HEAD. Producers and consumers
 // walk it independently with this iterator, each from a single loop.
 struct Prog { int step, layer, kind; };
 
@@ -158,7 +158,8 @@ __device__ __forceinline__ void prog_next(const MegaParams &p, Prog &g) {
     switch (g.kind) {
         case PROJ: case EMBED: g.kind = QKV; break;
         case QKV: g.kind = ATTN; break;
-        case ATTN: g.kind = OPROJ; break;
+        case ATTN: g.kind = MERGE; break;
+        case MERGE: g.kind = OPROJ; break;
         case OPROJ: g.kind = GATEUP; break;
         case GATEUP: g.kind = DOWN; break;
         case DOWN:
@@ -574,15 +575,29 @@ __device__ __forceinline__ float sum_partials(const Cta &c, const float *tbl, in
 // `len` elements per row (multiple of 8), rows `stride_s` apart in shared memory, starting at
 // element offset `dst_off`.
 __device__ __forceinline__ void stage_hilo(const Cta &c, const bf16_t *ghi, const bf16_t *glo, int gstride, int len, bf16_t *shi,
-                           bf16_t *slo, int sstride, int dst_off) {
-    int per_row = len / 8;
-    int total = c.p->R * per_row;
-    for (int i = c.tid; i < total; i += kConsumerThreads) {
-        int r = i / per_row, k = (i - r * per_row) * 8;
-        uint4 a = ldcg128(ghi + (size_t)r * gstride + k);
-        uint4 b = ldcg128(glo + (size_t)r * gstride + k);
-        *reinterpret_cast<uint4 *>(shi + (size_t)r * sstride + dst_off + k) = a;
-        *reinterpret_cast<uint4 *>(slo + (size_t)r * sstride + dst_off + k) = b;
+                                           bf16_t *slo, int sstride, int dst_off) {
+    const int per_row = len / 8;
+    const int total = c.p->R * per_row;
+    // four units per thread and round: eight loads in flight before the first store waits
+#pragma unroll 1
+    for (int i0 = c.tid; i0 < total; i0 += 4 * kConsumerThreads) {
+        uint4 a[4], b[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            int i = min(i0 + q * kConsumerThreads, total - 1);
+            int r = i / per_row, k = (i - r * per_row) * 8;
+            a[q] = ldcg128(ghi + (size_t)r * gstride + k);
+            b[q] = ldcg128(glo + (size_t)r * gstride + k);
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            int i = i0 + q * kConsumerThreads;
+            if (i < total) {
+                int r = i / per_row, k = (i - r * per_row) * 8;
+                *reinterpret_cast<uint4 *>(shi + (size_t)r * sstride + dst_off + k) = a[q];
+                *reinterpret_cast<uint4 *>(slo + (size_t)r * sstride + dst_off + k) = b[q];
+            }
+        }
     }
 }
 
@@ -796,7 +811,6 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
     const int dh = p.dh, half = dh >> 1, Gq = p.Hq / p.Hkv, M = p.M;
     float *qs = reinterpret_cast<float *>(c.scr);
     float *wp = qs + (size_t)M * Gq * dh;
-    const int wstride = dh + 2;
     const float qscale = rsqrtf((float)dh);
     const int max_tokens = min(kv.max_pages * p.page, p.max_ctx);   // positions beyond are flagged, not touched
     const int upt = dh >> 3;
@@ -804,7 +818,7 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
     const int total = attn_total(p, kv, posoff);
     for (int item = c.cta; item < total; item += c.grid) {
         const AttnItem it = attn_item(p, kv, posoff, item);
-        const int b = it.b, kvh = it.kvh, chunk = it.chunk, Lb = it.Lb, nch = it.nch;
+        const int b = it.b, kvh = it.kvh, chunk = it.chunk, Lb = it.Lb;
         const int base = Lb + posoff;              // position of row m = 0
         const int c0 = chunk * kAttnChunk;
         const int32_t *bt = kv.block_table + (size_t)b * kv.max_pages;
@@ -871,36 +885,56 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
         // the stage is free again (all consumer warps passed the barrier at the end of attn_rows)
         if (c.warp < kConsumerWarps / 2 && c.lane == 0) mbar_arrive(&c.misc->empty[slot]);
         c.stage++;
-        // -- last CTA of this (sequence, KV head) merges the chunks
-        __threadfence();
-        bar_sync(1, kConsumerThreads);
-        if (c.tid == 0) {
-            uint32_t old = atomicAdd(p.s.att_cnt + b * p.Hkv + kvh, 1u);
-            c.misc->flag = (old == (uint32_t)(nch - 1));
+        bar_sync(1, kConsumerThreads);   // the query / partial scratch is reused by the next item
+    }
+}
+
+// ---- merge of the chunk partials ------------------------------------------------------------------
+// After the grid barrier that ends the attention phase every (row, query head) has one partial
+// (o, m, l) per visible chunk. A unit of work is a quarter of one head's output vector; units are
+// dealt round-robin over the CTAs. Thread = (output element, chunk group): it adds its chunks in
+// ascending order, the chunk groups are then added in ascending order, so the summation order
+// depends only on the number of visible chunks, i.e. on the row's position.
+__device__ __forceinline__ void merge_phase(Cta &c, const KvPtrs &kv, int posoff) {
+    const MegaParams &p = *c.p;
+    const int dh = p.dh, M = p.M, wstride = dh + 2;
+    const int qe = dh >> 2;                          // output elements per unit (32 or 16)
+    const int ncg = kConsumerThreads / qe;           // chunk groups (8 or 16)
+    const int max_tokens = min(kv.max_pages * p.page, p.max_ctx);
+    float *ms = reinterpret_cast<float *>(c.scr);    // [max_chunks] chunk maxima
+    float *ls = ms + p.max_chunks;                   // [max_chunks] chunk denominators
+    float *red = ls + p.max_chunks;                  // [ncg][qe + 1] partial sums (+ denominators)
+    const int units = p.R * p.Hq * 4;
+    const int el = c.tid % qe, cg = c.tid / qe;
+    for (int u = c.cta; u < units; u += c.grid) {
+        const int r = u / (p.Hq * 4), rem = u - r * (p.Hq * 4);
+        const int hq = rem >> 2, e = (rem & 3) * qe + el;
+        const int b = r / M, m = r - b * M;
+        const int pos = min(kv.seq_lens[b] + posoff + m, max_tokens - 1);
+        const int ncm = pos / kAttnChunk + 1;        // chunks visible to this row
+        const float *src = p.s.att_part + ((size_t)r * p.Hq + hq) * p.max_chunks * wstride;
+        for (int i = c.tid; i < ncm; i += kConsumerThreads) {
+            ms[i] = ldcg_f32(src + (size_t)i * wstride + dh);
+            ls[i] = ldcg_f32(src + (size_t)i * wstride + dh + 1);
         }
         bar_sync(1, kConsumerThreads);
-        if (c.misc->flag) {
-            __threadfence();
-            for (int i = c.tid; i < M * Gq * dh; i += kConsumerThreads) {
-                int mh = i / dh, e = i - mh * dh;
-                int m = mh / Gq, h = mh - m * Gq;
-                int r = b * M + m, hq = kvh * Gq + h;
-                const float *src = p.s.att_part + ((size_t)r * p.Hq + hq) * p.max_chunks * wstride;
-                int ncm = min(base + m, max_tokens - 1) / kAttnChunk + 1;   // chunks visible to this row
-                float mx = -INFINITY;
-#pragma unroll 8
-                for (int ch = 0; ch < ncm; ++ch) mx = fmaxf(mx, ldcg_f32(src + (size_t)ch * wstride + dh));
-                float ov = 0.f, l = 0.f;
+        float mx = -INFINITY;
+        for (int i = 0; i < ncm; ++i) mx = fmaxf(mx, ms[i]);
+        float ov = 0.f, l = 0.f;
 #pragma unroll 4
-                for (int ch = 0; ch < ncm; ++ch) {
-                    float mc = ldcg_f32(src + (size_t)ch * wstride + dh);
-                    float f = (mc == -INFINITY) ? 0.f : expf(mc - mx);
-                    ov += f * ldcg_f32(src + (size_t)ch * wstride + e);
-                    l += f * ldcg_f32(src + (size_t)ch * wstride + dh + 1);
-                }
-                store_split(p.s.actO_hi, p.s.actO_lo, (size_t)r * p.qp + hq * dh + e, ov / l);
-            }
-            if (c.tid == 0) p.s.att_cnt[b * p.Hkv + kvh] = 0;
+        for (int ch = cg; ch < ncm; ch += ncg) {
+            const float mc = ms[ch];
+            const float f = (mc == -INFINITY) ? 0.f : expf(mc - mx);
+            ov += f * ldcg_f32(src + (size_t)ch * wstride + e);
+            l += f * ls[ch];
+        }
+        red[cg * (qe + 1) + el] = ov;
+        if (el == 0) red[cg * (qe + 1) + qe] = l;
+        bar_sync(1, kConsumerThreads);
+        if (c.tid < qe) {
+            float so = 0.f, sl = 0.f;
+            for (int i = 0; i < ncg; ++i) { so += red[i * (qe + 1) + c.tid]; sl += red[i * (qe + 1) + qe]; }
+            store_split(p.s.actO_hi, p.s.actO_lo, (size_t)r * p.qp + hq * dh + e, so / sl);
         }
         bar_sync(1, kConsumerThreads);
     }
@@ -958,7 +992,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
         Prog g;
         for (prog_begin(p, g); g.kind != DONE; prog_next(p, g)) {
             if (g.kind == ATTN) produce_attention(c, p.kvs[g.layer], (p.mode == 0) ? g.step : 0);
-            else if (g.kind != EMBED) produce_phase(c, g.kind, p.layers[g.layer]);
+            else if (g.kind != EMBED && g.kind != MERGE) produce_phase(c, g.kind, p.layers[g.layer]);
         }
         cp_async_wait_all();   // every copy this thread issued has landed before the CTA may exit
         PROF_FLUSH(c, 2, 4, c.warp == kConsumerWarps && c.lane == 0);
@@ -984,6 +1018,12 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
         PROF(c);
         if (kind == ATTN) {
             attention_phase(c, p.kvs[g.layer], (p.mode == 0) ? step : 0);
+            PROF(c);
+            grid_barrier(c);
+            continue;
+        }
+        if (kind == MERGE) {
+            merge_phase(c, p.kvs[g.layer], (p.mode == 0) ? step : 0);
             PROF(c);
             grid_barrier(c);
             continue;
