@@ -186,7 +186,7 @@ int launch_mega(fmtp_ctx *c, MegaParams &p, cudaStream_t st) {
     if (e != cudaSuccess) return cuda_fail(c, e);
     int err = 0;
     size_t smem = mega_smem_bytes(p);
-    int grid = mega_max_grid(smem, &err);
+    int grid = mega_max_grid(p, smem, &err);
     if (err) return cuda_fail(c, (cudaError_t)err);
     if (grid < 1) return FMTP_ESHAPE;
     if (grid > c->n_sm) grid = c->n_sm;

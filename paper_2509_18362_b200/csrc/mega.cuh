@@ -90,7 +90,7 @@ size_t mega_fixed_smem(int R);
 // Cooperative launch on `stream` with `grid` CTAs (one per SM). Returns the cudaError_t.
 int mega_launch(const MegaParams &p, int grid, cudaStream_t stream);
 // Largest co-resident grid for this shared-memory footprint on the current device.
-int mega_max_grid(size_t smem_bytes, int *err);
+int mega_max_grid(const MegaParams &p, size_t smem_bytes, int *err);
 
 // Verification kernel (verify.cu).
 int verify_launch(const bf16_t *logits, const int32_t *drafts, int B, int K, int V,

@@ -56,6 +56,7 @@ struct Misc {   // small shared-memory block
     float colred[kTileRows][kMaxRows];
     unsigned long long keyred[kConsumerWarps][kMaxRows];
     int tok[kMaxRows];
+    unsigned long long rowptr[kProducerWarps][32];   // tile row pointers, one line per producer warp
     int flag;
     uint32_t aborted;
 };
@@ -92,30 +93,29 @@ struct Cta {
     unsigned char *scr;    // per-phase scratch (activation staging / attention)
     unsigned char *ring;
     int cta, grid, tid, warp, lane;
-    uint32_t stage;        // running stage counter (same sequence in producer and consumers)
+    int slot;              // ring slot of the next stage (same sequence in producer and consumers)
+    uint32_t parity;       // mbarrier phase parity of that slot
     uint32_t bar_target;   // grid barrier generation
     int redbuf;
 };
 
+__device__ __forceinline__ void next_stage(Cta &c) {
+    if (++c.slot == c.p->n_stages) { c.slot = 0; c.parity ^= 1u; }
+}
 __device__ __forceinline__ void raise(const Cta &c, uint32_t bits) { atomicOr(c.p->s.status, bits); }
 
 __device__ __forceinline__ bool aborted(const Cta &c) { return *((volatile uint32_t *)&c.misc->aborted) != 0; }
 
-__device__ __forceinline__ void do_abort(const Cta &c) {
-    c.misc->aborted = 1;
-    atomicOr(c.p->s.status, kDevTimeout);
-    atomicExch(c.p->s.abort_flag, 1u);
-}
-
-// Bounded wait on an mbarrier phase. Returns false (and raises the abort flag) on timeout.
-__device__ __forceinline__ bool wait_bar(const Cta &c, uint64_t *bar, uint32_t parity) {
-    if (aborted(c)) return false;
+// Bounded wait on an mbarrier phase (kept inline: a real call makes ptxas ignore setmaxnreg), called
+// from every ring wait. Returns false on timeout or abort, after setting the status bits.
+__device__ __forceinline__ bool wait_bar_impl(Misc *misc, uint64_t *bar, uint32_t parity, uint32_t *abort_flag, uint32_t *status) {
+    if (*((volatile uint32_t *)&misc->aborted) != 0) return false;
     unsigned long long t0 = 0;
     for (uint32_t n = 0;; ++n) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((n & 255u) == 255u) {
-            if (ldcg_u32(c.p->s.abort_flag) != 0) {
-                c.misc->aborted = 1;
+            if (ldcg_u32(abort_flag) != 0) {
+                misc->aborted = 1;
                 return false;
             }
             unsigned long long now = global_timer_ns();
@@ -123,8 +123,19 @@ __device__ __forceinline__ bool wait_bar(const Cta &c, uint64_t *bar, uint32_t p
             else if (now - t0 > kWaitLimitNs) break;
         }
     }
-    do_abort(c);
+    misc->aborted = 1;
+    atomicOr(status, kDevTimeout);
+    atomicExch(abort_flag, 1u);
     return false;
+}
+__device__ __forceinline__ bool wait_bar(const Cta &c, uint64_t *bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;          // fast path: already complete
+    return wait_bar_impl(c.misc, bar, parity, c.p->s.abort_flag, c.p->s.status);
+}
+__device__ __forceinline__ void do_abort(const Cta &c) {
+    c.misc->aborted = 1;
+    atomicOr(c.p->s.status, kDevTimeout);
+    atomicExch(c.p->s.abort_flag, 1u);
 }
 
 // Grid-wide barrier among the consumer threads of all CTAs (the producer warp never joins).
@@ -233,31 +244,42 @@ __device__ __forceinline__ const bf16_t *tile_row_ptr(const Cta &c, int kind, co
 // stall the warp on every instruction (measured: 4.2 instead of 7.0 TB/s). Row pointers of the
 // next tile are computed one tile ahead so the subset-id lookup of the output head is off the
 // issue path.
-constexpr int kRowsPerProducer = kTileRows / kProducerWarps;   // 4
+constexpr int kRowsPerProducer = kTileRows / kProducerWarps;   // 8
 
-__device__ __forceinline__ void tile_ptrs(const Cta &c, int kind, const LayerPtrs &L, int vr0, int nv, int pw,
+// Row pointers of a tile for one producer warp: lane j computes the pointer of tile row j (one
+// subset-id lookup per lane, all in parallel), the warp exchanges them through its own line of a
+// small shared-memory table and every lane keeps the eight rows its warp copies in registers.
+// (No shuffles here or in the issue path: they would queue behind the cp.async traffic.)
+__device__ __forceinline__ void tile_ptrs(Cta &c, int kind, const LayerPtrs &L, int vr0, int nv, int pw,
                                           const unsigned char *(&out)[kRowsPerProducer]) {
+    unsigned long long *tbl = c.misc->rowptr[pw];
+    __syncwarp();
+    tbl[c.lane] = reinterpret_cast<unsigned long long>(tile_row_ptr(c, kind, L, vr0, nv, c.lane));
+    __syncwarp();
 #pragma unroll
-    for (int i = 0; i < kRowsPerProducer; ++i)
-        out[i] = reinterpret_cast<const unsigned char *>(tile_row_ptr(c, kind, L, vr0, nv, pw + i * kProducerWarps));
+    for (int i = 0; i < kRowsPerProducer; ++i) out[i] = reinterpret_cast<const unsigned char *>(tbl[pw + i * kProducerWarps]);
 }
 
 __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs &L) {
     const MegaParams &p = *c.p;
-    Geom g = geom(c, kind);
+    const Geom g = geom(c, kind);
     const int pw = c.warp - kConsumerWarps;
     const unsigned char *cur[kRowsPerProducer], *nxt[kRowsPerProducer];
 #pragma unroll
     for (int i = 0; i < kRowsPerProducer; ++i) nxt[i] = nullptr;
-    if (g.v0 < g.v1) tile_ptrs(c, kind, L, g.v0, min(g.cap, g.v1 - g.v0), pw, nxt);
     const uint32_t lane16 = (uint32_t)c.lane * 16u;
-    for (int vr0 = g.v0; vr0 < g.v1; vr0 += g.cap) {
+    const uint32_t rs = (uint32_t)p.row_stride;
+    // the loop starts one tile early: iteration t fetches the pointers of tile t + 1
+#pragma unroll 1
+    for (int vr0 = g.v0 - g.cap; vr0 < g.v1; vr0 += g.cap) {
 #pragma unroll
         for (int i = 0; i < kRowsPerProducer; ++i) cur[i] = nxt[i];
         if (vr0 + g.cap < g.v1) tile_ptrs(c, kind, L, vr0 + g.cap, min(g.cap, g.v1 - vr0 - g.cap), pw, nxt);
+        if (vr0 < g.v0) continue;
+#pragma unroll 1
         for (int ks = 0; ks < g.nks; ++ks) {
-            int slot = c.stage % p.n_stages;
-            uint32_t parity = (c.stage / p.n_stages) & 1u;
+            const int slot = c.slot;
+            const uint32_t parity = c.parity;
             bool ok = true;
             PROF_T0();
             if (c.lane == 0) ok = wait_bar(c, &c.misc->empty[slot], parity ^ 1u);
@@ -265,24 +287,23 @@ __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs 
             PROF_ACC(c, 2, pw == 0 && c.lane == 0);
             if (!ok) return;   // abort: stop issuing copies
             const int klen = min(p.KC, g.K - ks * p.KC);
-            const uint32_t dst0 = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + (uint32_t)pw * (uint32_t)p.row_stride + lane16;
+            const uint32_t dst0 = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + (uint32_t)pw * rs + lane16;
             const size_t koff = (size_t)ks * p.KC * 2 + lane16;
             if (klen == 512) {
-                // 1024 bytes per row: two instructions per row, eight per thread, all independent
-                uint32_t d[2 * kRowsPerProducer];
-                const unsigned char *q[2 * kRowsPerProducer];
+                // 1024 bytes per row: two instructions per row, sixteen per thread, all with their own
+                // address registers
+                uint32_t d[kRowsPerProducer];
+                const unsigned char *q[kRowsPerProducer];
 #pragma unroll
                 for (int i = 0; i < kRowsPerProducer; ++i) {
-                    d[2 * i] = dst0 + (uint32_t)(i * kProducerWarps) * (uint32_t)p.row_stride;
-                    d[2 * i + 1] = d[2 * i] + 512u;
-                    q[2 * i] = cur[i] + koff;
-                    q[2 * i + 1] = q[2 * i] + 512;
+                    q[i] = cur[i] + koff;
+                    d[i] = dst0 + (uint32_t)(i * kProducerWarps) * rs;
                 }
 #pragma unroll
                 for (int i = 0; i < kRowsPerProducer; ++i) {
                     if (cur[i] != nullptr) {
-                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d[2 * i]), "l"(q[2 * i]) : "memory");
-                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d[2 * i + 1]), "l"(q[2 * i + 1]) : "memory");
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d[i]), "l"(q[i]) : "memory");
+                        asm volatile("cp.async.cg.shared.global [%0+512], [%1+512], 16;" ::"r"(d[i]), "l"(q[i]) : "memory");
                     }
                 }
             } else {
@@ -290,17 +311,18 @@ __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs 
                 const int n16 = klen >> 3;
 #pragma unroll
                 for (int i = 0; i < kRowsPerProducer; ++i) {
-                    if (cur[i] != nullptr) {
+                    const unsigned char *rp = cur[i];
+                    if (rp != nullptr) {
                         for (int u = c.lane; u < n16; u += 32) {
-                            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst0 + (uint32_t)(i * kProducerWarps) * (uint32_t)p.row_stride + (uint32_t)(u - c.lane) * 16u),
-                                         "l"(cur[i] + koff + (size_t)(u - c.lane) * 16) : "memory");
+                            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst0 + (uint32_t)(i * kProducerWarps) * rs + (uint32_t)(u - c.lane) * 16u),
+                                         "l"(rp + koff + (size_t)(u - c.lane) * 16) : "memory");
                         }
                     }
                 }
             }
             cp_async_arrive(&c.misc->full[slot]);
             PROF_ACC(c, 3, pw == 0 && c.lane == 0);
-            c.stage++;
+            next_stage(c);
         }
     }
 }
@@ -472,8 +494,8 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
 #pragma unroll 1
         for (int ks = 0; ks < geo.nks; ++ks) {
             if (((stage0 + ks) & 1) == grp) {
-                const int slot = c.stage % p.n_stages;
-                const uint32_t parity = (c.stage / p.n_stages) & 1u;
+                const int slot = c.slot;
+                const uint32_t parity = c.parity;
                 PROF_T0();
                 wait_bar(c, &c.misc->full[slot], parity);
                 PROF_ACC(c, 0, c.tid == 0);
@@ -515,7 +537,7 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
                 if (c.lane == 0) mbar_arrive(&c.misc->empty[slot]);
                 PROF_ACC(c, 1, c.tid == 0);
             }
-            c.stage++;
+            next_stage(c);
         }
         // a warp whose stages all lay in the first segment parks them now
         if (kind == PROJ && !moved) park<two_sets>(acc, acd, acc0, acd0);
@@ -769,8 +791,8 @@ __device__ __forceinline__ void produce_attention(Cta &c, const KvPtrs &kv, int 
         const int c0 = it.chunk * kAttnChunk;
         const int n_old = max(0, min(kAttnChunk, it.Lb - c0));   // committed tokens of this chunk
         const int32_t *bt = kv.block_table + (size_t)it.b * kv.max_pages;
-        int slot = c.stage % p.n_stages;
-        uint32_t parity = (c.stage / p.n_stages) & 1u;
+        const int slot = c.slot;
+        const uint32_t parity = c.parity;
         bool ok = true;
         if (c.lane == 0) ok = wait_bar(c, &c.misc->empty[slot], parity ^ 1u);
         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -802,13 +824,15 @@ __device__ __forceinline__ void produce_attention(Cta &c, const KvPtrs &kv, int 
             }
         }
         cp_async_arrive(&c.misc->full[slot]);
-        c.stage++;
+        next_stage(c);
     }
 }
 
+template <int DH>
 __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int posoff) {
     const MegaParams &p = *c.p;
-    const int dh = p.dh, half = dh >> 1, Gq = p.Hq / p.Hkv, M = p.M;
+    constexpr int dh = DH, half = DH >> 1;
+    const int Gq = p.Hq / p.Hkv, M = p.M;
     float *qs = reinterpret_cast<float *>(c.scr);
     float *wp = qs + (size_t)M * Gq * dh;
     const float qscale = rsqrtf((float)dh);
@@ -822,8 +846,8 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
         const int base = Lb + posoff;              // position of row m = 0
         const int c0 = chunk * kAttnChunk;
         const int32_t *bt = kv.block_table + (size_t)b * kv.max_pages;
-        const int slot = c.stage % p.n_stages;
-        const uint32_t parity = (c.stage / p.n_stages) & 1u;
+        const int slot = c.slot;
+        const uint32_t parity = c.parity;
         bf16_t *sk = reinterpret_cast<bf16_t *>(c.ring + (size_t)slot * p.stage_bytes);
         bf16_t *sv = sk + (size_t)kAttnChunk * dh;
 
@@ -879,12 +903,11 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
         bar_sync(1, kConsumerThreads);
         PROF(c);
 
-        if (dh == 128) attn_rows<128>(c, sk, sv, qs, wp, b, kvh, chunk, base, max_tokens);
-        else attn_rows<64>(c, sk, sv, qs, wp, b, kvh, chunk, base, max_tokens);
+        attn_rows<DH>(c, sk, sv, qs, wp, b, kvh, chunk, base, max_tokens);
         PROF(c);
         // the stage is free again (all consumer warps passed the barrier at the end of attn_rows)
         if (c.warp < kConsumerWarps / 2 && c.lane == 0) mbar_arrive(&c.misc->empty[slot]);
-        c.stage++;
+        next_stage(c);
         bar_sync(1, kConsumerThreads);   // the query / partial scratch is reused by the next item
     }
 }
@@ -941,6 +964,9 @@ __device__ __forceinline__ void merge_phase(Cta &c, const KvPtrs &kv, int posoff
 }
 
 // ---- the kernel --------------------------------------------------------------------------------
+// One instantiation per (more than four activation rows?, head dimension): each contains only the
+// code it runs, which keeps it near the size of the instruction cache.
+template <bool TWO, int DH>
 __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant__ MegaParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     Cta c;
@@ -957,7 +983,8 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
     c.tid = threadIdx.x;
     c.warp = threadIdx.x >> 5;
     c.lane = threadIdx.x & 31;
-    c.stage = 0;
+    c.slot = 0;
+    c.parity = 0;
     c.bar_target = 0;
     c.redbuf = 0;
 #ifdef FMTP_PROF
@@ -1017,7 +1044,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
         ex.gnext = ex.to_next_layer ? p.layers[g.layer + 1].g_in : p.g_final;
         PROF(c);
         if (kind == ATTN) {
-            attention_phase(c, p.kvs[g.layer], (p.mode == 0) ? step : 0);
+            attention_phase<DH>(c, p.kvs[g.layer], (p.mode == 0) ? step : 0);
             PROF(c);
             grid_barrier(c);
             continue;
@@ -1152,8 +1179,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
         PROF(c);
 
         // ============ ... stream the weights ...
-        if (R > 4) consume_tiles<true>(c, kind, act, seg, ex);
-        else consume_tiles<false>(c, kind, act, seg, ex);
+        consume_tiles<TWO>(c, kind, act, seg, ex);
 
         // ============ ... and publish what the next phase needs besides the vector
         if (kind == PROJ) flush_sq(c, ex.sq, p.s.ssA, nullptr);
@@ -1233,12 +1259,20 @@ size_t mega_fixed_smem(int R) {
     return off;
 }
 
-int mega_max_grid(size_t smem_bytes, int *err) {
+namespace {
+const void *kernel_for(int R, int dh) {
+    if (dh == 128) return R > 4 ? (const void *)mega_kernel<true, 128> : (const void *)mega_kernel<false, 128>;
+    return R > 4 ? (const void *)mega_kernel<true, 64> : (const void *)mega_kernel<false, 64>;
+}
+}  // namespace
+
+int mega_max_grid(const MegaParams &p, size_t smem_bytes, int *err) {
     int dev = 0, sms = 0, per_sm = 0;
+    const void *fn = kernel_for(p.R, p.dh);
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(mega_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mega_kernel, kThreads, smem_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, smem_bytes);
     if (err) *err = (int)e;
     if (e != cudaSuccess) return 0;
     return sms * (per_sm > 0 ? 1 : 0);
@@ -1246,10 +1280,11 @@ int mega_max_grid(size_t smem_bytes, int *err) {
 
 int mega_launch(const MegaParams &p, int grid, cudaStream_t stream) {
     size_t smem = mega_smem_bytes(p);
-    cudaError_t e = cudaFuncSetAttribute(mega_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const void *fn = kernel_for(p.R, p.dh);
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
     void *args[] = {const_cast<MegaParams *>(&p)};
-    e = cudaLaunchCooperativeKernel((const void *)mega_kernel, dim3(grid), dim3(kThreads), args, smem, stream);
+    e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kThreads), args, smem, stream);
     return (int)e;
 }
 
