@@ -133,7 +133,7 @@ int configure(fmtp_ctx *c, MegaParams &p, int mode, int B, int M) {
     p.max_ctx = sh.max_ctx;
     p.mode = mode; p.B = B; p.M = M; p.R = B * M;
     const int R = p.R, Gq = p.Hq / p.Hkv;
-    size_t attn = ((size_t)M * Gq * p.dh + (size_t)kConsumerWarps * Gq * (p.dh + 2)) * 4;
+    size_t attn = ((size_t)M * Gq * p.dh + (size_t)kConsumerWarps * Gq * (p.dh + 2) + (size_t)Gq * (kConsumerWarps + 2)) * 4;
     size_t mrg = ((size_t)2 * c->max_chunks + (size_t)kConsumerThreads + 64) * 4;      // chunk-merge scratch
     if (mrg > attn) attn = mrg;
     size_t actd = (size_t)2 * R * act_stride(mode == 0 ? 2 * p.d : (p.d > p.qdim ? p.d : p.qdim)) * 2;

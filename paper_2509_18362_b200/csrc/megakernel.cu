@@ -583,11 +583,21 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
     }
 }
 
-// Sum over CTAs of a per-CTA partial-sums-of-squares table [grid][8], for activation row `col`.
-// Called by one full warp; fixed reduction tree => reproducible.
-__device__ __forceinline__ float sum_partials(const Cta &c, const float *tbl, int col) {
+// Sum over CTAs of a per-CTA partial-sums-of-squares table [grid][8], for activation row `col`,
+// by one full warp in a fixed reduction tree (reproducible). Split in two so that the loads can be
+// issued before other work and consumed after it (grid <= 32 * kPartialRegs).
+constexpr int kPartialRegs = 5;
+__device__ __forceinline__ void load_partials(const Cta &c, const float *tbl, int col, float (&v)[kPartialRegs]) {
+#pragma unroll
+    for (int q = 0; q < kPartialRegs; ++q) {
+        int i = c.lane + 32 * q;
+        v[q] = (i < c.grid) ? ldcg_f32(tbl + (size_t)i * kMaxRows + col) : 0.f;
+    }
+}
+__device__ __forceinline__ float reduce_partials(const float (&v)[kPartialRegs]) {
     float s = 0.f;
-    for (int i = c.lane; i < c.grid; i += 32) s += ldcg_f32(tbl + (size_t)i * kMaxRows + col);
+#pragma unroll
+    for (int q = 0; q < kPartialRegs; ++q) s += v[q];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     return s;
@@ -736,24 +746,33 @@ __device__ __forceinline__ void attn_rows(Cta &c, const bf16_t *sk, const bf16_t
             if (c.lane == 0) { w[DH] = mx; w[DH + 1] = sm; }
         }
         bar_sync(1, kConsumerThreads);
-        // ---- merge the 8 warps (fixed order) -> chunk partial in global memory
-        for (int i = c.tid; i < Gq * DH; i += kConsumerThreads) {
-            int h = i / DH, e = i - h * DH;
+        // ---- merge the 8 warps (fixed order) -> chunk partial in global memory.
+        // weight of warp w for head h: thread (h, w) computes it once
+        float *fw = wp + (size_t)kConsumerWarps * Gq * wstride;      // [Gq][8] weights, then [Gq][2] (m, l)
+        if (c.tid < Gq * kConsumerWarps) {
+            const int h = c.tid >> 3, w = c.tid & 7;
             float mx = -INFINITY;
 #pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) mx = fmaxf(mx, wp[((size_t)w * Gq + h) * wstride + DH]);
+            for (int q = 0; q < kConsumerWarps; ++q) mx = fmaxf(mx, wp[((size_t)q * Gq + h) * wstride + DH]);
+            const float mw = wp[((size_t)w * Gq + h) * wstride + DH];
+            fw[h * kConsumerWarps + w] = (mw == -INFINITY) ? 0.f : expf(mw - mx);
+            if (w == 0) fw[Gq * kConsumerWarps + 2 * h] = mx;
+        }
+        bar_sync(1, kConsumerThreads);
+        for (int i = c.tid; i < Gq * DH; i += kConsumerThreads) {
+            const int h = i / DH, e = i - h * DH;
             float ov = 0.f, l = 0.f;
 #pragma unroll
             for (int w = 0; w < kConsumerWarps; ++w) {
                 const float *pw = wp + ((size_t)w * Gq + h) * wstride;
-                float f = (pw[DH] == -INFINITY) ? 0.f : expf(pw[DH] - mx);
+                const float f = fw[h * kConsumerWarps + w];
                 ov += f * pw[e];
                 l += f * pw[DH + 1];
             }
-            int r = b * M + m, hq = kvh * Gq + h;
+            const int r = b * M + m, hq = kvh * Gq + h;
             float *dst = p.s.att_part + (((size_t)r * p.Hq + hq) * p.max_chunks + chunk) * wstride;
             dst[e] = ov;
-            if (e == 0) { dst[DH] = mx; dst[DH + 1] = l; }
+            if (e == 0) { dst[DH] = fw[Gq * kConsumerWarps + 2 * h]; dst[DH + 1] = l; }
         }
         bar_sync(1, kConsumerThreads);
     }
@@ -1084,11 +1103,24 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
         if (kind == PROJ) {
             // ---- x0 = W_p [ rms(h) ; rms(Emb(tok)) ]
             seg = p.d / p.KC;
+            // loads that do not depend on each other are issued first: the previous step's argmax key,
+            // the partial sums that normalise the recursed state, and that state itself
+            unsigned long long key = 0ull;
+            if (step > 0 && c.tid < R) key = ldcg_u64(p.s.keys + (size_t)(step - 1) * kMaxRows + c.tid);
+            float pvc[kPartialRegs], pvd[kPartialRegs];
+            const bool renorm = step > 0 && c.warp < R;
+            if (renorm) { load_partials(c, p.s.ssC, c.warp, pvc); load_partials(c, p.s.ssD, c.warp, pvd); }
+            if (step > 0) stage_hilo(c, p.s.actR_hi, p.s.actR_lo, p.dp, p.d, a_hi, a_lo, st, 0);
+            if (renorm) {
+                // recursed state: h = (x2*g_final) * s_x; rms(h) adds s_h = rsqrt(s_x^2 * mean((x2 g)^2) + eps)
+                float sx = rsqrtf(reduce_partials(pvc) / (float)p.d + p.eps);
+                float sy = reduce_partials(pvd) / (float)p.d;
+                if (c.lane == 0) c.misc->scale0[c.warp] = sx * rsqrtf(sx * sx * sy + p.eps);
+            }
             if (c.tid < R) {
                 int tok;
                 if (step == 0) tok = p.tokens[c.tid];
                 else {
-                    unsigned long long key = ldcg_u64(p.s.keys + (size_t)(step - 1) * kMaxRows + c.tid);
                     if ((key >> 32) == 0ull) raise(c, kDevAllNan);
                     tok = (int)argmax_key_id(key);
                     if (c.cta == 0) p.out_tokens[(size_t)c.tid * p.K + (step - 1)] = tok;
@@ -1097,7 +1129,6 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                 c.misc->tok[c.tid] = tok;
             }
             bar_sync(1, kConsumerThreads);
-            if (step > 0) stage_hilo(c, p.s.actR_hi, p.s.actR_lo, p.dp, p.d, a_hi, a_lo, st, 0);
 #pragma unroll 1
             for (int r = 0; r < R; ++r) {
                 float sqh = 0.f, sqe = 0.f;
@@ -1135,12 +1166,6 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                 if (c.lane == 0) { c.misc->ssred[c.warp][r][0] = sqh; c.misc->ssred[c.warp][r][1] = sqe; }
             }
             bar_sync(1, kConsumerThreads);
-            if (step > 0 && c.warp < R) {
-                // recursed state: h = (x2*g_final) * s_x; rms(h) adds s_h = rsqrt(s_x^2 * mean((x2 g)^2) + eps)
-                float sx = rsqrtf(sum_partials(c, p.s.ssC, c.warp) / (float)p.d + p.eps);
-                float sy = sum_partials(c, p.s.ssD, c.warp) / (float)p.d;
-                if (c.lane == 0) c.misc->scale0[c.warp] = sx * rsqrtf(sx * sx * sy + p.eps);
-            }
             if (c.tid < R) {
                 float sh = 0.f, se = 0.f;
                 for (int i = 0; i < kConsumerWarps; ++i) { sh += c.misc->ssred[i][c.tid][0]; se += c.misc->ssred[i][c.tid][1]; }
@@ -1159,10 +1184,13 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                 case DOWN:   ghi = p.s.actF_hi; glo = p.s.actF_lo; gstride = p.Fp; glen = p.Fp; break;   // pad beyond F is zero
                 default:     ghi = p.s.actH_hi; glo = p.s.actH_lo; sstab = p.s.ssC; break;               // HEAD
             }
+            float pv[kPartialRegs];
+            const bool norm = sstab != nullptr && c.warp < R;
+            if (norm) load_partials(c, sstab, c.warp, pv);       // in flight while the vector is staged
             if (kind == DOWN && !p.stage_F_in_smem) act = ActSrc{ghi, glo, gstride, false};
             else stage_hilo(c, ghi, glo, gstride, glen, a_hi, a_lo, st, 0);
-            if (sstab && c.warp < R) {
-                float sc = rsqrtf(sum_partials(c, sstab, c.warp) / (float)p.d + p.eps);
+            if (norm) {
+                float sc = rsqrtf(reduce_partials(pv) / (float)p.d + p.eps);
                 if (c.lane == 0) c.misc->scale0[c.warp] = sc;
             }
         }
