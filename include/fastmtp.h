@@ -190,6 +190,28 @@ int fastmtp_verify_accept_host(fmtp_ctx *ctx, const fmtp_bf16 *target_logits_hos
                                const int32_t *drafts_host, int B, int K, int V,
                                int32_t *out_accept_len_host, int32_t *out_bonus_host, void *stream);
 
+/* ---- verification without a context or any allocation ------------------------------------ */
+
+/* The paper has no counterpart for this call; it exists for hosts that cannot allocate. Same
+ * operation and same results as fastmtp_verify_accept, but it takes no context and no workspace:
+ * the per-row scratch lives in a fixed array inside the library (8.3 KB of device memory on every
+ * GPU that loads the library, held until the process exits). Meant for callers that only hold raw
+ * device pointers, or that run where creating device memory is impossible or would stall the GPU
+ * (an allocator that already owns all of it, a latency-critical decode loop). The call itself
+ * performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ *   Limit: B * (K + 1) <= FMTP_STATIC_VERIFY_MAX_ROWS, otherwise FMTP_ESHAPE and nothing is enqueued.
+ *   The first call on a device looks up the array's device address (once per device, with that
+ *   device current); make that first call outside any stream capture.
+ *   All calls share the one array: it is cleared on `stream` at the start of every call, and two
+ *   calls whose work overlaps on the GPU (different streams, no ordering) race on it.
+ * Arguments, layouts and the meaning of dev_status are those of fastmtp_verify_accept. */
+#define FMTP_STATIC_VERIFY_MAX_ROWS 1024
+int fastmtp_verify_accept_static(const fmtp_bf16 *target_logits, const int32_t *drafts,
+                                 int B, int K, int V,
+                                 int32_t *out_accept_len, int32_t *out_bonus, int32_t *out_argmax,
+                                 uint32_t *dev_status, void *stream);
+
 /* ---- target decoder step (Sec. 2.1: embedding, transformer layers F, output head W) ----- */
 
 /* Runs M new tokens per sequence through the n_layers-deep target stack with the same

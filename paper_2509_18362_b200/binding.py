@@ -25,7 +25,8 @@ DEV_BAD_TOKEN, DEV_BAD_PAGE, DEV_BAD_POS, DEV_TIMEOUT, DEV_ALL_NAN = 1, 2, 4, 8,
 
 EXPORTS = ["fmtp_create", "fmtp_destroy", "fmtp_workspace_bytes", "fmtp_set_workspace", "fmtp_strerror",
            "fmtp_last_cuda_error", "fmtp_launch_count", "fastmtp_draft", "fastmtp_draft_host",
-           "fastmtp_verify_accept", "fastmtp_verify_accept_host", "fastmtp_target_step"]
+           "fastmtp_verify_accept", "fastmtp_verify_accept_host", "fastmtp_verify_accept_static",
+           "fastmtp_target_step"]
 
 _p = C.c_void_p
 
@@ -79,6 +80,8 @@ lib.fastmtp_verify_accept.argtypes = [_p, _p, _p, C.c_int, C.c_int, C.c_int, _p,
 lib.fastmtp_verify_accept.restype = C.c_int
 lib.fastmtp_verify_accept_host.argtypes = [_p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p]
 lib.fastmtp_verify_accept_host.restype = C.c_int
+lib.fastmtp_verify_accept_static.argtypes = [_p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p, _p]
+lib.fastmtp_verify_accept_static.restype = C.c_int
 lib.fastmtp_target_step.argtypes = [_p, C.POINTER(fmtp_target_w), _p, C.POINTER(fmtp_kv), C.c_int, C.c_int,
                                     _p, _p, _p, _p, _p]
 lib.fastmtp_target_step.restype = C.c_int
@@ -124,6 +127,19 @@ def target_w(t: dict):
 def kv(t: dict) -> fmtp_kv:
     return fmtp_kv(t["k_pages"].data_ptr(), t["v_pages"].data_ptr(), t["block_table"].data_ptr(),
                    t["seq_lens"].data_ptr(), int(t["k_pages"].shape[0]), int(t["block_table"].shape[1]))
+
+
+STATIC_VERIFY_MAX_ROWS = 1024
+
+
+def fastmtp_verify_accept_static(target_logits, drafts, B, K, V, out_accept_len, out_bonus, out_argmax=None,
+                                 dev_status=None, stream=None):
+    """Verification through the entry point that needs no context and allocates nothing (its scratch
+    is a fixed array inside the library). Same arguments as Context.fastmtp_verify_accept."""
+    rc = lib.fastmtp_verify_accept_static(_ptr(target_logits), _ptr(drafts), B, K, V, _ptr(out_accept_len),
+                                          _ptr(out_bonus), _ptr(out_argmax), _ptr(dev_status), _stream(stream))
+    if rc != FMTP_OK:
+        raise FastMTPError(rc, "fastmtp_verify_accept_static")
 
 
 class Context:
