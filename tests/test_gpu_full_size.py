@@ -1,0 +1,88 @@
+"""Parity at the benchmark's full size: the 7B-class MTP head (d=3584, 28/4 heads of 128, ffn 18944,
+V=152064, subset 32768, 2048 cached tokens, K=3) in the launch configuration bench.py times, checked
+against the oracle on every draft, every hidden state and sampled subset logits."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fastmtp_oracle as O
+from paper_2509_18362_b200 import inputs as I
+from tests.gpu_util import close, copy_kv, ids_match
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def seven_b():
+    shape = I.QWEN7B
+    W = I.mtp_weights(shape, 1234)
+    from paper_2509_18362_b200 import binding as Bd
+    return shape, W, Bd.to_device(W)
+
+
+@pytest.mark.parametrize("B,ctx_lens,subset_kind", [(1, [2048], "uniform"), (3, [2048, 777, 1], "zipf")])
+def test_7b_draft_matches_oracle(seven_b, B, ctx_lens, subset_kind):
+    from paper_2509_18362_b200 import binding as Bd
+    shape, W, dW = seven_b
+    K, N, seed = 3, 32768, 1234
+    kv = I.paged_kv(shape, ctx_lens, K + 1, seed + 1)
+    h = I.hidden_bf16(seed + 2, (B, shape.d))
+    tok = I.token_ids(seed + 3, (B,), shape.vocab)
+    ids = I.subset_uniform(shape.vocab, N, seed + 4) if subset_kind == "uniform" else I.subset_zipf(shape.vocab, N, seed + 4)
+    ctx = Bd.Context(shape, max_rows=8, max_K=8, max_ctx=max(ctx_lens) + K + 1)
+    dkv = Bd.to_device(copy_kv(kv))
+    out_d = torch.full((B, K), -1, dtype=torch.int32, device="cuda")
+    out_h = torch.zeros((B, K, shape.d), dtype=torch.bfloat16, device="cuda")
+    out_l = torch.zeros((B, K, N), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx.fastmtp_draft(Bd.mtp_w(dW), Bd.bf16_tensor(h), torch.from_numpy(tok).cuda(), Bd.kv(dkv), B, K,
+                      torch.from_numpy(ids).cuda(), out_d, out_h, out_l, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    drafts = out_d.cpu().numpy()
+    # the production call (no debug logits) gives the same drafts
+    out_d2 = torch.full((B, K), -1, dtype=torch.int32, device="cuda")
+    dkv2 = Bd.to_device(copy_kv(kv))
+    ctx.fastmtp_draft(Bd.mtp_w(dW), Bd.bf16_tensor(h), torch.from_numpy(tok).cuda(), Bd.kv(dkv2), B, K,
+                      torch.from_numpy(ids).cuda(), out_d2)
+    torch.cuda.synchronize()
+    assert np.array_equal(out_d2.cpu().numpy(), drafts)
+
+    okv = copy_kv(kv)
+    ref = O.draft(shape, W, h, tok, okv, K, ids, forced=drafts)
+    exempt = ids_match(drafts, ref["drafts"], ref["gap"], "7B drafts")
+    close(out_h.float().cpu().numpy(), ref["h_out"], "7B h_out")
+    # sampled logits: 512 subset rows per (sequence, step), computed one by one by the oracle
+    g = I.rng(7, "logit-sample")
+    lg = out_l.cpu().numpy()
+    for b in range(B):
+        for k in range(K):
+            rows = g.choice(N, size=512, replace=False)
+            want = O.head_logits(ref["h_out"][b, k], W["lm_head"], ids[rows])
+            close(lg[b, k, rows], want, f"7B logits b={b} k={k}")
+    # K/V appended for the K new positions of every sequence
+    gk, gv = Bd.bf16_bits(dkv["k_pages"]), Bd.bf16_bits(dkv["v_pages"])
+    for b in range(B):
+        for k in range(K):
+            pos = ctx_lens[b] + k
+            page = int(kv["block_table"][b, pos // shape.page_size])
+            close(O.bf16_to_f64(gk[page, :, pos % shape.page_size]), O.bf16_to_f64(okv["k_pages"][page, :, pos % shape.page_size]), "7B K append")
+            close(O.bf16_to_f64(gv[page, :, pos % shape.page_size]), O.bf16_to_f64(okv["v_pages"][page, :, pos % shape.page_size]), "7B V append")
+    ctx.close()
+    O.clear_weight_memo()
+    print(f"7B B={B}: drafts {drafts.tolist()} near-tie exemptions {exempt}")
+
+
+def test_verify_accept_full_size():
+    """[64, 4, 152064] bf16 logits with planted prefix lengths: exact recovery, equal to the oracle."""
+    from paper_2509_18362_b200 import binding as Bd
+    ctx = Bd.Context(I.TINY, max_rows=8, max_K=8, max_ctx=64)
+    case = I.verify_case(64, 3, 152064, 4321)
+    acc = torch.zeros(64, dtype=torch.int32, device="cuda")
+    bon = torch.zeros(64, dtype=torch.int32, device="cuda")
+    ctx.fastmtp_verify_accept(Bd.bf16_tensor(case["logits"]), torch.from_numpy(case["drafts"]).cuda(), 64, 3, 152064, acc, bon)
+    torch.cuda.synchronize()
+    assert np.array_equal(acc.cpu().numpy(), case["length"])
+    ra, rb, _ = O.verify_accept(case["logits"][:8], case["drafts"][:8])        # oracle on a sample of the batch
+    assert np.array_equal(acc.cpu().numpy()[:8], ra) and np.array_equal(bon.cpu().numpy()[:8], rb)
+    ctx.close()
