@@ -664,7 +664,7 @@ __device__ __forceinline__ void flush_sq(const Cta &c, const SqAcc &q, float *tb
 // wp[8 warps][Gq][dh + 2] per-warp partial (o, m, l) of the row being processed.
 
 // One chunk of one KV head from shared memory, for every row of the call: each warp takes 8 tokens.
-// Scores: lane = (token, quarter of the head dimension); the four quarters are added with two
+// Scores: lane = (quarter of the head dimension, token); the four quarters are added with two
 // shuffles. Softmax statistics are per warp (merged across warps, then across chunks, in fixed
 // order). P*V: lane owns DH/32 output elements, probabilities are broadcast by shuffle.
 // The loop over query heads is a real loop (not unrolled) to keep this once-per-step code small.
@@ -676,8 +676,11 @@ __device__ __forceinline__ void attn_rows(Cta &c, const bf16_t *sk, const bf16_t
     const int Gq = p.Hq / p.Hkv, M = p.M;
     const int c0 = chunk * kAttnChunk;
     const int tl = c.warp * 8;                       // first token (within the chunk) of this warp
-    const int tkk = c.lane >> 2, part = c.lane & 3;
+    // lanes of a quarter-warp share `part`, so a 128-bit query load is one broadcast per quarter
+    // (with part = lane & 3 the four parts of a quarter hit the same banks: 4x the wavefronts)
+    const int tkk = c.lane & 7, part = c.lane >> 3;
     const int e0 = c.lane * EPL;
+    const uint32_t qs_u32 = smem_u32(qs);
     // this warp's K slice (token tkk, quarter `part`) and V rows (8 tokens x EPL elements) in registers
     float kf[SEG], vf[8][EPL];
     {
@@ -702,39 +705,46 @@ __device__ __forceinline__ void attn_rows(Cta &c, const bf16_t *sk, const bf16_t
             }
         }
     }
+    PROF(c);
 #pragma unroll 1
     for (int m = 0; m < M; ++m) {
         const int npos = min(base + m, max_tokens - 1);   // last visible position of this row
         const int nvis = min(8, npos - (c0 + tl) + 1);    // visible tokens of this warp (may be <= 0)
 #pragma unroll 1
         for (int h = 0; h < Gq; ++h) {
-            float s = 0.f;
-            const float4 *qv = reinterpret_cast<const float4 *>(qs + (size_t)(m * Gq + h) * DH + part * SEG);
+            // all query loads first (explicit shared-memory loads), then four independent partial sums
+            const uint32_t qa = qs_u32 + (uint32_t)(((m * Gq + h) * DH + part * SEG) * 4);
+            uint4 qw[SEG / 4];
+#pragma unroll
+            for (int i = 0; i < SEG / 4; ++i) qw[i] = lds128_u32(qa + 16 * i);
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
             for (int i = 0; i < SEG / 4; ++i) {
-                float4 q4 = qv[i];
-                s += q4.x * kf[4 * i] + q4.y * kf[4 * i + 1];
-                s += q4.z * kf[4 * i + 2] + q4.w * kf[4 * i + 3];
+                s0 += __uint_as_float(qw[i].x) * kf[4 * i];
+                s1 += __uint_as_float(qw[i].y) * kf[4 * i + 1];
+                s2 += __uint_as_float(qw[i].z) * kf[4 * i + 2];
+                s3 += __uint_as_float(qw[i].w) * kf[4 * i + 3];
             }
-            s += __shfl_xor_sync(0xffffffffu, s, 1);
-            s += __shfl_xor_sync(0xffffffffu, s, 2);
+            float s = (s0 + s1) + (s2 + s3);
+            s += __shfl_xor_sync(0xffffffffu, s, 8);
+            s += __shfl_xor_sync(0xffffffffu, s, 16);
             if (tkk >= nvis) s = -INFINITY;
             float mx = s;
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
             const float pe = (s == -INFINITY) ? 0.f : expf(s - mx);
             float sm = pe;
+            sm += __shfl_xor_sync(0xffffffffu, sm, 1);
+            sm += __shfl_xor_sync(0xffffffffu, sm, 2);
             sm += __shfl_xor_sync(0xffffffffu, sm, 4);
-            sm += __shfl_xor_sync(0xffffffffu, sm, 8);
-            sm += __shfl_xor_sync(0xffffffffu, sm, 16);
             // o[e] = sum over the warp's tokens (ascending) of p * V
             float o[EPL];
 #pragma unroll
             for (int e = 0; e < EPL; ++e) o[e] = 0.f;
 #pragma unroll
             for (int tk = 0; tk < 8; ++tk) {
-                const float pr = __shfl_sync(0xffffffffu, pe, tk * 4);
+                const float pr = __shfl_sync(0xffffffffu, pe, tk);
                 if (tk < nvis) {
 #pragma unroll
                     for (int e = 0; e < EPL; ++e) o[e] += pr * vf[tk][e];
@@ -745,7 +755,9 @@ __device__ __forceinline__ void attn_rows(Cta &c, const bf16_t *sk, const bf16_t
             for (int e = 0; e < EPL; ++e) w[e0 + e] = o[e];
             if (c.lane == 0) { w[DH] = mx; w[DH + 1] = sm; }
         }
+        PROF(c);
         bar_sync(1, kConsumerThreads);
+        PROF(c);
         // ---- merge the 8 warps (fixed order) -> chunk partial in global memory.
         // weight of warp w for head h: thread (h, w) computes it once
         float *fw = wp + (size_t)kConsumerWarps * Gq * wstride;      // [Gq][8] weights, then [Gq][2] (m, l)
@@ -759,6 +771,7 @@ __device__ __forceinline__ void attn_rows(Cta &c, const bf16_t *sk, const bf16_t
             if (w == 0) fw[Gq * kConsumerWarps + 2 * h] = mx;
         }
         bar_sync(1, kConsumerThreads);
+        PROF(c);
         for (int i = c.tid; i < Gq * DH; i += kConsumerThreads) {
             const int h = i / DH, e = i - h * DH;
             float ov = 0.f, l = 0.f;
