@@ -357,14 +357,41 @@ __device__ __forceinline__ void store_split(bf16_t *hi, bf16_t *lo, size_t idx, 
     lo[idx] = l;
 }
 
+// Operands of the epilogue that do not depend on the dot product (residual value, norm gains, the
+// token id of a head row): loaded when the tile starts, so their latency hides behind the stream.
+struct EpiPre { float resid, g0, g1; int id; };
+__device__ __forceinline__ EpiPre epi_prefetch(const Cta &c, int kind, const EpiCtx &x, int row, int col, bool valid) {
+    const MegaParams &p = *c.p;
+    EpiPre e;
+    e.resid = 0.f; e.g0 = 0.f; e.g1 = 0.f; e.id = row;
+    if (!valid) return e;
+    switch (kind) {
+        case PROJ: e.g0 = bf16bits_f32(x.L->g_in[row]); break;
+        case OPROJ:
+            e.resid = ldcg_f32(p.s.x0 + (size_t)col * p.d + row);
+            e.g0 = bf16bits_f32(x.L->g_post[row]);
+            break;
+        case DOWN:
+            e.resid = ldcg_f32(p.s.x1 + (size_t)col * p.d + row);
+            e.g0 = bf16bits_f32(x.gnext[row]);
+            if (p.mode == 0) e.g1 = bf16bits_f32(p.g_hnorm[row]);
+            break;
+        case HEAD:
+            if (p.ids) e.id = p.ids[row];
+            break;
+        default: break;
+    }
+    return e;
+}
+
 // Epilogue of one (virtual row, activation row): what the phase does with the finished dot product.
-__device__ __forceinline__ void epilogue(const Cta &c, int kind, EpiCtx &x, int row, int col, float v, float up) {
+__device__ __forceinline__ void epilogue(const Cta &c, int kind, EpiCtx &x, const EpiPre &pre, int row, int col, float v, float up) {
     const MegaParams &p = *c.p;
     const Scratch &s = p.s;
     switch (kind) {
         case PROJ: {
             s.x0[(size_t)col * p.d + row] = v;
-            store_split(s.actD_hi, s.actD_lo, (size_t)col * p.dp + row, v * bf16bits_f32(x.L->g_in[row]));
+            store_split(s.actD_hi, s.actD_lo, (size_t)col * p.dp + row, v * pre.g0);
             x.sq.a += v * v;
             break;
         }
@@ -372,9 +399,9 @@ __device__ __forceinline__ void epilogue(const Cta &c, int kind, EpiCtx &x, int 
             s.qkv[(size_t)col * (p.qdim + 2 * p.kvdim) + row] = v * c.misc->scale0[col];
             break;
         case OPROJ: {
-            float r = ldcg_f32(s.x0 + (size_t)col * p.d + row) + v;
+            float r = pre.resid + v;
             s.x1[(size_t)col * p.d + row] = r;
-            store_split(s.actP_hi, s.actP_lo, (size_t)col * p.dp + row, r * bf16bits_f32(x.L->g_post[row]));
+            store_split(s.actP_hi, s.actP_lo, (size_t)col * p.dp + row, r * pre.g0);
             x.sq.a += r * r;
             break;
         }
@@ -385,8 +412,8 @@ __device__ __forceinline__ void epilogue(const Cta &c, int kind, EpiCtx &x, int 
             break;
         }
         case DOWN: {
-            float r = ldcg_f32(s.x1 + (size_t)col * p.d + row) + v;
-            float y = r * bf16bits_f32(x.gnext[row]);
+            float r = pre.resid + v;
+            float y = r * pre.g0;
             x.sq.a += r * r;
             if (x.to_next_layer) {
                 s.x0[(size_t)col * p.d + row] = r;
@@ -394,14 +421,14 @@ __device__ __forceinline__ void epilogue(const Cta &c, int kind, EpiCtx &x, int 
             } else {
                 store_split(s.actH_hi, s.actH_lo, (size_t)col * p.dp + row, y);
                 if (p.mode == 0) {
-                    store_split(s.actR_hi, s.actR_lo, (size_t)col * p.dp + row, y * bf16bits_f32(p.g_hnorm[row]));
+                    store_split(s.actR_hi, s.actR_lo, (size_t)col * p.dp + row, y * pre.g1);
                     x.sq.b += y * y;
                 }
             }
             break;
         }
         default: {   // HEAD
-            int id = p.ids ? p.ids[row] : row;
+            int id = pre.id;
             if ((unsigned)id >= (unsigned)p.V) id = 0;
             float lv = v;
             if (p.mode == 1) {
@@ -478,6 +505,9 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
     const uint4 zero = make_uint4(0, 0, 0, 0);
     for (int vr0 = geo.v0; vr0 < geo.v1; vr0 += geo.cap) {
         const int nv = min(geo.cap, geo.v1 - vr0);
+        const int erow = c.tid >> 3, ecol = c.tid & 7;               // this thread's epilogue element
+        const bool evalid = erow < ((kind == GATEUP) ? min(nv, 16) : nv) && ecol < R;
+        const EpiPre pre = epi_prefetch(c, kind, ex, vr0 + erow, ecol, evalid);
         float acc[2][2][4], acd[2][2][4], acc0[2][4], acd0[2][4];
 #pragma unroll
         for (int i = 0; i < 2; ++i)
@@ -565,9 +595,8 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
         bar_sync(1, kConsumerThreads);
         {
             const float *rb = c.red + (size_t)c.redbuf * kConsumerWarps * kTileRows * R;
-            const int row = c.tid >> 3, col = c.tid & 7;
-            const int rlim = (kind == GATEUP) ? min(nv, 16) : nv;
-            if (row < rlim && col < R) {
+            const int row = erow, col = ecol;
+            if (evalid) {
                 float a = 0.f, b = 0.f;
 #pragma unroll
                 for (int w = 0; w < kConsumerWarps; ++w) a += rb[(size_t)w * kTileRows * R + row * R + col];
@@ -575,7 +604,7 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
 #pragma unroll
                     for (int w = 0; w < kConsumerWarps; ++w) b += rb[(size_t)w * kTileRows * R + (row + 16) * R + col];
                 }
-                epilogue(c, kind, ex, vr0 + row, col, a, b);
+                epilogue(c, kind, ex, pre, vr0 + row, col, a, b);
             }
         }
         c.redbuf ^= 1;
@@ -634,19 +663,27 @@ __device__ __forceinline__ void stage_hilo(const Cta &c, const bf16_t *ghi, cons
 }
 
 __device__ __forceinline__ void flush_sq(const Cta &c, const SqAcc &q, float *tblA, float *tblB) {
-    // thread (row = tid>>3, col = tid&7)
-    int row = c.tid >> 3, col = c.tid & 7;
-    for (int which = 0; which < 2; ++which) {
-        float *tbl = which ? tblB : tblA;
-        if (!tbl) continue;
-        bar_sync(1, kConsumerThreads);
-        c.misc->colred[row][col] = which ? q.b : q.a;
-        bar_sync(1, kConsumerThreads);
-        if (c.tid < kMaxRows) {
-            float s = 0.f;
-            for (int i = 0; i < kTileRows; ++i) s += c.misc->colred[i][c.tid];
-            tbl[(size_t)c.cta * kMaxRows + c.tid] = s;
+    // thread (row slot = tid>>3, col = tid&7): the four row slots of a warp are added by shuffle, the
+    // eight warps in ascending order by the first eight threads
+    float a = q.a, b = q.b;
+    a += __shfl_xor_sync(0xffffffffu, a, 8);
+    a += __shfl_xor_sync(0xffffffffu, a, 16);
+    b += __shfl_xor_sync(0xffffffffu, b, 8);
+    b += __shfl_xor_sync(0xffffffffu, b, 16);
+    if (c.lane < kMaxRows) {
+        c.misc->colred[c.warp][c.lane] = a;
+        c.misc->colred[kConsumerWarps + c.warp][c.lane] = b;
+    }
+    bar_sync(1, kConsumerThreads);
+    if (c.tid < kMaxRows) {
+        float sa = 0.f, sb = 0.f;
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) {
+            sa += c.misc->colred[w][c.tid];
+            sb += c.misc->colred[kConsumerWarps + w][c.tid];
         }
+        if (tblA) tblA[(size_t)c.cta * kMaxRows + c.tid] = sa;
+        if (tblB) tblB[(size_t)c.cta * kMaxRows + c.tid] = sb;
     }
 }
 
