@@ -148,10 +148,9 @@ int configure(fmtp_ctx *c, MegaParams &p, int mode, int B, int M) {
     size_t avail = (size_t)c->smem_optin;
     int st_noF = fixed + base < avail ? (int)((avail - fixed - base) / p.stage_bytes) : 0;
     int st_F = fixed + withF < avail ? (int)((avail - fixed - withF) / p.stage_bytes) : 0;
-    bool useF;
-    if (c->stage_F_pref == 0) useF = false;
-    else if (c->stage_F_pref == 1) useF = st_F >= 2;
-    else useF = st_F >= 4 || st_F >= st_noF;
+    // the ffn-wide input of the down projection is used once per CTA, so by default it is read from
+    // global memory (fetched one stage ahead) and the shared memory goes to a deeper ring
+    bool useF = (c->stage_F_pref == 1) && st_F >= 2;
     p.stage_F_in_smem = useF ? 1 : 0;
     p.scratch_smem = (int)(useF ? withF : base);
     int ns = useF ? st_F : st_noF;

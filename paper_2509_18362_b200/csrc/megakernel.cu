@@ -516,11 +516,22 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
                 acc[i][0][j] = acc[i][1][j] = acd[i][0][j] = acd[i][1][j] = 0.f;
                 acc0[i][j] = acd0[i][j] = 0.f;
             }
+        // activations read from global memory (the ffn-wide vector of the down projection is not staged
+        // in shared memory): this warp's four B fragments of its next stage are fetched one stage ahead
+        uint4 bnext[4] = {zero, zero, zero, zero};
+        const bool gfast = !two_sets && !act.in_smem && (geo.K % p.KC) == 0 && p.KC == 512;
         bool moved = false;
         // which half of the warps takes a stage depends only on the stage's index within the phase,
         // never on how many stages the CTA has seen before: the summation order of a row must not
         // depend on the batch or on earlier calls
         const int stage0 = ((vr0 - geo.v0) / geo.cap) * geo.nks;
+        if (gfast && has0) {
+            const int ks0 = ((stage0 & 1) == grp) ? 0 : 1;          // first stage this warp owns
+            if (ks0 < geo.nks) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) bnext[j] = ldcg128(abase + aoff0 + (size_t)ks0 * p.KC + (wi + 4 * j) * 32);
+            }
+        }
 #pragma unroll 1
         for (int ks = 0; ks < geo.nks; ++ks) {
             if (((stage0 + ks) & 1) == grp) {
@@ -538,19 +549,29 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
                 const uint32_t sb = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + t * 16 + g * rs;
                 const size_t kbase = (size_t)ks * p.KC;
                 // chunks wi, wi+4, wi+8, wi+12
-                if (!two_sets && nchunk == 16 && act.in_smem) {
-                    // common case (full 512-wide stage, at most four activation rows staged in shared
-                    // memory): two batches of two chunks, all loads of a batch issued before its MMAs
-                    const uint32_t ab = smem_u32(abase + aoff0 + kbase);
+                if (!two_sets && nchunk == 16 && (act.in_smem || gfast)) {
+                    // common case (full 512-wide stage, at most four activation rows): two batches of
+                    // two chunks, all loads of a batch issued before its MMAs
+                    uint4 bq[4];
+                    if (act.in_smem) {
+                        const uint32_t ab = smem_u32(abase + aoff0 + kbase);
 #pragma unroll
-                    for (int ch = wi; ch < 16; ch += 8) {
-                        uint4 b0 = zero, b1 = zero;
+                        for (int j = 0; j < 4; ++j) bq[j] = has0 ? lds128_u32(ab + (wi + 4 * j) * 64) : zero;
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) bq[j] = bnext[j];
+                        if (has0 && ks + 2 < geo.nks) {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) bnext[j] = ldcg128(abase + aoff0 + kbase + 2 * p.KC + (wi + 4 * j) * 32);
+                        }
+                    }
+#pragma unroll
+                    for (int b2 = 0; b2 < 2; ++b2) {
+                        const int ch = wi + 8 * b2;
                         Frag f0 = load_frag(sb + ch * 64, rs);
-                        if (has0) b0 = lds128_u32(ab + ch * 64);
                         Frag f1 = load_frag(sb + (ch + 4) * 64, rs);
-                        if (has0) b1 = lds128_u32(ab + (ch + 4) * 64);
-                        mma_chunk(acc, f0, b0);
-                        mma_chunk(acc, f1, b1);
+                        mma_chunk(acc, f0, bq[2 * b2]);
+                        mma_chunk(acc, f1, bq[2 * b2 + 1]);
                     }
                 } else {
 #pragma unroll 1
