@@ -122,18 +122,22 @@ int configure(fmtp_ctx *c, MegaParams &p, int mode, int B, int M) {
     p.dp = c->dp; p.qp = c->qp; p.Fp = c->Fp;
     p.eps = sh.rms_eps;
     p.KC = c->KC;
-    p.row_stride = p.KC * 2 + 64;
+    p.row_stride = p.KC * 2;
     p.stage_bytes = kTileRows * p.row_stride;
     {   // a stage also has to hold one 64-token K/V chunk of a KV head
         int kvb = 2 * kAttnChunk * p.dh * 2;
         if (kvb > p.stage_bytes) p.stage_bytes = kvb;
+        // ... and, once K/V sit in registers, the per-warp attention partials that reuse the buffer
+        const int gq = p.Hq / p.Hkv;
+        int wpb = (kConsumerWarps * gq * (p.dh + 2) + gq * (kConsumerWarps + 2)) * 4;
+        if (wpb > p.stage_bytes) p.stage_bytes = wpb;
         p.stage_bytes = (p.stage_bytes + 127) & ~127;
     }
     p.max_chunks = c->max_chunks;
     p.max_ctx = sh.max_ctx;
     p.mode = mode; p.B = B; p.M = M; p.R = B * M;
     const int R = p.R, Gq = p.Hq / p.Hkv;
-    size_t attn = ((size_t)M * Gq * p.dh + (size_t)kConsumerWarps * Gq * (p.dh + 2) + (size_t)Gq * (kConsumerWarps + 2)) * 4;
+    size_t attn = (size_t)M * Gq * p.dh * 4;
     size_t mrg = ((size_t)2 * c->max_chunks + (size_t)kConsumerThreads + 64) * 4;      // chunk-merge scratch
     if (mrg > attn) attn = mrg;
     size_t actd = (size_t)2 * R * act_stride(mode == 0 ? 2 * p.d : (p.d > p.qdim ? p.d : p.qdim)) * 2;

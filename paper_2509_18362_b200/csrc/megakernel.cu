@@ -267,7 +267,11 @@ __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs 
     const unsigned char *cur[kRowsPerProducer], *nxt[kRowsPerProducer];
 #pragma unroll
     for (int i = 0; i < kRowsPerProducer; ++i) nxt[i] = nullptr;
+    // rows are stored without padding; in odd rows the two 64-byte halves of every 128 bytes are
+    // swapped, which keeps the consumers' 128-bit fragment loads free of bank conflicts. All rows of a
+    // producer warp have the parity of pw.
     const uint32_t lane16 = (uint32_t)c.lane * 16u;
+    const uint32_t lane16d = (uint32_t)(c.lane ^ ((pw & 1) << 2)) * 16u;
     const uint32_t rs = (uint32_t)p.row_stride;
     // the loop starts one tile early: iteration t fetches the pointers of tile t + 1
 #pragma unroll 1
@@ -287,7 +291,7 @@ __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs 
             PROF_ACC(c, 2, pw == 0 && c.lane == 0);
             if (!ok) return;   // abort: stop issuing copies
             const int klen = min(p.KC, g.K - ks * p.KC);
-            const uint32_t dst0 = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + (uint32_t)pw * rs + lane16;
+            const uint32_t dst0 = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + (uint32_t)pw * rs + lane16d;
             const size_t koff = (size_t)ks * p.KC * 2 + lane16;
             if (klen == 512) {
                 // 1024 bytes per row: two instructions per row, sixteen per thread, all with their own
@@ -547,6 +551,7 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
                 const int klen = min(p.KC, geo.K - ks * p.KC);
                 const int nchunk = (klen + 31) >> 5;
                 const uint32_t sb = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + t * 16 + g * rs;
+                const int par = g & 1;                    // odd rows: 64-byte halves swapped
                 const size_t kbase = (size_t)ks * p.KC;
                 // chunks wi, wi+4, wi+8, wi+12
                 if (!two_sets && nchunk == 16 && (act.in_smem || gfast)) {
@@ -568,15 +573,15 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
 #pragma unroll
                     for (int b2 = 0; b2 < 2; ++b2) {
                         const int ch = wi + 8 * b2;
-                        Frag f0 = load_frag(sb + ch * 64, rs);
-                        Frag f1 = load_frag(sb + (ch + 4) * 64, rs);
+                        Frag f0 = load_frag(sb + (ch ^ par) * 64, rs);
+                        Frag f1 = load_frag(sb + ((ch + 4) ^ par) * 64, rs);
                         mma_chunk(acc, f0, bq[2 * b2]);
                         mma_chunk(acc, f1, bq[2 * b2 + 1]);
                     }
                 } else {
 #pragma unroll 1
                     for (int ch = wi; ch < nchunk; ch += 4) {
-                        Frag f0 = load_frag(sb + ch * 64, rs);
+                        Frag f0 = load_frag(sb + (ch ^ par) * 64, rs);
                         uint4 b0 = zero, d0 = zero;
                         if (has0) b0 = act.in_smem ? lds128(abase + aoff0 + kbase + ch * 32) : ldcg128(abase + aoff0 + kbase + ch * 32);
                         if (has1) d0 = act.in_smem ? lds128(abase + aoff1 + kbase + ch * 32) : ldcg128(abase + aoff1 + kbase + ch * 32);
@@ -718,8 +723,8 @@ __device__ __forceinline__ void flush_sq(const Cta &c, const SqAcc &q, float *tb
 // the 64 K rows. The consumers add the positions this launch produced (earlier draft steps from
 // the pages, this call's rows from the QKV scratch, rotated and rounded to bf16 exactly as they
 // are stored) into the same stage buffer and then work from shared memory only.
-// Scratch layout (floats): qs[M*Gq][dh] rotated, pre-scaled queries of one KV head;
-// wp[8 warps][Gq][dh + 2] per-warp partial (o, m, l) of the row being processed.
+// Scratch: qs[M*Gq][dh] rotated, pre-scaled queries of one KV head. The per-warp partials
+// wp[8 warps][Gq][dh + 2] (o, m, l) reuse the stage buffer once K and V are in registers.
 
 // One chunk of one KV head from shared memory, for every row of the call: each warp takes 8 tokens.
 // Scores: lane = (quarter of the head dimension, token); the four quarters are added with two
@@ -727,7 +732,7 @@ __device__ __forceinline__ void flush_sq(const Cta &c, const SqAcc &q, float *tb
 // order). P*V: lane owns DH/32 output elements, probabilities are broadcast by shuffle.
 // The loop over query heads is a real loop (not unrolled) to keep this once-per-step code small.
 template <int DH>
-__device__ __forceinline__ void attn_rows(Cta &c, const bf16_t *sk, const bf16_t *sv, const float *qs, float *wp,
+__device__ __forceinline__ void attn_rows(Cta &c, bf16_t *sk, const bf16_t *sv, const float *qs,
                                           int b, int kvh, int chunk, int base, int max_tokens) {
     const MegaParams &p = *c.p;
     constexpr int SEG = DH / 4, EPL = DH / 32, wstride = DH + 2;
@@ -763,6 +768,10 @@ __device__ __forceinline__ void attn_rows(Cta &c, const bf16_t *sk, const bf16_t
             }
         }
     }
+    // K and V now live in registers: the stage buffer is reused for the per-warp partials
+    // wp[8 warps][Gq][DH + 2] (o, m, l) and the merge weights behind them
+    bar_sync(1, kConsumerThreads);
+    float *wp = reinterpret_cast<float *>(sk);
     PROF(c);
 #pragma unroll 1
     for (int m = 0; m < M; ++m) {
@@ -924,7 +933,6 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
     constexpr int dh = DH, half = DH >> 1;
     const int Gq = p.Hq / p.Hkv, M = p.M;
     float *qs = reinterpret_cast<float *>(c.scr);
-    float *wp = qs + (size_t)M * Gq * dh;
     const float qscale = rsqrtf((float)dh);
     const int max_tokens = min(kv.max_pages * p.page, p.max_ctx);   // positions beyond are flagged, not touched
     const int upt = dh >> 3;
@@ -993,7 +1001,7 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
         bar_sync(1, kConsumerThreads);
         PROF(c);
 
-        attn_rows<DH>(c, sk, sv, qs, wp, b, kvh, chunk, base, max_tokens);
+        attn_rows<DH>(c, sk, sv, qs, b, kvh, chunk, base, max_tokens);
         PROF(c);
         // the stage is free again (all consumer warps passed the barrier at the end of attn_rows)
         if (c.warp < kConsumerWarps / 2 && c.lane == 0) mbar_arrive(&c.misc->empty[slot]);
