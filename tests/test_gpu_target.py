@@ -149,27 +149,27 @@ def _gpu_greedy(gpu, prompt, n_new):
     return out
 
 
-def test_speculative_loop_is_token_identical_to_greedy_on_gpu():
-    """Draft with the MTP head, score [last, drafts] with the target in one call, accept with
-    fastmtp_verify_accept: the emitted sequence equals plain greedy decoding by the same
-    library; and the first tokens agree with the oracle's greedy run up to near ties."""
+def speculative_vs_greedy(shape, seed, K, n_new, prompt_len, N, max_ctx, n_oracle):
+    """Greedy decoding and speculative decoding (MTP drafts, every other round drafts that are right for a
+    planted number of positions) by the library on the same random model; returns both token lists and
+    the accepted lengths, after checking the first n_oracle greedy tokens against the oracle."""
     Bd = _binding()
-    shape = I.TINY.with_layers(2)
-    K, n_new = 3, 40
-    Wt = I.target_weights(shape, 501)
-    Wm = I.mtp_weights(shape, 502, embed=Wt["embed"], lm_head=Wt["lm_head"])
-    prompt = [int(t) for t in I.token_ids(503, (19,), shape.vocab)]
-    ids = I.subset_uniform(shape.vocab, 1024, 504)
-    mk = lambda: [I.empty_paged_kv(shape, 1, 128, 510 + l) for l in range(2)]
+    L = shape.n_layers
+    Wt = I.target_weights(shape, seed)
+    Wm = I.mtp_weights(shape, seed + 1, embed=Wt["embed"], lm_head=Wt["lm_head"])
+    prompt = [int(t) for t in I.token_ids(seed + 2, (prompt_len,), shape.vocab)]
+    ids = I.subset_uniform(shape.vocab, N, seed + 3)
+    mk = lambda: [I.empty_paged_kv(shape, 1, max_ctx, seed + 10 + l) for l in range(L)]
 
-    g = GpuTarget(shape, Wt, mk(), 128)
+    g = GpuTarget(shape, Wt, mk(), max_ctx)
     ref = _gpu_greedy(g, prompt, n_new + K + 1)
     g.close()
 
-    gpu = GpuTarget(shape, Wt, mk(), 128)
-    dWm = Bd.to_device(Wm)
+    gpu = GpuTarget(shape, Wt, mk(), max_ctx)
+    dWm = dict(Bd.to_device({k: v for k, v in Wm.items() if k not in ("embed", "lm_head")}),
+               embed=gpu.dW["embed"], lm_head=gpu.dW["lm_head"])          # shared with the target, one copy
     wm = Bd.mtp_w(dWm)
-    mkv = Bd.to_device(I.empty_paged_kv(shape, 1, 128, 520))
+    mkv = Bd.to_device(I.empty_paged_kv(shape, 1, max_ctx, seed + 20))
     dids = torch.from_numpy(ids).cuda()
     # prefill the target; feed the MTP cache with pairs (h_j, t_{j+1}) one position per call
     hs = []
@@ -217,19 +217,29 @@ def test_speculative_loop_is_token_identical_to_greedy_on_gpu():
         pend_t = new
         rnd += 1
     gpu.close()
-    assert out[:n_new] == ref[:n_new]
-    assert {0, 1, 2, 3} <= set(accepted)
 
-    # oracle greedy on the first tokens, teacher-forced on near ties
+    # oracle greedy on the first tokens, teacher-forced on near ties (logits of the newest row only)
     okvs = mk()
-    _, lg = O.target_forward(shape, Wt, np.array([prompt]), okvs)
+    hh, _ = O.target_forward(shape, Wt, np.array([prompt]), okvs, want_logits=False)
     for kv in okvs:
         kv["seq_lens"][0] = len(prompt)
-    row = lg[0, -1]
-    for i in range(12):
+    row = O.head_logits(hh[0, -1], Wt["lm_head"])
+    for i in range(n_oracle):
         t, _ = O.argmax_token(O.round_bf16(row))
         assert t == ref[i] or _bf16_gap(row) < GAP_TOL, f"token {i}: oracle {t}, gpu {ref[i]}"
-        _, lg = O.target_forward(shape, Wt, np.array([[ref[i]]]), okvs)
+        hh, _ = O.target_forward(shape, Wt, np.array([[ref[i]]]), okvs, want_logits=False)
         for kv in okvs:
             kv["seq_lens"][0] += 1
-        row = lg[0, 0]
+        row = O.head_logits(hh[0, 0], Wt["lm_head"])
+    O.clear_weight_memo()
+    return ref, out, accepted
+
+
+def test_speculative_loop_is_token_identical_to_greedy_on_gpu():
+    """Draft with the MTP head, score [last, drafts] with the target in one call, accept with
+    fastmtp_verify_accept: the emitted sequence equals plain greedy decoding by the same
+    library; and the first tokens agree with the oracle's greedy run up to near ties."""
+    K, n_new = 3, 40
+    ref, out, accepted = speculative_vs_greedy(I.TINY.with_layers(2), 501, K, n_new, 19, 1024, 128, 12)
+    assert out[:n_new] == ref[:n_new]
+    assert {0, 1, 2, 3} <= set(accepted)
