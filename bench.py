@@ -44,6 +44,8 @@ def parse_args():
     ap.add_argument("--shape", default="7b", choices=["7b", "tiny"])
     ap.add_argument("--seed", type=int, default=1234)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="vocabulary-compression sweep on one GPU: subset size x batch x draft steps, one JSON line each")
     return ap.parse_args()
 
 
@@ -350,8 +352,58 @@ def run_ours(a):
         dist.destroy_process_group()
 
 
+def run_sweep(a):
+    """Subset size {8192 .. full} (Zipf-weighted draws) x batch {1, 4} x K {1, 3, 5} on the 7B-class head at
+    context 2048: device-timed draft calls only, one JSON line per point."""
+    import torch
+    import __graft_entry__ as G
+    G.build()
+    from paper_2509_18362_b200 import binding as Bd
+    from paper_2509_18362_b200 import inputs as I
+    torch.cuda.set_device(0)
+    s = I.QWEN7B if a.shape == "7b" else I.TINY
+    W = I.mtp_weights(s, a.seed)
+    dW = Bd.to_device(W)
+    w = Bd.mtp_w(dW)
+    peak, peak_kind = load_peaks()
+    sizes = [8192, 16384, 32768, 65536, s.vocab] if a.shape == "7b" else [256, 1024, s.vocab]
+    for B in (1, 4):
+        ctx_lens = [a.ctx] * B
+        kv = I.paged_kv(s, ctx_lens, 6, a.seed + 1)
+        dkv = Bd.to_device(kv)
+        ckv = Bd.kv(dkv)
+        dh = Bd.bf16_tensor(I.hidden_bf16(a.seed + 2, (B, s.d)))
+        dtok = torch.from_numpy(I.token_ids(a.seed + 3, (B,), s.vocab)).cuda()
+        ctx = Bd.Context(s, max_rows=8, max_K=8, max_ctx=a.ctx + 8)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for N in sizes:
+            ids = None if N >= s.vocab else torch.from_numpy(I.subset_zipf(s.vocab, N, a.seed + 4)).cuda()
+            for K in (1, 3, 5):
+                out_d = torch.zeros((B, K), dtype=torch.int32, device="cuda")
+                for _ in range(5):
+                    ctx.fastmtp_draft(w, dh, dtok, ckv, B, K, ids, out_d, None, None, status)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                n = 50
+                e0.record()
+                for _ in range(n):
+                    ctx.fastmtp_draft(w, dh, dtok, ckv, B, K, ids, out_d, None, None, status)
+                e1.record()
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1) / n
+                nbytes = sum(algorithmic_bytes_per_draft_step(s, B, N, ctx_lens, k) for k in range(K))
+                print(json.dumps({"sweep": True, "subset": N, "batch": B, "draft_steps": K, "ctx": a.ctx,
+                                  "us_per_draft_step": ms * 1e3 / K, "draft_tokens_per_s": B * K / (ms * 1e-3),
+                                  "mb_per_step": nbytes / K / 1e6, "gbs": nbytes / (ms * 1e-3) / 1e9,
+                                  "frac_of_" + peak_kind: nbytes / (ms * 1e-3) / 1e9 / peak}), flush=True)
+        assert int(status.item()) == 0
+        ctx.close()
+
+
 def main():
     a = parse_args()
+    if a.sweep:
+        return run_sweep(a)
     if a.impl == "reference":
         run_reference(a)
     else:
