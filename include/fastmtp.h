@@ -58,7 +58,10 @@ typedef enum {
 /* Model geometry and capacity limits (fixed for the life of a context).
  * Supported: head_dim in {64, 128}; d, n_q_heads*head_dim and ffn multiples of 16 with
  * d a multiple of 64; n_q_heads a multiple of n_kv_heads with at most 8 query heads per
- * KV head; max_rows <= 8 (rows = batch x rows-per-sequence handled in one call). */
+ * KV head; max_rows <= 4096 (rows = batch x rows-per-sequence handled in one call). A call with
+ * more rows than one launch takes (8, fewer when the input vectors of that many rows do not fit
+ * in shared memory) runs as consecutive launches over groups of whole sequences on the same
+ * stream; a sequence's results do not depend on how the batch is grouped. */
 typedef struct {
     int32_t d, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
     int32_t n_layers;      /* target decoder depth (fastmtp_target_step); the MTP head has 1 */

@@ -61,7 +61,9 @@ struct Carver {
 // Lays the scratch buffers out inside the workspace (base == nullptr: size query only).
 size_t layout(fmtp_ctx *c, unsigned char *base) {
     const fmtp_shape &sh = c->shape;
-    const int R = sh.max_rows, d = sh.d;
+    const int R = sh.max_rows < kMaxRows ? sh.max_rows : kMaxRows;   // rows of one launch
+    const int RB = sh.max_rows;                                     // rows of one call (host staging)
+    const int d = sh.d;
     const int qdim = sh.n_q_heads * sh.head_dim, kvdim = sh.n_kv_heads * sh.head_dim;
     Carver cv;
     cv.base = base;
@@ -97,9 +99,9 @@ size_t layout(fmtp_ctx *c, unsigned char *base) {
     s.rope_sin = sinb;
     c->vkeys = cv.take<unsigned long long>(kVerifyMaxRows);
     c->vcounter = cv.take<uint32_t>(1);
-    c->st_h = cv.take<bf16_t>((size_t)R * d);
-    c->st_tok = cv.take<int32_t>((size_t)R);
-    c->st_out = cv.take<int32_t>((size_t)R * (sh.max_K > 1 ? sh.max_K : 1) + 2 * kVerifyMaxRows);
+    c->st_h = cv.take<bf16_t>((size_t)RB * d);
+    c->st_tok = cv.take<int32_t>((size_t)RB);
+    c->st_out = cv.take<int32_t>((size_t)RB * (sh.max_K > 1 ? sh.max_K : 1) + 2 * kVerifyMaxRows);
     c->st_status = cv.take<uint32_t>(1);
     return align_up(cv.off, 256);
 }
@@ -199,6 +201,21 @@ int launch_mega(fmtp_ctx *c, MegaParams &p, cudaStream_t st) {
     return FMTP_OK;
 }
 
+// Sequences per launch for a call of B sequences with M rows each: a call with more rows than one
+// launch takes runs as several launches over groups of whole sequences. The largest group is the
+// one whose input vectors still leave a ring of three stages (two at worst); 0 if even one
+// sequence does not fit.
+int group_size(fmtp_ctx *c, int mode, int B, int M) {
+    int gmax = kMaxRows / M;
+    if (gmax > B) gmax = B;
+    for (int want = 3; want >= 2; --want)
+        for (int g = gmax; g >= 1; --g) {
+            MegaParams tmp;
+            if (configure(c, tmp, mode, g, M) == FMTP_OK && tmp.n_stages >= want) return g;
+        }
+    return 0;
+}
+
 int status_to_code(uint32_t st) {
     if (st & FMTP_DEV_TIMEOUT) return FMTP_ETIMEOUT;
     if (st) return FMTP_EBOUNDS;
@@ -231,7 +248,7 @@ int fmtp_create(const fmtp_shape *sh, fmtp_ctx **out) {
         return FMTP_EINVAL;
     if (sh->head_dim != 64 && sh->head_dim != 128) return FMTP_ESHAPE;
     if (sh->d % 64 || sh->ffn % 16 || sh->n_q_heads % sh->n_kv_heads || sh->n_q_heads / sh->n_kv_heads > 8 ||
-        sh->max_rows > kMaxRows || sh->n_layers > kMaxLayers)
+        sh->max_rows > 4096 || sh->n_layers > kMaxLayers)
         return FMTP_ESHAPE;
     int dev = 0, major = 0, sms = 0, optin = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -259,6 +276,7 @@ int fmtp_create(const fmtp_shape *sh, fmtp_ctx **out) {
     c->stages_cap = kMaxStages;
     if (const char *v = std::getenv("FMTP_STAGES")) { int n = std::atoi(v); if (n >= 2 && n <= kMaxStages) c->stages_cap = n; }
     c->ws_need = layout(c, nullptr);
+    if (group_size(c, 0, kMaxRows, 1) < 1) { delete c; return FMTP_ESHAPE; }
     c->pinned_bytes = (size_t)sh->max_rows * sh->d * 2 + (size_t)sh->max_rows * 4 * (2 + (sh->max_K > 1 ? sh->max_K : 1)) +
                       2 * kVerifyMaxRows * 4 + 256;
     e = cudaMallocHost(&c->pinned, c->pinned_bytes);
@@ -319,23 +337,33 @@ int fastmtp_draft(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_last, con
     if (!aligned16(w->embed) || !aligned16(w->lm_head) || !aligned16(w->g_hnorm) || !aligned16(w->g_enorm) ||
         !aligned16(w->w_proj) || !aligned16(w->g_final) || !aligned16(h_last) || !layer_ok(w->layer) || !kv_ok(*kv))
         return FMTP_EINVAL;
-    MegaParams p;
-    int rc = configure(c, p, 0, B, 1);
-    if (rc) return rc;
-    p.K = K;
-    p.N = subset ? N : c->shape.vocab;
-    p.ids = subset;
-    p.h_last = h_last;
-    p.tokens = tok_last;
-    p.out_tokens = out_drafts;
-    p.out_h = out_h;
-    p.out_logits_f32 = out_logits;
-    p.user_status = dev_status;
-    p.embed = w->embed; p.lm_head = w->lm_head; p.g_hnorm = w->g_hnorm; p.g_enorm = w->g_enorm;
-    p.w_proj = w->w_proj; p.g_final = w->g_final;
-    set_layer(p.layers[0], w->layer);
-    set_kv(p.kvs[0], *kv);
-    return launch_mega(c, p, static_cast<cudaStream_t>(stream));
+    const int G = group_size(c, 0, B, 1);
+    if (G < 1) return FMTP_ESHAPE;
+    const int Neff = subset ? N : c->shape.vocab;
+    for (int b0 = 0; b0 < B; b0 += G) {
+        const int Bg = (B - b0 < G) ? B - b0 : G;
+        MegaParams p;
+        int rc = configure(c, p, 0, Bg, 1);
+        if (rc) return rc;
+        p.K = K;
+        p.N = Neff;
+        p.ids = subset;
+        p.h_last = h_last + (size_t)b0 * c->shape.d;
+        p.tokens = tok_last + b0;
+        p.out_tokens = out_drafts + (size_t)b0 * K;
+        p.out_h = out_h ? out_h + (size_t)b0 * K * c->shape.d : nullptr;
+        p.out_logits_f32 = out_logits ? out_logits + (size_t)b0 * K * Neff : nullptr;
+        p.user_status = dev_status;
+        p.embed = w->embed; p.lm_head = w->lm_head; p.g_hnorm = w->g_hnorm; p.g_enorm = w->g_enorm;
+        p.w_proj = w->w_proj; p.g_final = w->g_final;
+        set_layer(p.layers[0], w->layer);
+        set_kv(p.kvs[0], *kv);
+        p.kvs[0].block_table += (size_t)b0 * kv->max_pages_per_seq;
+        p.kvs[0].seq_lens += b0;
+        rc = launch_mega(c, p, static_cast<cudaStream_t>(stream));
+        if (rc) return rc;
+    }
+    return FMTP_OK;
 }
 
 int fastmtp_draft_host(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_host, const int32_t *tok_host,
@@ -433,21 +461,35 @@ int fastmtp_target_step(fmtp_ctx *c, const fmtp_target_w *w, const int32_t *toke
     if (!w->embed || !w->lm_head || !w->g_final || !w->layers) return FMTP_EINVAL;
     if (!aligned16(w->embed) || !aligned16(w->lm_head) || !aligned16(w->g_final)) return FMTP_EINVAL;
     for (int l = 0; l < nl; ++l) if (!layer_ok(w->layers[l]) || !kv_ok(kvs[l])) return FMTP_EINVAL;
-    MegaParams p;
-    int rc = configure(c, p, 1, B, M);
-    if (rc) return rc;
-    p.K = 1;
-    p.n_layers = nl;
-    p.N = c->shape.vocab;
-    p.ids = nullptr;
-    p.tokens = tokens;
-    p.out_tokens = out_argmax;
-    p.out_h = out_h;
-    p.out_logits_bf16 = out_logits;
-    p.user_status = dev_status;
-    p.embed = w->embed; p.lm_head = w->lm_head; p.g_final = w->g_final;
-    for (int l = 0; l < nl; ++l) { set_layer(p.layers[l], w->layers[l]); set_kv(p.kvs[l], kvs[l]); }
-    return launch_mega(c, p, static_cast<cudaStream_t>(stream));
+    if (M > kMaxRows) return FMTP_ESHAPE;                // the rows of one sequence share a launch
+    const int G = group_size(c, 1, B, M);
+    if (G < 1) return FMTP_ESHAPE;
+    const int V = c->shape.vocab, d = c->shape.d;
+    for (int b0 = 0; b0 < B; b0 += G) {
+        const int Bg = (B - b0 < G) ? B - b0 : G;
+        MegaParams p;
+        int rc = configure(c, p, 1, Bg, M);
+        if (rc) return rc;
+        p.K = 1;
+        p.n_layers = nl;
+        p.N = V;
+        p.ids = nullptr;
+        p.tokens = tokens + (size_t)b0 * M;
+        p.out_tokens = out_argmax ? out_argmax + (size_t)b0 * M : nullptr;
+        p.out_h = out_h ? out_h + (size_t)b0 * M * d : nullptr;
+        p.out_logits_bf16 = out_logits ? out_logits + (size_t)b0 * M * V : nullptr;
+        p.user_status = dev_status;
+        p.embed = w->embed; p.lm_head = w->lm_head; p.g_final = w->g_final;
+        for (int l = 0; l < nl; ++l) {
+            set_layer(p.layers[l], w->layers[l]);
+            set_kv(p.kvs[l], kvs[l]);
+            p.kvs[l].block_table += (size_t)b0 * kvs[l].max_pages_per_seq;
+            p.kvs[l].seq_lens += b0;
+        }
+        rc = launch_mega(c, p, static_cast<cudaStream_t>(stream));
+        if (rc) return rc;
+    }
+    return FMTP_OK;
 }
 
 }  // extern "C"

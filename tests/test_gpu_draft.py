@@ -30,7 +30,7 @@ def run_draft_case(shape, seed, B, L, K, N, subset="uniform", want_logits=True, 
         ids = I.subset_zipf(shape.vocab, N, seed + 4)
     n_head = shape.vocab if ids is None else len(ids)
 
-    ctx = Bd.Context(shape, max_rows=8, max_K=8, max_ctx=max_ctx or (max(L) + K + 1))
+    ctx = Bd.Context(shape, max_rows=max(8, B), max_K=8, max_ctx=max_ctx or (max(L) + K + 1))
     dW = Bd.to_device(W)
     dkv = Bd.to_device(copy_kv(kv))
     dh = Bd.bf16_tensor(h)
@@ -90,6 +90,14 @@ def test_tiny_config_batch1():
 def test_tiny_shapes_ragged(B, L, K, N):
     got, ref = run_draft_case(I.TINY, 77 + B, B, L, K, N)
     check_draft(got, ref, f"tiny B={B} K={K} N={N}")
+
+
+def test_batch_larger_than_one_launch():
+    """20 sequences with ragged contexts: three launches (8 + 8 + 4 rows) behind one call."""
+    L = [int(x) for x in I.context_lengths(20, 0, 200, 9)]
+    got, ref = run_draft_case(I.TINY, 808, 20, L, 3, 1024, subset="zipf")
+    check_draft(got, ref, "tiny B=20")
+    assert got["launches"] == 3
 
 
 def test_odd_geometry():

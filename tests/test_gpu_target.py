@@ -108,6 +108,30 @@ def test_target_step_prefill_decode_verify(n_layers):
     gpu.close()
 
 
+def test_target_step_more_rows_than_one_launch():
+    """5 sequences x 4 rows = 20 rows: the call runs groups of two sequences (8 rows) per launch."""
+    shape = I.TINY.with_layers(2)
+    Wt = I.target_weights(shape, 611)
+    B, M = 5, 4
+    kvs = [I.empty_paged_kv(shape, B, 32, 620 + l) for l in range(2)]
+    okvs = [copy_kv(kv) for kv in kvs]
+    Bd = _binding()
+    gpu = GpuTarget(shape, Wt, kvs, 64)
+    gpu.ctx.close()
+    gpu.ctx = Bd.Context(shape, max_rows=32, max_K=8, max_ctx=64)
+    for it in range(2):
+        t = I.token_ids(630 + it, (B, M), shape.vocab)
+        h, l, a = gpu.step(t)
+        rh, rl = O.target_forward(shape, Wt, t, okvs)
+        close(h.float().cpu().numpy(), rh, "target h 20 rows")
+        close(l.float().cpu().numpy(), rl, "target logits 20 rows")
+        gpu.advance(M)
+        for kv in okvs:
+            kv["seq_lens"] += M
+    assert gpu.ctx.launch_count == 6
+    gpu.close()
+
+
 def test_rows_do_not_depend_on_rows_per_call():
     """A position's hidden state and logits are bit-identical whether it is scored alone (M=1)
     or as one of several rows (M=4): the property that makes verification lossless."""
