@@ -40,6 +40,8 @@ def parse_args():
     ap.add_argument("--subset", type=int, default=32768, help="compressed vocabulary size (0 = full vocabulary)")
     ap.add_argument("--subset-kind", default="uniform", choices=["uniform", "zipf"])
     ap.add_argument("--ctx", type=int, default=2048, help="cached context tokens per sequence")
+    ap.add_argument("--ctx-min", type=int, default=0, help="with --ctx-max: ragged contexts, uniform integers in [min, max]")
+    ap.add_argument("--ctx-max", type=int, default=0)
     ap.add_argument("--draft-steps", type=int, default=3)
     ap.add_argument("--shape", default="7b", choices=["7b", "tiny"])
     ap.add_argument("--seed", type=int, default=1234)
@@ -128,7 +130,10 @@ def make_inputs(a, rank):
     N = a.subset if 0 < a.subset < s.vocab else s.vocab
     K = a.draft_steps
     W = I.mtp_weights(s, a.seed)                     # same model on every replica
-    ctx_lens = [a.ctx] * a.batch
+    if a.ctx_max > 0:
+        ctx_lens = [int(x) for x in I.context_lengths(a.batch, a.ctx_min, a.ctx_max, seed + 6)]
+    else:
+        ctx_lens = [a.ctx] * a.batch
     kv = I.paged_kv(s, ctx_lens, K + 1, seed + 1)
     h = I.hidden_bf16(seed + 2, (a.batch, s.d))
     tok = I.token_ids(seed + 3, (a.batch,), s.vocab)
@@ -144,7 +149,8 @@ def make_inputs(a, rank):
 
 def workload_name(a, s, N):
     return (f"{a.shape} MTP head draft+verify: d={s.d} Hq/Hkv={s.n_q_heads}/{s.n_kv_heads} dh={s.head_dim} "
-            f"ffn={s.ffn} V={s.vocab} subset={N}({a.subset_kind}) ctx={a.ctx} page={s.page_size}")
+            f"ffn={s.ffn} V={s.vocab} subset={N}({a.subset_kind}) "
+            + (f"ctx=uniform[{a.ctx_min},{a.ctx_max}]" if a.ctx_max > 0 else f"ctx={a.ctx}") + f" page={s.page_size}")
 
 
 def cpu_oracle_sample(s, W, kv, h, tok, ids, vcase, K, seconds=12.0, max_calls=6):
@@ -228,7 +234,7 @@ def run_ours(a):
 
     s, N, K, W, kv, h, tok, ids, vcase, ctx_lens = make_inputs(a, rank)
     B = a.batch
-    ctx = Bd.Context(s, max_rows=max(8, B), max_K=max(8, K), max_ctx=a.ctx + K + 1)
+    ctx = Bd.Context(s, max_rows=max(8, B), max_K=max(8, K), max_ctx=max(ctx_lens) + K + 1)
     dW = Bd.to_device(W)
     w = Bd.mtp_w(dW)
     dkv = Bd.to_device(kv)
@@ -353,7 +359,7 @@ def run_ours(a):
 
 
 def run_sweep(a):
-    """Subset size {8192 .. full} (Zipf-weighted draws) x batch {1, 4} x K {1, 3, 5} on the 7B-class head at
+    """Subset size {8192 .. full} (Zipf-weighted draws) x batch {1, 4, 16, 32} x K {1, 3, 5} on the 7B-class head at
     context 2048: device-timed draft calls only, one JSON line per point."""
     import torch
     import __graft_entry__ as G
@@ -367,14 +373,14 @@ def run_sweep(a):
     w = Bd.mtp_w(dW)
     peak, peak_kind = load_peaks()
     sizes = [8192, 16384, 32768, 65536, s.vocab] if a.shape == "7b" else [256, 1024, s.vocab]
-    for B in (1, 4):
+    for B in (1, 4, 16, 32):
         ctx_lens = [a.ctx] * B
         kv = I.paged_kv(s, ctx_lens, 6, a.seed + 1)
         dkv = Bd.to_device(kv)
         ckv = Bd.kv(dkv)
         dh = Bd.bf16_tensor(I.hidden_bf16(a.seed + 2, (B, s.d)))
         dtok = torch.from_numpy(I.token_ids(a.seed + 3, (B,), s.vocab)).cuda()
-        ctx = Bd.Context(s, max_rows=8, max_K=8, max_ctx=a.ctx + 8)
+        ctx = Bd.Context(s, max_rows=max(8, B), max_K=8, max_ctx=a.ctx + 8)
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
         for N in sizes:
             ids = None if N >= s.vocab else torch.from_numpy(I.subset_zipf(s.vocab, N, a.seed + 4)).cuda()
@@ -384,7 +390,7 @@ def run_sweep(a):
                     ctx.fastmtp_draft(w, dh, dtok, ckv, B, K, ids, out_d, None, None, status)
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 torch.cuda.synchronize()
-                n = 50
+                n = 50 if B <= 4 else 10
                 e0.record()
                 for _ in range(n):
                     ctx.fastmtp_draft(w, dh, dtok, ckv, B, K, ids, out_d, None, None, status)
