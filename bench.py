@@ -285,12 +285,10 @@ def run_ours(a):
             dist.barrier()
             torch.cuda.synchronize()
 
+    from paper_2509_18362_b200 import replicas
+
     def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(ms, dist, device="cuda")
 
     sampler = ClockSampler(local)
     for _ in range(max(a.warmup, 3)):
@@ -341,8 +339,8 @@ def run_ours(a):
         return
 
     ms_per_step = ms_total / a.steps
-    value = world * B * K * a.steps / (ms_total * 1e-3)
-    e2e_value = world * B * K * n_e2e / (ms_e2e * 1e-3)
+    value = replicas.job_throughput(B * K, world, a.steps, ms_total)
+    e2e_value = replicas.job_throughput(B * K, world, n_e2e, ms_e2e)
     bytes_launch = sum(algorithmic_bytes_per_draft_step(s, B, N, ctx_lens, k) for k in range(K))
     peak, peak_kind = load_peaks()
     achieved = bytes_launch / (draft_ms * 1e-3) / 1e9

@@ -128,6 +128,14 @@ int fmtp_last_cuda_error(const fmtp_ctx *ctx);
 /* Number of kernel launches this context has enqueued so far. */
 long long fmtp_launch_count(const fmtp_ctx *ctx);
 
+/* Diagnostic (no counterpart in the paper): runs a one-warp kernel that waits, with the library's
+ * bounded wait loop and a limit of `limit_ms` milliseconds (1..1000), for an event that never comes.
+ * On expiry the kernel ORs FMTP_DEV_TIMEOUT into *dev_status (dev, 1 word), optionally stores the
+ * nanoseconds it waited in *dev_waited_ns (dev, may be NULL) and returns normally: nothing hangs,
+ * traps or faults, and later calls on the same device work as before. The decoder kernel's own waits
+ * (ring stages, grid barriers) use the same loop with a 2 s limit. */
+int fmtp_selftest_wait_timeout(uint32_t *dev_status, int limit_ms, unsigned long long *dev_waited_ns, void *stream);
+
 /* ---- draft: Sec. 2.3 "Drafting phase", Sec. 2.1 steps k=1 / k>1, Sec. 2.2 Eq. 3 -------- */
 
 /* Recursive K-step draft for B sequences.

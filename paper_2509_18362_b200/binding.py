@@ -24,7 +24,7 @@ FMTP_OK = 0
 DEV_BAD_TOKEN, DEV_BAD_PAGE, DEV_BAD_POS, DEV_TIMEOUT, DEV_ALL_NAN = 1, 2, 4, 8, 16
 
 EXPORTS = ["fmtp_create", "fmtp_destroy", "fmtp_workspace_bytes", "fmtp_set_workspace", "fmtp_strerror",
-           "fmtp_last_cuda_error", "fmtp_launch_count", "fastmtp_draft", "fastmtp_draft_host",
+           "fmtp_last_cuda_error", "fmtp_launch_count", "fmtp_selftest_wait_timeout", "fastmtp_draft", "fastmtp_draft_host",
            "fastmtp_verify_accept", "fastmtp_verify_accept_host", "fastmtp_verify_accept_static",
            "fastmtp_target_step"]
 
@@ -70,6 +70,8 @@ lib.fmtp_last_cuda_error.argtypes = [_p]
 lib.fmtp_last_cuda_error.restype = C.c_int
 lib.fmtp_launch_count.argtypes = [_p]
 lib.fmtp_launch_count.restype = C.c_longlong
+lib.fmtp_selftest_wait_timeout.argtypes = [_p, C.c_int, _p, _p]
+lib.fmtp_selftest_wait_timeout.restype = C.c_int
 lib.fastmtp_draft.argtypes = [_p, C.POINTER(fmtp_mtp_w), _p, _p, C.POINTER(fmtp_kv), C.c_int, C.c_int, _p, C.c_int,
                               _p, _p, _p, _p, _p]
 lib.fastmtp_draft.restype = C.c_int
@@ -127,6 +129,13 @@ def target_w(t: dict):
 def kv(t: dict) -> fmtp_kv:
     return fmtp_kv(t["k_pages"].data_ptr(), t["v_pages"].data_ptr(), t["block_table"].data_ptr(),
                    t["seq_lens"].data_ptr(), int(t["k_pages"].shape[0]), int(t["block_table"].shape[1]))
+
+
+def fmtp_selftest_wait_timeout(dev_status, limit_ms, dev_waited_ns=None, stream=None):
+    """Launches the bounded-wait probe (a wait that must run out); see include/fastmtp.h."""
+    rc = lib.fmtp_selftest_wait_timeout(_ptr(dev_status), int(limit_ms), _ptr(dev_waited_ns), _stream(stream))
+    if rc != FMTP_OK:
+        raise FastMTPError(rc, "fmtp_selftest_wait_timeout")
 
 
 STATIC_VERIFY_MAX_ROWS = 1024

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfastmtp.so")
-SOURCES = ["api.cu", "megakernel.cu", "verify.cu", "noalloc.cu"]
+SOURCES = ["api.cu", "megakernel.cu", "verify.cu", "noalloc.cu", "selftest.cu"]
 HEADERS = ["mega.cuh", "ptx.cuh", os.path.join("..", "..", "include", "fastmtp.h")]
 
 

@@ -89,3 +89,21 @@ def test_host_entry_point():
     ra, rb, _ = O.verify_accept(case["logits"], case["drafts"])
     assert np.array_equal(a, ra) and np.array_equal(bonus, rb)
     ctx.close()
+
+
+def test_a_wait_that_runs_out_sets_the_timeout_flag_and_leaves_the_device_usable():
+    """Failure detection without a fault: the library's bounded wait, given an event that never comes and a
+    20 ms limit, reports FMTP_DEV_TIMEOUT through the status word and returns; the next call works."""
+    Bd, ctx = _ctx()
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    Bd.fmtp_selftest_wait_timeout(st, 20, waited)
+    torch.cuda.synchronize()
+    assert int(st.item()) & Bd.DEV_TIMEOUT
+    assert 20e6 <= int(waited.item()) < 500e6            # gave up soon after the limit
+    with pytest.raises(Bd.FastMTPError):
+        Bd.fmtp_selftest_wait_timeout(st, 5000)          # limits above one second are refused on the host
+    case = I.verify_case(3, 2, 999, 5)
+    a, bonus, _ = _run(Bd, ctx, case["logits"], case["drafts"])
+    assert np.array_equal(a, case["length"])
+    ctx.close()
