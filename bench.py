@@ -46,6 +46,9 @@ def parse_args():
     ap.add_argument("--shape", default="7b", choices=["7b", "tiny"])
     ap.add_argument("--seed", type=int, default=1234)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--target-layers", type=int, default=0,
+                    help="instead of the draft path, time fastmtp_target_step on a random target of this many layers "
+                         "(1 row and draft-steps+1 rows per sequence); one JSON line per row count")
     ap.add_argument("--sweep", action="store_true",
                     help="vocabulary-compression sweep on one GPU: subset size x batch x draft steps, one JSON line each")
     return ap.parse_args()
@@ -423,8 +426,58 @@ def run_sweep(a):
         ctx.close()
 
 
+def run_target(a):
+    """Device-timed fastmtp_target_step on a random target model of --target-layers layers at the
+    chosen width: M = 1 (plain decode) and M = draft-steps + 1 (verification rows), batch --batch,
+    --ctx cached tokens per layer. The bytes counted are every layer weight and the full output
+    head once, the cached K/V of every layer, and the logits written."""
+    import torch
+    import __graft_entry__ as G
+    G.build()
+    from paper_2509_18362_b200 import binding as Bd
+    from paper_2509_18362_b200 import inputs as I
+    torch.cuda.set_device(0)
+    nl, B = a.target_layers, a.batch
+    s = (I.QWEN7B if a.shape == "7b" else I.TINY).with_layers(nl)
+    Wt = I.target_weights(s, a.seed)
+    dW = Bd.to_device(Wt)
+    w, keep = Bd.target_w(dW)
+    peak, peak_kind = load_peaks()
+    qd, kvd = s.n_q_heads * s.head_dim, s.n_kv_heads * s.head_dim
+    layer_w = s.d * (qd + 2 * kvd) + qd * s.d + 3 * s.d * s.ffn
+    for M in (1, a.draft_steps + 1):
+        kvs = [I.paged_kv(s, [a.ctx] * B, M + 1, a.seed + 10 + l, tag="tkv%d" % l) for l in range(nl)]
+        dkvs = [Bd.to_device(kv) for kv in kvs]
+        ckvs = [Bd.kv(k) for k in dkvs]
+        ctx = Bd.Context(s, max_rows=max(8, B * M), max_K=8, max_ctx=a.ctx + M + 1)
+        tok = torch.from_numpy(I.token_ids(a.seed + 3, (B, M), s.vocab)).cuda()
+        out_l = torch.zeros((B, M, s.vocab), dtype=torch.bfloat16, device="cuda")
+        out_a = torch.zeros((B, M), dtype=torch.int32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for _ in range(5):
+            ctx.fastmtp_target_step(w, tok, ckvs, B, M, None, out_l, out_a, status)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        n, l0 = 30, ctx.launch_count
+        e0.record()
+        for _ in range(n):
+            ctx.fastmtp_target_step(w, tok, ckvs, B, M, None, out_l, out_a, status)
+        e1.record()
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0, f"device status {int(status.item()):#x}"
+        ms = e0.elapsed_time(e1) / n
+        nbytes = 2 * (nl * layer_w + s.vocab * s.d) + nl * B * 2 * 2 * kvd * (a.ctx + M) + 2 * B * M * (s.vocab + s.d)
+        print(json.dumps({"target_step": True, "layers": nl, "batch": B, "rows_per_seq": M, "ctx": a.ctx, "ms": ms,
+                          "launches_per_call": (ctx.launch_count - l0) // n,
+                          "us_per_layer_incl_head": ms * 1e3 / nl, "mb": nbytes / 1e6, "gbs": nbytes / (ms * 1e-3) / 1e9,
+                          "frac_of_" + peak_kind: nbytes / (ms * 1e-3) / 1e9 / peak}), flush=True)
+        ctx.close()
+
+
 def main():
     a = parse_args()
+    if a.target_layers > 0:
+        return run_target(a)
     if a.sweep:
         return run_sweep(a)
     if a.impl == "reference":
