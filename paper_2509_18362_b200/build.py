@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfastmtp.so")
-SOURCES = ["api.cu", "megakernel.cu", "verify.cu", "noalloc.cu", "selftest.cu"]
-HEADERS = ["mega.cuh", "ptx.cuh", os.path.join("..", "..", "include", "fastmtp.h")]
+SOURCES = ["api.cu", "megakernel.cu", "batched.cu", "verify.cu", "noalloc.cu", "selftest.cu"]
+HEADERS = ["mega.cuh", "ptx.cuh", "umma.cuh", "skinny_gemm.cuh", "batched.cuh", os.path.join("..", "..", "include", "fastmtp.h")]
 
 
 def _sources():

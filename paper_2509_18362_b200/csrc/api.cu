@@ -3,6 +3,7 @@
 // kernels of megakernel.cu and verify.cu.
 #include "../../include/fastmtp.h"
 #include "mega.cuh"
+#include "batched.cuh"
 
 #include <cmath>
 #include <cstdlib>
@@ -38,6 +39,10 @@ struct fmtp_ctx {
     size_t vstage_bytes;
     int last_cuda;
     long long launches;
+    // batched draft path (more sequences than one persistent-kernel launch takes)
+    BatchedShape bsh;
+    BatchedWs bws;
+    int batched_min;           // calls with at least this many sequences take the batched path (env FMTP_BATCHED_MIN)
 };
 
 namespace {
@@ -103,7 +108,9 @@ size_t layout(fmtp_ctx *c, unsigned char *base) {
     c->st_tok = cv.take<int32_t>((size_t)RB);
     c->st_out = cv.take<int32_t>((size_t)RB * (sh.max_K > 1 ? sh.max_K : 1) + 2 * kVerifyMaxRows);
     c->st_status = cv.take<uint32_t>(1);
-    return align_up(cv.off, 256);
+    size_t off = align_up(cv.off, 256);
+    off += batched_layout(c->bws, base ? base + off : nullptr, c->bsh);
+    return align_up(off, 256);
 }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -275,8 +282,14 @@ int fmtp_create(const fmtp_shape *sh, fmtp_ctx **out) {
     if (const char *v = std::getenv("FMTP_STAGE_F")) c->stage_F_pref = std::atoi(v);
     c->stages_cap = kMaxStages;
     if (const char *v = std::getenv("FMTP_STAGES")) { int n = std::atoi(v); if (n >= 2 && n <= kMaxStages) c->stages_cap = n; }
+    c->bsh.d = sh->d; c->bsh.Hq = sh->n_q_heads; c->bsh.Hkv = sh->n_kv_heads; c->bsh.dh = sh->head_dim; c->bsh.F = sh->ffn;
+    c->bsh.V = sh->vocab; c->bsh.page = sh->page_size; c->bsh.max_ctx = sh->max_ctx; c->bsh.max_K = sh->max_K;
+    c->bsh.max_rows = sh->max_rows; c->bsh.eps = sh->rms_eps;
     c->ws_need = layout(c, nullptr);
-    if (group_size(c, 0, kMaxRows, 1) < 1) { delete c; return FMTP_ESHAPE; }
+    const int g1 = group_size(c, 0, kMaxRows, 1);
+    if (g1 < 1) { delete c; return FMTP_ESHAPE; }
+    c->batched_min = g1 + 1;
+    if (const char *v = std::getenv("FMTP_BATCHED_MIN")) { int n = std::atoi(v); if (n >= 1) c->batched_min = n; }
     c->pinned_bytes = (size_t)sh->max_rows * sh->d * 2 + (size_t)sh->max_rows * 4 * (2 + (sh->max_K > 1 ? sh->max_K : 1)) +
                       2 * kVerifyMaxRows * 4 + 256;
     e = cudaMallocHost(&c->pinned, c->pinned_bytes);
@@ -337,9 +350,37 @@ int fastmtp_draft(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_last, con
     if (!aligned16(w->embed) || !aligned16(w->lm_head) || !aligned16(w->g_hnorm) || !aligned16(w->g_enorm) ||
         !aligned16(w->w_proj) || !aligned16(w->g_final) || !aligned16(h_last) || !layer_ok(w->layer) || !kv_ok(*kv))
         return FMTP_EINVAL;
+    const int Neff = subset ? N : c->shape.vocab;
+    if (B >= c->batched_min) {
+        // more sequences than one launch of the persistent kernel takes: groups of up to 64 sequences, every
+        // weight streamed once per step and group by the tensor-core GEMM path
+        for (int b0 = 0; b0 < B; b0 += kBatchRows) {
+            BatchedCall bc;
+            std::memset(&bc, 0, sizeof(bc));
+            bc.sh = c->bsh; bc.ws = c->bws;
+            bc.rope_cos = c->s.rope_cos; bc.rope_sin = c->s.rope_sin;
+            bc.n_sm = c->n_sm; bc.smem_optin = c->smem_optin;
+            bc.B = (B - b0 < kBatchRows) ? B - b0 : kBatchRows;
+            bc.K = K; bc.N = Neff; bc.ids = subset;
+            bc.h_last = h_last + (size_t)b0 * c->shape.d;
+            bc.tok_last = tok_last + b0;
+            bc.out_drafts = out_drafts + (size_t)b0 * K;
+            bc.out_h = out_h ? out_h + (size_t)b0 * K * c->shape.d : nullptr;
+            bc.out_logits = out_logits ? out_logits + (size_t)b0 * K * Neff : nullptr;
+            bc.user_status = dev_status;
+            bc.embed = w->embed; bc.lm_head = w->lm_head; bc.g_hnorm = w->g_hnorm; bc.g_enorm = w->g_enorm;
+            bc.w_proj = w->w_proj; bc.g_final = w->g_final;
+            set_layer(bc.layer, w->layer);
+            set_kv(bc.kv, *kv);
+            bc.kv.block_table += (size_t)b0 * kv->max_pages_per_seq;
+            bc.kv.seq_lens += b0;
+            int err = batched_draft(bc, static_cast<cudaStream_t>(stream), &c->launches);
+            if (err) return cuda_fail(c, (cudaError_t)err);
+        }
+        return FMTP_OK;
+    }
     const int G = group_size(c, 0, B, 1);
     if (G < 1) return FMTP_ESHAPE;
-    const int Neff = subset ? N : c->shape.vocab;
     for (int b0 = 0; b0 < B; b0 += G) {
         const int Bg = (B - b0 < G) ? B - b0 : G;
         MegaParams p;

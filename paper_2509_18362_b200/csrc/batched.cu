@@ -1,0 +1,536 @@
+// Batched draft path (Sec. 2.1 recursion, Sec. 2.2 Eq. 3 compressed head) for groups of up to 64
+// sequences: per step, six weight-streaming tcgen05 GEMMs (skinny_gemm.cuh) and the small
+// row-wise kernels between them (norms, rotary embedding + cache append, attention, residuals).
+// All kernels of a call are enqueued on the caller's stream; none waits on another CTA.
+#include "batched.cuh"
+#include "skinny_gemm.cuh"
+
+namespace fmtp {
+
+namespace {
+
+constexpr uint32_t kDevBadToken = 0x1u, kDevBadPage = 0x2u, kDevBadPos = 0x4u, kDevAllNan = 0x10u;
+constexpr int kRowThreads = 256;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+__device__ __forceinline__ float block_sum(float v, float *red) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    for (int w = 0; w < nw; ++w) t += red[w];     // same order on every thread
+    return t;
+}
+
+__device__ __forceinline__ void store_hilo(bf16_t *xop, int ld, int r, int j, float v) {
+    uint16_t hi, lo;
+    split_bf16(v, hi, lo);
+    xop[(size_t)(2 * r) * ld + j] = hi;
+    xop[(size_t)(2 * r + 1) * ld + j] = lo;
+}
+
+// ---- step input: [rms(h; g_h) ; rms(Emb(tok); g_e)] as the projection's operand; also turns the
+// previous step's argmax key into its draft token. One block per sequence.
+struct PrologueArgs {
+    int step, K, d, V, ld, only_tokens;
+    float eps;
+    const bf16_t *h_last;
+    const int32_t *tok_last;
+    const float *hout;
+    const unsigned long long *keys_prev;
+    int32_t *out_drafts;
+    const bf16_t *embed, *g_h, *g_e;
+    bf16_t *xop;
+    uint32_t *status, *user_status;
+};
+
+__global__ void __launch_bounds__(kRowThreads) prologue_kernel(const PrologueArgs a) {
+    __shared__ float red[32];
+    __shared__ int s_tok;
+    const int r = blockIdx.x, tid = threadIdx.x;
+    if (tid == 0) {
+        int tok;
+        if (a.step == 0) tok = a.tok_last[r];
+        else {
+            const unsigned long long key = a.keys_prev[r];
+            if ((key >> 32) == 0ull) atomicOr(a.status, kDevAllNan);
+            tok = (int)argmax_key_id(key);
+            a.out_drafts[(size_t)r * a.K + (a.step - 1)] = tok;
+        }
+        if ((unsigned)tok >= (unsigned)a.V) { atomicOr(a.status, kDevBadToken); tok = 0; }
+        s_tok = tok;
+    }
+    __syncthreads();
+    if (a.only_tokens) {
+        // last kernel of the call: hand the status word (earlier kernels' flags and this block's) to the caller
+        if (tid == 0 && a.user_status) {
+            __threadfence();
+            const uint32_t st = *reinterpret_cast<volatile uint32_t *>(a.status);
+            if (st) atomicOr(a.user_status, st);
+        }
+        return;
+    }
+    const bf16_t *erow = a.embed + (size_t)s_tok * a.d;
+    float sh = 0.f, se = 0.f;
+    for (int j = tid; j < a.d; j += kRowThreads) {
+        const float h = a.step == 0 ? bf16bits_f32(a.h_last[(size_t)r * a.d + j]) : a.hout[(size_t)r * a.d + j];
+        const float e = bf16bits_f32(erow[j]);
+        sh += h * h;
+        se += e * e;
+    }
+    sh = block_sum(sh, red);
+    se = block_sum(se, red);
+    const float rh = 1.0f / sqrtf(sh / (float)a.d + a.eps), re = 1.0f / sqrtf(se / (float)a.d + a.eps);
+    for (int j = tid; j < a.d; j += kRowThreads) {
+        const float h = a.step == 0 ? bf16bits_f32(a.h_last[(size_t)r * a.d + j]) : a.hout[(size_t)r * a.d + j];
+        const float e = bf16bits_f32(erow[j]);
+        store_hilo(a.xop, a.ld, r, j, h * rh * bf16bits_f32(a.g_h[j]));
+        store_hilo(a.xop, a.ld, r, a.d + j, e * re * bf16bits_f32(a.g_e[j]));
+    }
+}
+
+// ---- after a split-K GEMM: x = (residual ? x : 0) + sum of the partials; operand of the next
+// GEMM = rms(x; gain) as hi/lo. With `final`: the normed vector is the step's output hidden state.
+struct PostArgs {
+    int d, splits, rows, ldp, ld, residual, final, K, step;
+    float eps;
+    const float *partial;
+    float *x, *hout;
+    bf16_t *out_h;
+    const bf16_t *gain;
+    bf16_t *xop;
+};
+
+__global__ void __launch_bounds__(kRowThreads) post_kernel(const PostArgs a) {
+    __shared__ float red[32];
+    const int r = blockIdx.x, tid = threadIdx.x;
+    float ss = 0.f;
+    for (int j = tid; j < a.d; j += kRowThreads) {
+        float v = a.residual ? a.x[(size_t)r * a.d + j] : 0.f;
+        for (int s = 0; s < a.splits; ++s) v += a.partial[((size_t)s * a.rows + r) * a.ldp + j];
+        a.x[(size_t)r * a.d + j] = v;
+        ss += v * v;
+    }
+    ss = block_sum(ss, red);
+    const float rs = 1.0f / sqrtf(ss / (float)a.d + a.eps);
+    for (int j = tid; j < a.d; j += kRowThreads) {
+        const float n = a.x[(size_t)r * a.d + j] * rs * bf16bits_f32(a.gain[j]);
+        store_hilo(a.xop, a.ld, r, j, n);
+        if (a.final) {
+            a.hout[(size_t)r * a.d + j] = n;
+            if (a.out_h) a.out_h[((size_t)r * a.K + a.step) * a.d + j] = f32_bf16bits(n);
+        }
+    }
+}
+
+// ---- after the QKV GEMM: sum the partials, rotate q and k at the row's position, keep q in fp32,
+// append k and v (rounded to bf16) to the paged cache. Block = (head, sequence), dh/2 threads.
+struct QkvArgs {
+    int qdim, kvdim, dh, Hq, Hkv, splits, rows, ldp, page, max_ctx, step;
+    const float *partial;
+    float *q;
+    KvPtrs kv;
+    const float *rope_cos, *rope_sin;
+    uint32_t *status;
+};
+
+__global__ void qkv_finish_kernel(const QkvArgs a) {
+    const int head = blockIdx.x, r = blockIdx.y, e = threadIdx.x, half = a.dh >> 1;
+    const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
+    const int pos_true = a.kv.seq_lens[r] + a.step;
+    const int pos = min(pos_true, max_tokens - 1);
+    const int col = head * a.dh;              // q heads, then k heads, then v heads: the GEMM's row order
+    float lo = 0.f, hi = 0.f;
+    for (int s = 0; s < a.splits; ++s) {
+        const float *pp = a.partial + ((size_t)s * a.rows + r) * a.ldp + col;
+        lo += pp[e];
+        hi += pp[e + half];
+    }
+    if (head < a.Hq + a.Hkv) {
+        const float cs = a.rope_cos[(size_t)pos * half + e], sn = a.rope_sin[(size_t)pos * half + e];
+        const float x = lo, y = hi;
+        lo = x * cs - y * sn;
+        hi = y * cs + x * sn;
+    }
+    if (head < a.Hq) {
+        a.q[(size_t)r * a.qdim + col + e] = lo;
+        a.q[(size_t)r * a.qdim + col + e + half] = hi;
+        return;
+    }
+    if (pos_true >= max_tokens) {             // no slot for this position: flagged, nothing written
+        if (head == a.Hq && e == 0) atomicOr(a.status, kDevBadPos);
+        return;
+    }
+    const bool is_k = head < a.Hq + a.Hkv;
+    const int kvh = is_k ? head - a.Hq : head - a.Hq - a.Hkv;
+    int page = a.kv.block_table[(size_t)r * a.kv.max_pages + pos / a.page];
+    if ((unsigned)page >= (unsigned)a.kv.num_pages) { atomicOr(a.status, kDevBadPage); page = 0; }
+    bf16_t *dst = (is_k ? a.kv.k_pages : a.kv.v_pages) + (((size_t)page * a.Hkv + kvh) * a.page + (pos % a.page)) * a.dh;
+    dst[e] = f32_bf16bits(lo);
+    dst[e + half] = f32_bf16bits(hi);
+}
+
+// ---- attention over one 256-token chunk of one (sequence, KV head): the Hq/Hkv query heads of
+// the group share the K/V stream. Scores and the weighted sum run on mma.sync.m16n8k16 with the
+// query (and the probabilities) as the A operand, rows 0-7 the high bf16 parts of the heads and
+// rows 8-15 the low parts, so both products carry fp32-accurate inputs. Each warp owns 16 tokens of
+// every 64-token block and keeps its own running (max, sum, output); the four warps merge in
+// fixed order at the end. Output: unnormalised o, running max m and sum l per head and chunk.
+struct AttnArgs {
+    int Hq, Hkv, dh, page, max_ctx, step, max_chunks;
+    const float *q;              // [rows][Hq*dh]
+    KvPtrs kv;
+    float *att_part;             // [rows][Hq][max_chunks][dh+2]
+    uint32_t *status;
+};
+
+constexpr int kAttnBlk = 64;                 // tokens per pipeline stage
+constexpr int kAttnStages = 3;
+constexpr int kAttnThreads = 128;
+
+template <int DH>
+__global__ void __launch_bounds__(kAttnThreads) attn_chunk_kernel(const AttnArgs a) {
+    constexpr int ROWB = DH * 2 + 16;                       // padded row: conflict-free fragment loads
+    constexpr int STAGE = 2 * kAttnBlk * ROWB;              // K block then V block
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int chunk = blockIdx.x, kvh = blockIdx.y, r = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
+    const int n_ctx = min(a.kv.seq_lens[r] + a.step, max_tokens - 1) + 1;     // visible positions 0 .. n_ctx-1
+    const int t0 = chunk * kBatchAttnChunk;
+    if (t0 >= n_ctx) return;
+    const int n_tok = min(kBatchAttnChunk, n_ctx - t0);
+    const int n_blk = (n_tok + kAttnBlk - 1) / kAttnBlk;
+    const int gq = a.Hq / a.Hkv;
+    const int32_t *bt = a.kv.block_table + (size_t)r * a.kv.max_pages;
+
+    // ---- K/V copies: thread copies 16-byte pieces; a 64-token block of K or V is 64 x DH*2 bytes
+    auto issue = [&](int blk) {
+        unsigned char *st = smem + (size_t)(blk % kAttnStages) * STAGE;
+        constexpr int PIECES = DH / 8;                      // 16-byte pieces per row
+        for (int i = tid; i < kAttnBlk * PIECES; i += kAttnThreads) {
+            const int t = i / PIECES, pc = i - t * PIECES;
+            int pos = t0 + blk * kAttnBlk + t;
+            const uint32_t ok = pos < n_ctx ? 16u : 0u;
+            if (pos >= n_ctx) pos = n_ctx - 1;
+            int page = bt[pos / a.page];
+            if ((unsigned)page >= (unsigned)a.kv.num_pages) { atomicOr(a.status, kDevBadPage); page = 0; }
+            const size_t off = (((size_t)page * a.Hkv + kvh) * a.page + (pos % a.page)) * DH + pc * 8;
+            cp_async16_off<0>(smem_u32(st + t * ROWB + pc * 16), a.kv.k_pages + off, ok);
+            cp_async16_off<0>(smem_u32(st + kAttnBlk * ROWB + t * ROWB + pc * 16), a.kv.v_pages + off, ok);
+        }
+        cp_async_commit();
+    };
+    issue(0);
+    if (n_blk > 1) issue(1); else cp_async_commit();
+
+    // ---- query fragments: A rows 0-7 = hi parts of heads 0..gq-1, rows 8-15 = lo parts
+    const int hrow = lane >> 2, kq = (lane & 3) * 2;
+    const float scale = rsqrtf((float)DH);
+    uint32_t qa[DH / 16][4];
+    {
+        const float *qh = a.q + ((size_t)r * a.Hq + (size_t)kvh * gq + hrow) * DH;
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks) {
+            float v0 = 0.f, v1 = 0.f, v2 = 0.f, v3 = 0.f;
+            if (hrow < gq) {
+                v0 = qh[ks * 16 + kq] * scale; v1 = qh[ks * 16 + kq + 1] * scale;
+                v2 = qh[ks * 16 + kq + 8] * scale; v3 = qh[ks * 16 + kq + 9] * scale;
+            }
+            uint16_t h0, l0, h1, l1, h2, l2, h3, l3;
+            split_bf16(v0, h0, l0); split_bf16(v1, h1, l1); split_bf16(v2, h2, l2); split_bf16(v3, h3, l3);
+            qa[ks][0] = (uint32_t)h0 | ((uint32_t)h1 << 16);      // row hrow,     k = kq, kq+1
+            qa[ks][1] = (uint32_t)l0 | ((uint32_t)l1 << 16);      // row hrow + 8
+            qa[ks][2] = (uint32_t)h2 | ((uint32_t)h3 << 16);      // row hrow,     k = kq+8, kq+9
+            qa[ks][3] = (uint32_t)l2 | ((uint32_t)l3 << 16);
+        }
+    }
+    float m_run = -INFINITY, l_run = 0.f;       // of head hrow, this warp's tokens (replicated on the 4 lanes of a row)
+    float o[DH / 8][2];                          // o[nt][j]: head hrow, dim nt*8 + kq + j
+#pragma unroll
+    for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = 0.f;
+
+    for (int blk = 0; blk < n_blk; ++blk) {
+        if (blk + 2 < n_blk) issue(blk + 2); else cp_async_commit();
+        cp_async_wait_group<2>();
+        __syncthreads();
+        const unsigned char *sk = smem + (size_t)(blk % kAttnStages) * STAGE;
+        const unsigned char *sv = sk + kAttnBlk * ROWB;
+        const int tw = warp * 16;                              // this warp's tokens inside the block
+        const int tbase = t0 + blk * kAttnBlk + tw;
+        if (tbase < n_ctx) {
+            // scores: two n-tiles of 8 tokens
+            float s[2][4];
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+                s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+                const unsigned char *krow = sk + (size_t)(tw + nt * 8 + hrow) * ROWB;     // B column n = token lane/4
+#pragma unroll
+                for (int ks = 0; ks < DH / 16; ++ks) {
+                    const uint32_t b0 = *reinterpret_cast<const uint32_t *>(krow + (ks * 16 + kq) * 2);
+                    const uint32_t b1 = *reinterpret_cast<const uint32_t *>(krow + (ks * 16 + kq + 8) * 2);
+                    mma_bf16(s[nt], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+                }
+            }
+            // thread holds, for head hrow: tokens tw + nt*8 + kq + {0,1}: hi part in [0],[1], lo part in [2],[3]
+            float sc[4];
+            float mx = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    float v = s[nt][j] + s[nt][j + 2];
+                    if (tbase + nt * 8 + kq + j >= n_ctx) v = -INFINITY;
+                    sc[nt * 2 + j] = v;
+                    mx = fmaxf(mx, v);
+                }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m_run, mx);                 // finite: the warp's first token is visible
+            const float corr = expf(m_run - m_new);               // 0 on the first block (m_run = -inf)
+            float psum = 0.f;
+            uint32_t pa[4];
+            {
+                float pr[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { pr[i] = expf(sc[i] - m_new); psum += pr[i]; }
+                uint16_t h0, l0, h1, l1, h2, l2, h3, l3;
+                split_bf16(pr[0], h0, l0); split_bf16(pr[1], h1, l1); split_bf16(pr[2], h2, l2); split_bf16(pr[3], h3, l3);
+                pa[0] = (uint32_t)h0 | ((uint32_t)h1 << 16);      // row hrow,   tokens kq, kq+1
+                pa[1] = (uint32_t)l0 | ((uint32_t)l1 << 16);      // row hrow+8
+                pa[2] = (uint32_t)h2 | ((uint32_t)h3 << 16);      // row hrow,   tokens 8+kq, 8+kq+1
+                pa[3] = (uint32_t)l2 | ((uint32_t)l3 << 16);
+            }
+            psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+            psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+            l_run = l_run * corr + psum;
+            m_run = m_new;
+            // weighted sum: B[k = token][n = dim] read with a transposing ldmatrix from V[token][dim]
+#pragma unroll
+            for (int nt = 0; nt < DH / 8; ++nt) {
+                uint32_t b0, b1;
+                const unsigned char *vrow = sv + (size_t)(tw + (lane & 15)) * ROWB + nt * 16;
+                asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];"
+                             : "=r"(b0), "=r"(b1) : "r"(smem_u32(vrow)));
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                mma_bf16(acc, pa[0], pa[1], pa[2], pa[3], b0, b1);
+                o[nt][0] = o[nt][0] * corr + acc[0] + acc[2];
+                o[nt][1] = o[nt][1] * corr + acc[1] + acc[3];
+            }
+        }
+        __syncthreads();
+    }
+    cp_async_wait_group<0>();
+    // ---- merge the four warps (fixed order) and write the chunk's partial
+    float *mo = reinterpret_cast<float *>(smem);                 // [4][8][DH + 2]
+    __syncthreads();
+    {
+        float *dst = mo + ((size_t)warp * 8 + hrow) * (DH + 2);
+#pragma unroll
+        for (int nt = 0; nt < DH / 8; ++nt) { dst[nt * 8 + kq] = o[nt][0]; dst[nt * 8 + kq + 1] = o[nt][1]; }
+        if ((lane & 3) == 0) { dst[DH] = m_run; dst[DH + 1] = l_run; }
+    }
+    __syncthreads();
+    for (int i = tid; i < gq * DH; i += kAttnThreads) {
+        const int h = i / DH, j = i - h * DH;
+        float m = -INFINITY;
+        for (int w = 0; w < 4; ++w) m = fmaxf(m, mo[((size_t)w * 8 + h) * (DH + 2) + DH]);
+        float acc = 0.f, l = 0.f;
+        for (int w = 0; w < 4; ++w) {
+            const float *src = mo + ((size_t)w * 8 + h) * (DH + 2);
+            const float f = src[DH] == -INFINITY ? 0.f : expf(src[DH] - m);
+            acc += src[j] * f;
+            l += src[DH + 1] * f;
+        }
+        float *out = a.att_part + (((size_t)r * a.Hq + (size_t)kvh * gq + h) * a.max_chunks + chunk) * (DH + 2);
+        out[j] = acc;
+        if (j == 0) { out[DH] = m; out[DH + 1] = l; }
+    }
+}
+
+// ---- combine a head's chunk partials in ascending order; write the O-projection's operand.
+struct MergeArgs {
+    int Hq, dh, page, max_ctx, step, max_chunks, ld;
+    KvPtrs kv;
+    const float *att_part;
+    bf16_t *xop;
+};
+
+__global__ void attn_merge_kernel(const MergeArgs a) {
+    const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x;
+    const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
+    const int n_ctx = min(a.kv.seq_lens[r] + a.step, max_tokens - 1) + 1;
+    const int n_chunks = (n_ctx + kBatchAttnChunk - 1) / kBatchAttnChunk;
+    const float *base = a.att_part + ((size_t)r * a.Hq + head) * a.max_chunks * (a.dh + 2);
+    float m = -INFINITY;
+    for (int c = 0; c < n_chunks; ++c) m = fmaxf(m, base[(size_t)c * (a.dh + 2) + a.dh]);
+    float acc = 0.f, l = 0.f;
+    for (int c = 0; c < n_chunks; ++c) {
+        const float *src = base + (size_t)c * (a.dh + 2);
+        const float f = expf(src[a.dh] - m);
+        acc += src[j] * f;
+        l += src[a.dh + 1] * f;
+    }
+    store_hilo(a.xop, a.ld, r, head * a.dh + j, acc / l);
+}
+
+int pick_splits(int n_tiles, int n_kb, int n_sm) {
+    int best = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= kBatchMaxSplits; ++s) {
+        if (s > 1 && n_kb / s < 8) break;
+        const int items = n_tiles * s;
+        const int waves = (items + n_sm - 1) / n_sm;
+        const double eff = (double)items / ((double)waves * n_sm);
+        if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
+    }
+    return best;
+}
+
+}  // namespace
+
+size_t batched_layout(BatchedWs &ws, unsigned char *base, const BatchedShape &sh) {
+    const int rows = sh.max_rows < kBatchRows ? sh.max_rows : kBatchRows;
+    const int qdim = sh.Hq * sh.dh, kvdim = sh.Hkv * sh.dh;
+    const int widest_in = 2 * sh.d > qdim ? 2 * sh.d : qdim;
+    const int widest_out = sh.d > qdim + 2 * kvdim ? sh.d : qdim + 2 * kvdim;
+    ws.rows = rows;
+    ws.ld0 = (int)align_up((size_t)widest_in, 64);
+    ws.ldF = (int)align_up((size_t)sh.F, 64);
+    ws.ldp = (int)align_up((size_t)widest_out, 128);
+    ws.max_chunks = (sh.max_ctx + kBatchAttnChunk - 1) / kBatchAttnChunk;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        off = align_up(off, 256);
+        unsigned char *p = base ? base + off : nullptr;
+        off += bytes;
+        return p;
+    };
+    ws.xop0 = reinterpret_cast<bf16_t *>(take((size_t)128 * ws.ld0 * 2));
+    ws.xopF = reinterpret_cast<bf16_t *>(take((size_t)128 * ws.ldF * 2));
+    ws.partial = reinterpret_cast<float *>(take((size_t)kBatchMaxSplits * rows * ws.ldp * 4));
+    ws.x = reinterpret_cast<float *>(take((size_t)rows * sh.d * 4));
+    ws.hout = reinterpret_cast<float *>(take((size_t)rows * sh.d * 4));
+    ws.q = reinterpret_cast<float *>(take((size_t)rows * qdim * 4));
+    ws.att_part = reinterpret_cast<float *>(take((size_t)rows * sh.Hq * ws.max_chunks * (sh.dh + 2) * 4));
+    ws.keys_bytes = (size_t)(sh.max_K > 1 ? sh.max_K : 1) * kBatchRows * 8 + 256;
+    ws.keys = reinterpret_cast<unsigned long long *>(take(ws.keys_bytes));
+    ws.status = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned char *>(ws.keys) + ws.keys_bytes - 256);
+    if (!base) ws.status = nullptr;
+    return align_up(off, 256);
+}
+
+int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
+    const BatchedShape &sh = c.sh;
+    const BatchedWs &ws = c.ws;
+    const int B = c.B, K = c.K, d = sh.d;
+    const int qdim = sh.Hq * sh.dh, kvdim = sh.Hkv * sh.dh;
+    const int NB = (2 * B + 15) / 16 * 16;
+    cudaError_t e = cudaMemsetAsync(ws.keys, 0, ws.keys_bytes, st);     // argmax keys and the status word
+    if (e != cudaSuccess) return (int)e;
+
+    auto gemm = [&](GemmArgs &g, int n_rows, int Kdim, int lda, const bf16_t *x, int ldx) -> int {
+        g.n_rows = n_rows; g.K = Kdim; g.lda = lda; g.x = x; g.ldx = ldx; g.NB = NB; g.R = B;
+        g.status = ws.status;
+        const int n_tiles = (n_rows + kGemmTileM - 1) / kGemmTileM, n_kb = (Kdim + kGemmBK - 1) / kGemmBK;
+        g.splits = g.epi == EPI_PARTIAL ? pick_splits(n_tiles, n_kb, c.n_sm) : 1;
+        g.kb_per_split = (n_kb + g.splits - 1) / g.splits;
+        g.splits = (n_kb + g.kb_per_split - 1) / g.kb_per_split;      // no empty range
+        g.partial = ws.partial; g.ldp = ws.ldp;
+        ++*launches;
+        return skinny_gemm_launch(g, c.n_sm, c.smem_optin, st);
+    };
+    auto post = [&](int splits, int residual, int final, const bf16_t *gain, int step) -> int {
+        PostArgs a{};
+        a.d = d; a.splits = splits; a.rows = B; a.ldp = ws.ldp; a.ld = ws.ld0; a.residual = residual; a.final = final;
+        a.K = K; a.step = step; a.eps = sh.eps; a.partial = ws.partial; a.x = ws.x; a.hout = ws.hout;
+        a.out_h = c.out_h; a.gain = gain; a.xop = ws.xop0;
+        post_kernel<<<B, kRowThreads, 0, st>>>(a);
+        ++*launches;
+        return (int)cudaGetLastError();
+    };
+    int rc = 0;
+    const size_t attn_smem = (size_t)kAttnStages * 2 * kAttnBlk * (sh.dh * 2 + 16);
+    if (sh.dh == 128) e = cudaFuncSetAttribute(attn_chunk_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
+    else e = cudaFuncSetAttribute(attn_chunk_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
+    if (e != cudaSuccess) return (int)e;
+
+    for (int step = 0; step <= K; ++step) {
+        PrologueArgs pa{};
+        pa.step = step; pa.K = K; pa.d = d; pa.V = sh.V; pa.ld = ws.ld0; pa.only_tokens = step == K ? 1 : 0;
+        pa.eps = sh.eps; pa.h_last = c.h_last; pa.tok_last = c.tok_last; pa.hout = ws.hout;
+        pa.keys_prev = step > 0 ? ws.keys + (size_t)(step - 1) * kBatchRows : nullptr;
+        pa.out_drafts = c.out_drafts; pa.embed = c.embed; pa.g_h = c.g_hnorm; pa.g_e = c.g_enorm;
+        pa.xop = ws.xop0; pa.status = ws.status; pa.user_status = c.user_status;
+        prologue_kernel<<<B, kRowThreads, 0, st>>>(pa);
+        ++*launches;
+        if ((rc = (int)cudaGetLastError())) return rc;
+        if (step == K) break;
+
+        GemmArgs g{};
+        // x = W_p [rms(h); rms(e)]
+        g.a[0] = c.w_proj; g.a_rows[0] = d; g.n_seg = 1; g.epi = EPI_PARTIAL;
+        if ((rc = gemm(g, d, 2 * d, 2 * d, ws.xop0, ws.ld0))) return rc;
+        if ((rc = post(g.splits, 0, 0, c.layer.g_in, step))) return rc;
+        // q, k, v
+        g = GemmArgs{};
+        g.a[0] = c.layer.wq; g.a[1] = c.layer.wk; g.a[2] = c.layer.wv;
+        g.a_rows[0] = qdim; g.a_rows[1] = kvdim; g.a_rows[2] = kvdim; g.n_seg = 3; g.epi = EPI_PARTIAL;
+        if ((rc = gemm(g, qdim + 2 * kvdim, d, d, ws.xop0, ws.ld0))) return rc;
+        {
+            QkvArgs a{};
+            a.qdim = qdim; a.kvdim = kvdim; a.dh = sh.dh; a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.splits = g.splits; a.rows = B;
+            a.ldp = ws.ldp; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = step; a.partial = ws.partial; a.q = ws.q;
+            a.kv = c.kv; a.rope_cos = c.rope_cos; a.rope_sin = c.rope_sin; a.status = ws.status;
+            qkv_finish_kernel<<<dim3(sh.Hq + 2 * sh.Hkv, B), sh.dh / 2, 0, st>>>(a);
+            ++*launches;
+            if ((rc = (int)cudaGetLastError())) return rc;
+        }
+        {
+            AttnArgs a{};
+            a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.dh = sh.dh; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = step;
+            a.max_chunks = ws.max_chunks; a.q = ws.q; a.kv = c.kv; a.att_part = ws.att_part; a.status = ws.status;
+            const dim3 grid(ws.max_chunks, sh.Hkv, B);
+            if (sh.dh == 128) attn_chunk_kernel<128><<<grid, kAttnThreads, attn_smem, st>>>(a);
+            else attn_chunk_kernel<64><<<grid, kAttnThreads, attn_smem, st>>>(a);
+            ++*launches;
+            if ((rc = (int)cudaGetLastError())) return rc;
+            MergeArgs m{};
+            m.Hq = sh.Hq; m.dh = sh.dh; m.page = sh.page; m.max_ctx = sh.max_ctx; m.step = step; m.max_chunks = ws.max_chunks;
+            m.ld = ws.ld0; m.kv = c.kv; m.att_part = ws.att_part; m.xop = ws.xop0;
+            attn_merge_kernel<<<dim3(sh.Hq, B), sh.dh, 0, st>>>(m);
+            ++*launches;
+            if ((rc = (int)cudaGetLastError())) return rc;
+        }
+        // x += W_o o
+        g = GemmArgs{};
+        g.a[0] = c.layer.wo; g.a_rows[0] = d; g.n_seg = 1; g.epi = EPI_PARTIAL;
+        if ((rc = gemm(g, d, qdim, qdim, ws.xop0, ws.ld0))) return rc;
+        if ((rc = post(g.splits, 1, 0, c.layer.g_post, step))) return rc;
+        // act = silu(W_gate n) * (W_up n), written as the down projection's operand
+        g = GemmArgs{};
+        g.a[0] = c.layer.w_gate; g.a_up = c.layer.w_up; g.a_rows[0] = sh.F; g.n_seg = 1; g.epi = EPI_SWIGLU;
+        g.xop_out = ws.xopF; g.ld_out = ws.ldF;
+        if ((rc = gemm(g, sh.F, d, d, ws.xop0, ws.ld0))) return rc;
+        // x += W_down act; h_out = rms(x; g_final)
+        g = GemmArgs{};
+        g.a[0] = c.layer.w_down; g.a_rows[0] = d; g.n_seg = 1; g.epi = EPI_PARTIAL;
+        if ((rc = gemm(g, d, sh.F, sh.F, ws.xopF, ws.ldF))) return rc;
+        if ((rc = post(g.splits, 1, 1, c.g_final, step))) return rc;
+        // compressed head + argmax (Eq. 3)
+        g = GemmArgs{};
+        g.a[0] = c.lm_head; g.a_rows[0] = c.N; g.n_seg = 1; g.epi = EPI_ARGMAX;
+        g.row_ids = c.ids; g.V = sh.V;
+        g.keys = ws.keys + (size_t)step * kBatchRows;
+        g.logits = c.out_logits ? c.out_logits + (size_t)step * c.N : nullptr;
+        g.logits_stride = (long long)K * c.N;
+        if ((rc = gemm(g, c.N, d, d, ws.xop0, ws.ld0))) return rc;
+    }
+    return 0;
+}
+
+}  // namespace fmtp

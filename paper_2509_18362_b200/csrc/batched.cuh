@@ -1,0 +1,57 @@
+// Batched draft path: the K recursive MTP steps for 5..64 sequences per group as a sequence of
+// kernels on one stream, with every weight matrix streamed once per step by the tcgen05 GEMM of
+// skinny_gemm.cuh. (Up to four or eight sequences run in the persistent kernel of megakernel.cu.)
+#pragma once
+#include "mega.cuh"
+
+namespace fmtp {
+
+constexpr int kBatchRows = 64;        // sequences per group (activation columns = 2 x rows <= 128)
+constexpr int kBatchAttnChunk = 256;  // context tokens per attention work item
+constexpr int kBatchMaxSplits = 8;
+
+struct BatchedWs {
+    bf16_t *xop0;                 // [128][ld0]  hi/lo activation operand (projection, QKV, O-proj, MLP and head inputs)
+    bf16_t *xopF;                 // [128][ldF]  hi/lo SwiGLU activation (input of the down projection)
+    float *partial;               // [kBatchMaxSplits][rows][ldp] split-K partial sums
+    float *x;                     // [rows][d]   residual stream
+    float *hout;                  // [rows][d]   final-normed hidden state (recursed in fp32)
+    float *q;                     // [rows][qdim] rotated queries
+    float *att_part;              // [rows][Hq][max_chunks][dh + 2]  (o, m, l) per context chunk
+    unsigned long long *keys;     // [max_K][kBatchRows] argmax keys
+    uint32_t *status;
+    int ld0, ldF, ldp, max_chunks, rows;
+    size_t keys_bytes;
+};
+
+struct BatchedShape {
+    int d, Hq, Hkv, dh, F, V, page, max_ctx, max_K, max_rows;
+    float eps;
+};
+
+// Carves the buffers out of `base` (nullptr: size query); returns the bytes used.
+size_t batched_layout(BatchedWs &ws, unsigned char *base, const BatchedShape &sh);
+
+struct BatchedCall {
+    BatchedShape sh;
+    BatchedWs ws;
+    const float *rope_cos, *rope_sin;     // [max_ctx][dh/2]
+    int n_sm, smem_optin;
+    int B, K, N;
+    const int32_t *ids;                   // subset or NULL
+    const bf16_t *h_last;                 // [B][d]
+    const int32_t *tok_last;              // [B]
+    int32_t *out_drafts;                  // [B][K]
+    bf16_t *out_h;                        // [B][K][d] or NULL
+    float *out_logits;                    // [B][K][N] or NULL
+    uint32_t *user_status;
+    const bf16_t *embed, *lm_head, *g_hnorm, *g_enorm, *w_proj, *g_final;
+    LayerPtrs layer;
+    KvPtrs kv;
+};
+
+// Enqueues all K steps for one group of B <= kBatchRows sequences. Returns a cudaError_t (0 = ok)
+// and adds the kernels launched to *launches.
+int batched_draft(const BatchedCall &c, cudaStream_t stream, long long *launches);
+
+}  // namespace fmtp

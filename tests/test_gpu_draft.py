@@ -92,12 +92,63 @@ def test_tiny_shapes_ragged(B, L, K, N):
     check_draft(got, ref, f"tiny B={B} K={K} N={N}")
 
 
-def test_batch_larger_than_one_launch():
-    """20 sequences with ragged contexts: three launches (8 + 8 + 4 rows) behind one call."""
-    L = [int(x) for x in I.context_lengths(20, 0, 200, 9)]
-    got, ref = run_draft_case(I.TINY, 808, 20, L, 3, 1024, subset="zipf")
-    check_draft(got, ref, "tiny B=20")
-    assert got["launches"] == 3
+@pytest.mark.parametrize("B,lo,hi,K,N,subset", [
+    (20, 0, 200, 3, 1024, "zipf"),        # 20 sequences, ragged contexts below one attention chunk
+    (64, 0, 700, 2, 1000, "uniform"),     # a full group; contexts up to three 256-token attention chunks; ragged subset
+    (9, 250, 260, 4, None, "uniform"),    # contexts crossing the chunk boundary during the K steps; full vocabulary
+    (70, 0, 90, 1, 37, "uniform"),        # two groups (64 + 6); fewer head rows than one 128-row tile
+])
+def test_batched_path_matches_oracle(B, lo, hi, K, N, subset):
+    """More sequences than one persistent-kernel launch takes: the tensor-core GEMM path (every weight
+    streamed once per step for the whole group)."""
+    L = [int(x) for x in I.context_lengths(B, lo, hi, 9 + B)]
+    got, ref = run_draft_case(I.TINY, 800 + B, B, L, K, N, subset=subset, max_ctx=hi + K + 2)
+    check_draft(got, ref, f"tiny batched B={B}")
+    assert got["launches"] > 3            # a sequence of kernels per step, not one persistent launch per group
+    for b in (0, B - 1):
+        for k in range(K):
+            lg = O.head_logits(ref["h_out"][b, k], ref["W"]["lm_head"], ref["ids"])
+            close(got["logits"][b, k], lg, f"tiny batched logits b={b} step {k}")
+
+
+def test_batched_path_odd_geometry():
+    """head_dim 128, 7 query heads per KV head, ffn and d not multiples of the GEMM's 64-wide K block
+    or 128-row tile, 12 sequences."""
+    shape = I.Shape(d=448, n_q_heads=7, n_kv_heads=1, head_dim=128, ffn=1200, vocab=3001, n_layers=1,
+                    rms_eps=1e-6, rope_theta=1e6, page_size=16)
+    L = [int(x) for x in I.context_lengths(12, 0, 400, 3)]
+    got, ref = run_draft_case(shape, 6, 12, L, 3, 777, subset="zipf")
+    check_draft(got, ref, "odd geometry batched")
+
+
+def test_batched_path_bit_reproducible_and_batch_invariant():
+    """Two runs agree bit for bit, and a sequence's result is the same in a group of 12 and of 40."""
+    L = [int(x) for x in I.context_lengths(40, 0, 300, 5)]
+    a, _ = run_draft_case(I.TINY, 4711, 40, L, 3, 1024)
+    b, _ = run_draft_case(I.TINY, 4711, 40, L, 3, 1024)
+    assert np.array_equal(a["drafts"], b["drafts"]) and np.array_equal(a["h_out"], b["h_out"])
+    assert np.array_equal(a["logits"], b["logits"]) and np.array_equal(a["k_pages"], b["k_pages"])
+    # the first 12 sequences alone (same seeds => same weights and inputs for those rows)
+    Bd = _binding()
+    shape = I.TINY
+    W = I.mtp_weights(shape, 4711)
+    kv = I.paged_kv(shape, L, 4, 4712)
+    h = I.hidden_bf16(4713, (40, shape.d))
+    tok = I.token_ids(4714, (40,), shape.vocab)
+    ids = I.subset_uniform(shape.vocab, 1024, 4715)
+    ctx = Bd.Context(shape, max_rows=64, max_K=8, max_ctx=max(L) + 4)
+    dW, dkv = Bd.to_device(W), Bd.to_device(copy_kv(kv))
+    sub = dict(dkv)
+    sub["block_table"] = dkv["block_table"][:12].contiguous()
+    sub["seq_lens"] = dkv["seq_lens"][:12].contiguous()
+    out_d = torch.zeros((12, 3), dtype=torch.int32, device="cuda")
+    out_h = torch.zeros((12, 3, shape.d), dtype=torch.bfloat16, device="cuda")
+    ctx.fastmtp_draft(Bd.mtp_w(dW), Bd.bf16_tensor(h[:12]), torch.from_numpy(tok[:12]).cuda(), Bd.kv(sub), 12, 3,
+                      torch.from_numpy(ids).cuda(), out_d, out_h)
+    torch.cuda.synchronize()
+    assert np.array_equal(out_d.cpu().numpy(), a["drafts"][:12])
+    assert np.array_equal(out_h.float().cpu().numpy(), a["h_out"][:12])
+    ctx.close()
 
 
 def test_odd_geometry():
