@@ -352,6 +352,7 @@ int fastmtp_draft(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_last, con
         return FMTP_EINVAL;
     const int Neff = subset ? N : c->shape.vocab;
     if (B >= c->batched_min) {
+        if (out_h && !aligned16(out_h)) return FMTP_EINVAL;
         // more sequences than one launch of the persistent kernel takes: groups of up to 64 sequences, every
         // weight streamed once per step and group by the tensor-core GEMM path
         for (int b0 = 0; b0 < B; b0 += kBatchRows) {

@@ -10,7 +10,7 @@ namespace fmtp {
 namespace {
 
 constexpr uint32_t kDevBadToken = 0x1u, kDevBadPage = 0x2u, kDevBadPos = 0x4u, kDevAllNan = 0x10u;
-constexpr int kRowThreads = 256;
+constexpr int kRowThreads = 512;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -48,6 +48,30 @@ struct PrologueArgs {
     uint32_t *status, *user_status;
 };
 
+// eight consecutive values -> hi/lo bf16, one 16-byte store each
+__device__ __forceinline__ void store_hilo8(bf16_t *xop, int ld, int r, int j, const float (&v)[8]) {
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint16_t h0, l0, h1, l1;
+        split_bf16(v[2 * i], h0, l0);
+        split_bf16(v[2 * i + 1], h1, l1);
+        hi[i] = (uint32_t)h0 | ((uint32_t)h1 << 16);
+        lo[i] = (uint32_t)l0 | ((uint32_t)l1 << 16);
+    }
+    *reinterpret_cast<uint4 *>(xop + (size_t)(2 * r) * ld + j) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<uint4 *>(xop + (size_t)(2 * r + 1) * ld + j) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+}
+__device__ __forceinline__ void unpack_bf16x8(const uint4 &u, float (&v)[8]) {
+    v[0] = bf16lo_f32(u.x); v[1] = bf16hi_f32(u.x); v[2] = bf16lo_f32(u.y); v[3] = bf16hi_f32(u.y);
+    v[4] = bf16lo_f32(u.z); v[5] = bf16hi_f32(u.z); v[6] = bf16lo_f32(u.w); v[7] = bf16hi_f32(u.w);
+}
+__device__ __forceinline__ void load_f32x8(const float *p, float (&v)[8]) {
+    const float4 a = *reinterpret_cast<const float4 *>(p), b = *reinterpret_cast<const float4 *>(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+
+// Each thread owns eight consecutive columns per pass (d % 64 == 0), so every load and store is 16 bytes.
 __global__ void __launch_bounds__(kRowThreads) prologue_kernel(const PrologueArgs a) {
     __shared__ float red[32];
     __shared__ int s_tok;
@@ -76,20 +100,28 @@ __global__ void __launch_bounds__(kRowThreads) prologue_kernel(const PrologueArg
     }
     const bf16_t *erow = a.embed + (size_t)s_tok * a.d;
     float sh = 0.f, se = 0.f;
-    for (int j = tid; j < a.d; j += kRowThreads) {
-        const float h = a.step == 0 ? bf16bits_f32(a.h_last[(size_t)r * a.d + j]) : a.hout[(size_t)r * a.d + j];
-        const float e = bf16bits_f32(erow[j]);
-        sh += h * h;
-        se += e * e;
+    for (int j = tid * 8; j < a.d; j += kRowThreads * 8) {
+        float h[8], e[8];
+        if (a.step == 0) unpack_bf16x8(*reinterpret_cast<const uint4 *>(a.h_last + (size_t)r * a.d + j), h);
+        else load_f32x8(a.hout + (size_t)r * a.d + j, h);
+        unpack_bf16x8(*reinterpret_cast<const uint4 *>(erow + j), e);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { sh += h[i] * h[i]; se += e[i] * e[i]; }
     }
     sh = block_sum(sh, red);
     se = block_sum(se, red);
     const float rh = 1.0f / sqrtf(sh / (float)a.d + a.eps), re = 1.0f / sqrtf(se / (float)a.d + a.eps);
-    for (int j = tid; j < a.d; j += kRowThreads) {
-        const float h = a.step == 0 ? bf16bits_f32(a.h_last[(size_t)r * a.d + j]) : a.hout[(size_t)r * a.d + j];
-        const float e = bf16bits_f32(erow[j]);
-        store_hilo(a.xop, a.ld, r, j, h * rh * bf16bits_f32(a.g_h[j]));
-        store_hilo(a.xop, a.ld, r, a.d + j, e * re * bf16bits_f32(a.g_e[j]));
+    for (int j = tid * 8; j < a.d; j += kRowThreads * 8) {
+        float h[8], e[8], gh[8], ge[8];
+        if (a.step == 0) unpack_bf16x8(*reinterpret_cast<const uint4 *>(a.h_last + (size_t)r * a.d + j), h);
+        else load_f32x8(a.hout + (size_t)r * a.d + j, h);
+        unpack_bf16x8(*reinterpret_cast<const uint4 *>(erow + j), e);
+        unpack_bf16x8(*reinterpret_cast<const uint4 *>(a.g_h + j), gh);
+        unpack_bf16x8(*reinterpret_cast<const uint4 *>(a.g_e + j), ge);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { h[i] = h[i] * rh * gh[i]; e[i] = e[i] * re * ge[i]; }
+        store_hilo8(a.xop, a.ld, r, j, h);
+        store_hilo8(a.xop, a.ld, r, a.d + j, e);
     }
 }
 
@@ -109,20 +141,46 @@ __global__ void __launch_bounds__(kRowThreads) post_kernel(const PostArgs a) {
     __shared__ float red[32];
     const int r = blockIdx.x, tid = threadIdx.x;
     float ss = 0.f;
-    for (int j = tid; j < a.d; j += kRowThreads) {
-        float v = a.residual ? a.x[(size_t)r * a.d + j] : 0.f;
-        for (int s = 0; s < a.splits; ++s) v += a.partial[((size_t)s * a.rows + r) * a.ldp + j];
-        a.x[(size_t)r * a.d + j] = v;
-        ss += v * v;
+    for (int j = tid * 8; j < a.d; j += kRowThreads * 8) {
+        float v[8], part[kBatchMaxSplits][8];
+        // every load of this pass is issued before the first use
+#pragma unroll
+        for (int s = 0; s < kBatchMaxSplits; ++s)
+            if (s < a.splits) load_f32x8(a.partial + ((size_t)s * a.rows + r) * a.ldp + j, part[s]);
+        if (a.residual) load_f32x8(a.x + (size_t)r * a.d + j, v);
+        else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = 0.f;
+        }
+#pragma unroll
+        for (int s = 0; s < kBatchMaxSplits; ++s)
+            if (s < a.splits) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] += part[s][i];
+            }
+        *reinterpret_cast<float4 *>(a.x + (size_t)r * a.d + j) = make_float4(v[0], v[1], v[2], v[3]);
+        *reinterpret_cast<float4 *>(a.x + (size_t)r * a.d + j + 4) = make_float4(v[4], v[5], v[6], v[7]);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ss += v[i] * v[i];
     }
     ss = block_sum(ss, red);
     const float rs = 1.0f / sqrtf(ss / (float)a.d + a.eps);
-    for (int j = tid; j < a.d; j += kRowThreads) {
-        const float n = a.x[(size_t)r * a.d + j] * rs * bf16bits_f32(a.gain[j]);
-        store_hilo(a.xop, a.ld, r, j, n);
+    for (int j = tid * 8; j < a.d; j += kRowThreads * 8) {
+        float v[8], gn[8];
+        load_f32x8(a.x + (size_t)r * a.d + j, v);
+        unpack_bf16x8(*reinterpret_cast<const uint4 *>(a.gain + j), gn);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = v[i] * rs * gn[i];
+        store_hilo8(a.xop, a.ld, r, j, v);
         if (a.final) {
-            a.hout[(size_t)r * a.d + j] = n;
-            if (a.out_h) a.out_h[((size_t)r * a.K + a.step) * a.d + j] = f32_bf16bits(n);
+            *reinterpret_cast<float4 *>(a.hout + (size_t)r * a.d + j) = make_float4(v[0], v[1], v[2], v[3]);
+            *reinterpret_cast<float4 *>(a.hout + (size_t)r * a.d + j + 4) = make_float4(v[4], v[5], v[6], v[7]);
+            if (a.out_h) {
+                uint32_t o[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) o[i] = (uint32_t)f32_bf16bits(v[2 * i]) | ((uint32_t)f32_bf16bits(v[2 * i + 1]) << 16);
+                *reinterpret_cast<uint4 *>(a.out_h + ((size_t)r * a.K + a.step) * a.d + j) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
         }
     }
 }

@@ -1,4 +1,4 @@
-// Weight-streaming GEMM for 8..64 activation rows on the sm_100a tensor cores (tcgen05 + TMEM).
+// Weight-streaming GEMM for 5..64 activation rows on the sm_100a tensor cores (tcgen05 + TMEM).
 //
 //   D[m, n] = sum_k A[m, k] * X[n, k]      m: weight rows (128 per tile, the MMA's M)
 //                                          n: activation columns (NB = 16..128, the MMA's N)
@@ -7,9 +7,14 @@
 // the high part of activation row r and n = 2r + 1 the low part, so the pair carries an fp32
 // value) is small and re-read from L2 for every tile. One CTA per SM walks a static list of work
 // items (tile, K range). Roles: warps 0-3 epilogue (TMEM -> registers -> global), warp 4 issues
-// the MMAs, warps 5-8 copy 64-wide K slices of A and X into a shared-memory ring with 16-byte
-// cp.async, laid out as the MMA's 128-byte-swizzled K-major tiles. Accumulators are double
-// buffered in TMEM so the epilogue of one item overlaps the MMAs of the next.
+// the MMAs, warps 5-12 copy A and X into a shared-memory ring with 16-byte cp.async, laid out as
+// the MMA's 128-byte-swizzled K-major tiles (64 K elements wide). A ring stage holds KA such
+// 64-wide blocks that are requested back to back, so a weight row is read in pieces of KA x 128
+// contiguous bytes. Accumulators are double buffered in TMEM so the epilogue of one item overlaps
+// the MMAs of the next.
+//
+// A stage's barrier counts one asynchronous arrival per copy thread (cp.async.mbarrier.arrive), so a
+// stage is published the moment its bytes have landed.
 //
 // Every wait is time-bounded; on expiry the CTA raises the timeout flag, drains and returns.
 #pragma once
@@ -17,15 +22,17 @@
 
 namespace fmtp {
 
-constexpr int kGemmThreads = 288;
-constexpr int kGemmBK = 64;                 // K elements per ring stage: one 128-byte swizzle row
+constexpr int kGemmProducers = 256;          // eight copy warps
+constexpr int kGemmThreads = 160 + kGemmProducers;
+constexpr int kGemmBK = 64;                 // K elements per swizzled block: one 128-byte row
 constexpr int kGemmTileM = 128;
 constexpr int kGemmMaxStages = 10;
 constexpr unsigned long long kGemmWaitNs = 2000000000ull;
 
 enum GemmEpilogue {
     EPI_PARTIAL = 0,   // fp32 partial sums  partial[split][r][m] = D[m,2r] + D[m,2r+1]
-    EPI_SWIGLU = 1,    // two accumulators (gate, up): act = silu(g) * u, written as the hi/lo operand of the next GEMM
+    EPI_SWIGLU = 1,    // a tile holds 64 gate rows and the 64 up rows of the same indices: act = silu(g) * u, written as the
+                       // hi/lo operand of the next GEMM
     EPI_ARGMAX = 2,    // per activation row the maximum of (logit, row id) as a packed key (atomicMax), optional fp32 logits
 };
 
@@ -33,10 +40,10 @@ struct GemmArgs {
     const bf16_t *a[3];          // up to three matrices whose rows are concatenated (q, k, v); [rows][lda] bf16
     int a_rows[3];
     int n_seg;
-    const bf16_t *a_up;          // EPI_SWIGLU: the second matrix (same shape as a[0])
+    const bf16_t *a_up;          // EPI_SWIGLU: the up matrix (a[0] is the gate matrix, same shape)
     const int32_t *row_ids;      // optional: GEMM row m reads a[0][row_ids[m]] (compressed output head)
     int V;                       // rows of a[0] when row_ids is used (ids outside are clamped and flagged)
-    int n_rows, K, lda;          // K % 8 == 0
+    int n_rows, K, lda;          // output rows (EPI_SWIGLU: ffn indices); K % 8 == 0
     const bf16_t *x;             // [NB][ldx] bf16
     int ldx, NB, R;              // NB % 16 == 0, 2R <= NB <= 128
     int splits, kb_per_split;    // K is cut into `splits` ranges of kb_per_split 64-wide blocks
@@ -50,6 +57,7 @@ struct GemmArgs {
     long long logits_stride;
     uint32_t *status;
     int n_stages;
+    int force_ka;                // 0: pick the blocks per stage from the shared memory available
 };
 
 struct GemmSmem {
@@ -57,18 +65,11 @@ struct GemmSmem {
     uint64_t tfull[2], tempty[2], drain;
     uint32_t tmem_base, abort_flag;
     unsigned long long kmax[4][64];
+    float exch[64][17];          // EPI_SWIGLU: up-row sums handed to the gate rows' threads
 };
 
-__host__ __device__ inline int gemm_stage_bytes(int NB, bool dual) {
-    return (dual ? 2 : 1) * kGemmTileM * 128 + NB * 128;
-}
-__host__ inline size_t gemm_smem_bytes(int NB, bool dual, int stages) {
-    return 1024 + (size_t)stages * gemm_stage_bytes(NB, dual) + sizeof(GemmSmem);
-}
-__host__ inline int gemm_pick_stages(int NB, bool dual, int smem_optin) {
-    int s = (int)((smem_optin - 1024 - (int)sizeof(GemmSmem)) / gemm_stage_bytes(NB, dual));
-    return s > kGemmMaxStages ? kGemmMaxStages : s;
-}
+__host__ __device__ inline int gemm_kblock_bytes(int NB) { return kGemmTileM * 128 + NB * 128; }
+__host__ __device__ inline int gemm_tile_rows(int epi) { return epi == EPI_SWIGLU ? 64 : kGemmTileM; }
 
 __device__ __forceinline__ bool gemm_wait(GemmSmem *sm, uint64_t *bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -103,75 +104,55 @@ __device__ __forceinline__ bool epi_any(bool flag) {
 // State of one producer thread's walk over the ring.
 struct GemmProducer {
     uint32_t dst0;            // shared address of this thread's chunk in row r0 of stage 0
-    int stage_bytes, S, nb16, c;
+    int stage_bytes, kblock_bytes, S, c;
     int stage;
     uint32_t phase;
-    int pending, arrive_stage;   // copy groups issued but not yet published, and the stage the oldest one filled
 };
 
-// Copies this thread's share of K block kb + J (if it is inside the item) into the next ring stage
-// and publishes the stage filled LAG blocks earlier (LAG + 1 copy groups stay in flight per thread). Source addresses are the per-row
-// pointers plus the immediate J * 128 bytes, so four blocks go out before a pointer register is
-// rewritten. Returns false when a wait gave up.
-template <bool DUAL, int LAG, int J>
-__device__ __forceinline__ bool produce_kblock(const GemmArgs &g, GemmSmem *sm, GemmProducer &pr, int kb, int kb1,
-                                               const bf16_t *(&ap)[8], const bf16_t *(&up)[8],
-                                               const bf16_t *(&xp)[8], const uint32_t (&aok)[8]) {
-    if (kb + J >= kb1) return true;
-    if (!gemm_wait(sm, &sm->empty[pr.stage], pr.phase ^ 1u)) return false;
+// Copies this thread's share of K block kb + J (if it is inside the item) into block J of the
+// current stage. Source addresses are the per-row pointers plus the immediate J * 128 bytes, so
+// all blocks of a stage go out before a pointer register is rewritten.
+template <int J>
+__device__ __forceinline__ void produce_kblock(const GemmArgs &g, const GemmProducer &pr, int kb, int kb1,
+                                               const bf16_t *(&ap)[4], const bf16_t *(&xp)[4],
+                                               const uint32_t (&aok)[4], const uint32_t (&xok)[4]) {
+    if (kb + J >= kb1) return;
     const bool kvalid = (kb + J) * kGemmBK + pr.c * 8 < g.K;
-    const uint32_t dst = pr.dst0 + (uint32_t)pr.stage * pr.stage_bytes;
-    const uint32_t dx = dst + (DUAL ? 32768 : 16384);
+    const uint32_t dst = pr.dst0 + (uint32_t)pr.stage * pr.stage_bytes + (uint32_t)J * pr.kblock_bytes;
+    const uint32_t dx = dst + 16384;
     if (kvalid) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) cp_async16_off<J * 128>(dst + i * 2048, ap[i], aok[i]);
-        if (DUAL) {
+        for (int i = 0; i < 4; ++i) cp_async16_off<J * 128>(dst + i * 4096, ap[i], aok[i]);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) cp_async16_off<J * 128>(dst + 16384 + i * 2048, up[i], aok[i]);
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-            if (i < pr.nb16) cp_async16_off<J * 128>(dx + i * 2048, xp[i], 16u);
+        for (int i = 0; i < 4; ++i)
+            if (xok[i]) cp_async16_off<J * 128>(dx + i * 4096, xp[i], 16u);
     } else {   // this chunk column lies beyond K: zeros, nothing is read
 #pragma unroll
-        for (int i = 0; i < 8; ++i) cp_async16_off<0>(dst + i * 2048, g.a[0], 0u);
-        if (DUAL) {
+        for (int i = 0; i < 4; ++i) cp_async16_off<0>(dst + i * 4096, g.a[0], 0u);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) cp_async16_off<0>(dst + 16384 + i * 2048, g.a[0], 0u);
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-            if (i < pr.nb16) cp_async16_off<0>(dx + i * 2048, g.a[0], 0u);
+        for (int i = 0; i < 4; ++i)
+            if (xok[i]) cp_async16_off<0>(dx + i * 4096, g.a[0], 0u);
     }
-    cp_async_commit();
-    if (++pr.pending > LAG) {     // the oldest group has landed: publish its stage
-        cp_async_wait_group<LAG>();
-        fence_proxy_async();
-        mbar_arrive(&sm->full[pr.arrive_stage]);
-        if (++pr.arrive_stage == pr.S) pr.arrive_stage = 0;
-        --pr.pending;
-    }
-    if (++pr.stage == pr.S) { pr.stage = 0; pr.phase ^= 1u; }
-    return true;
 }
 
-template <bool DUAL, int LAG>
+// KA 64-wide K blocks per ring stage; every stage of the ring can be in flight.
+template <int KA>
 __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const GemmArgs g) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     unsigned char *ring = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
     const int S = g.n_stages;
-    const int stage_bytes = gemm_stage_bytes(g.NB, DUAL);
+    const int kblock_bytes = gemm_kblock_bytes(g.NB);
+    const int stage_bytes = KA * kblock_bytes;
     GemmSmem *sm = reinterpret_cast<GemmSmem *>(ring + (size_t)S * stage_bytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    const int acc_cols = (g.NB + 31) & ~31;                 // TMEM columns of one accumulator
-    const int buf_cols = acc_cols * (DUAL ? 2 : 1);         // ... of one buffer
+    const int buf_cols = (g.NB + 31) & ~31;                 // TMEM columns of one accumulator buffer
     uint32_t alloc_cols = 32;
     while ((int)alloc_cols < 2 * buf_cols) alloc_cols <<= 1;
 
     if (tid == 0) {
-        for (int s = 0; s < S; ++s) { mbar_init(&sm->full[s], 128); mbar_init(&sm->empty[s], 1); }
+        for (int s = 0; s < S; ++s) { mbar_init(&sm->full[s], kGemmProducers); mbar_init(&sm->empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&sm->tfull[b], 1); mbar_init(&sm->tempty[b], 128); }
         mbar_init(&sm->drain, 1);
         sm->abort_flag = 0;
@@ -186,33 +167,40 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
     tc_fence_after_sync();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&sm->tmem_base);
 
-    const int n_tiles = (g.n_rows + kGemmTileM - 1) / kGemmTileM;
+    const int tile_rows = gemm_tile_rows(g.epi);
+    const int n_tiles = (g.n_rows + tile_rows - 1) / tile_rows;
     const int n_items = n_tiles * g.splits;
     const int n_kb = (g.K + kGemmBK - 1) / kGemmBK;
 
     if (warp >= 5) {
-        // ================= producers: 128 threads, thread pt copies chunk column c of rows r0 + 16 i
+        // ================= producers: thread pt copies chunk column c of tile rows r0 + 32 i
         const int pt = tid - 160;
         const int c = pt & 7, r0 = pt >> 3;
         GemmProducer pr;
         pr.dst0 = smem_u32(ring) + (uint32_t)(r0 * 128 + ((c ^ (r0 & 7)) << 4));
-        pr.stage_bytes = stage_bytes; pr.S = S; pr.nb16 = g.NB >> 4; pr.c = c;
-        pr.stage = 0; pr.phase = 0; pr.pending = 0; pr.arrive_stage = 0;
+        pr.stage_bytes = stage_bytes; pr.kblock_bytes = kblock_bytes; pr.S = S; pr.c = c;
+        pr.stage = 0; pr.phase = 0;
         bool ok_run = true;
         for (int item = blockIdx.x; item < n_items && ok_run; item += gridDim.x) {
             const int tile = item / g.splits, split = item - tile * g.splits;
             const int kb0 = split * g.kb_per_split;
             int kb1 = kb0 + g.kb_per_split;
             if (kb1 > n_kb) kb1 = n_kb;
-            const bf16_t *ap[8];
-            const bf16_t *up[8];
-            uint32_t aok[8];
+            const bf16_t *ap[4];
+            uint32_t aok[4], xok[4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                int m = tile * kGemmTileM + r0 + 16 * i;
+            for (int i = 0; i < 4; ++i) {
+                const int tr = r0 + 32 * i;
+                const bf16_t *base = g.a[0];
+                int m;
+                if (g.epi == EPI_SWIGLU) {             // tile rows 0-63: gate rows, 64-127: the up rows of the same indices
+                    m = tile * 64 + (tr & 63);
+                    if (tr >= 64) base = g.a_up;
+                } else {
+                    m = tile * kGemmTileM + tr;
+                }
                 aok[i] = m < g.n_rows ? 16u : 0u;
                 if (m >= g.n_rows) m = g.n_rows - 1;
-                const bf16_t *base = g.a[0];
                 int row = m;
                 if (g.row_ids) {
                     int id = g.row_ids[m];
@@ -225,33 +213,32 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
                         if (row >= g.a_rows[1]) { row -= g.a_rows[1]; base = g.a[2]; }
                     }
                 }
-                const size_t off = (size_t)row * g.lda + (size_t)kb0 * kGemmBK + c * 8;
-                ap[i] = base + off;
-                if (DUAL) up[i] = g.a_up + off;
+                ap[i] = base + (size_t)row * g.lda + (size_t)kb0 * kGemmBK + c * 8;
             }
-            const bf16_t *xp[8];
+            const bf16_t *xp[4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                int n = r0 + 16 * i;
+            for (int i = 0; i < 4; ++i) {
+                int n = r0 + 32 * i;
+                xok[i] = n < g.NB ? 1u : 0u;
                 if (n >= g.NB) n = g.NB - 1;
                 xp[i] = g.x + (size_t)n * g.ldx + (size_t)kb0 * kGemmBK + c * 8;
             }
-            for (int kb = kb0; kb < kb1 && ok_run; kb += 4) {
-                ok_run = produce_kblock<DUAL, LAG, 0>(g, sm, pr, kb, kb1, ap, up, xp, aok) &&
-                         produce_kblock<DUAL, LAG, 1>(g, sm, pr, kb, kb1, ap, up, xp, aok) &&
-                         produce_kblock<DUAL, LAG, 2>(g, sm, pr, kb, kb1, ap, up, xp, aok) &&
-                         produce_kblock<DUAL, LAG, 3>(g, sm, pr, kb, kb1, ap, up, xp, aok);
+            for (int kb = kb0; kb < kb1; kb += KA) {
+                if (!gemm_wait(sm, &sm->empty[pr.stage], pr.phase ^ 1u)) { ok_run = false; break; }
+                produce_kblock<0>(g, pr, kb, kb1, ap, xp, aok, xok);
+                if constexpr (KA > 1) produce_kblock<1>(g, pr, kb, kb1, ap, xp, aok, xok);
+                if constexpr (KA > 2) {
+                    produce_kblock<2>(g, pr, kb, kb1, ap, xp, aok, xok);
+                    produce_kblock<3>(g, pr, kb, kb1, ap, xp, aok, xok);
+                }
+                // this thread's arrival on the stage's barrier fires when its copies above have landed
+                cp_async_arrive(&sm->full[pr.stage]);
+                if (++pr.stage == S) { pr.stage = 0; pr.phase ^= 1u; }
 #pragma unroll
-                for (int i = 0; i < 8; ++i) { ap[i] += 4 * kGemmBK; if (DUAL) up[i] += 4 * kGemmBK; xp[i] += 4 * kGemmBK; }
+                for (int i = 0; i < 4; ++i) { ap[i] += KA * kGemmBK; xp[i] += KA * kGemmBK; }
             }
         }
-        cp_async_wait_group<0>();
-        fence_proxy_async();
-        while (pr.pending > 0) {
-            mbar_arrive(&sm->full[pr.arrive_stage]);
-            if (++pr.arrive_stage == S) pr.arrive_stage = 0;
-            --pr.pending;
-        }
+        cp_async_wait_all();
     } else if (warp == 4) {
         // ================= MMA issue: one thread
         if (lane == 0) {
@@ -268,17 +255,20 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
                 if (!gemm_wait(sm, &sm->tempty[buf], tphase[buf] ^ 1u)) break;
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + (uint32_t)(buf * buf_cols);
-                for (int kb = kb0; kb < kb1; ++kb) {
+                for (int kb = kb0; kb < kb1; kb += KA) {
                     if (!gemm_wait(sm, &sm->full[stage], phase)) { ok_run = false; break; }
+                    fence_proxy_async();          // the copies' shared-memory writes, before the tensor core reads them
                     tc_fence_after_sync();
-                    const uint32_t sa = smem_u32(ring) + (uint32_t)stage * stage_bytes;
-                    const uint32_t sb = sa + (DUAL ? 32768 : 16384);
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const bool acc = (kb > kb0) || (ks > 0);
-                        const uint64_t bd = umma_smem_desc(sb + ks * 32);
-                        umma_bf16(d0, umma_smem_desc(sa + ks * 32), bd, idesc, acc);
-                        if (DUAL) umma_bf16(d0 + acc_cols, umma_smem_desc(sa + 16384 + ks * 32), bd, idesc, acc);
+                    for (int j = 0; j < KA; ++j) {
+                        if (kb + j < kb1) {
+                            const uint32_t sa = smem_u32(ring) + (uint32_t)stage * stage_bytes + (uint32_t)j * kblock_bytes;
+                            const uint32_t sb = sa + 16384;
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks)
+                                umma_bf16(d0, umma_smem_desc(sa + ks * 32), umma_smem_desc(sb + ks * 32), idesc,
+                                          (kb + j > kb0) || (ks > 0));
+                        }
                     }
                     umma_commit(&sm->empty[stage]);
                     if (++stage == S) { stage = 0; phase ^= 1u; }
@@ -294,7 +284,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
         }
         __syncwarp();
     } else {
-        // ================= epilogue: thread = one weight row of the tile (TMEM lane 32*warp + lane)
+        // ================= epilogue: thread = one row of the tile (TMEM lane 32*warp + lane)
         uint32_t tphase[2] = {0, 0};
         int buf = 0;
         for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
@@ -302,7 +292,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
             // the 128 epilogue threads agree on the outcome of the wait before any of them moves on
             if (epi_any(!gemm_wait(sm, &sm->tfull[buf], tphase[buf]))) break;
             tc_fence_after_sync();
-            const int m = tile * kGemmTileM + warp * 32 + lane;
+            const int tr = warp * 32 + lane;
+            const int m = g.epi == EPI_SWIGLU ? tile * 64 + (tr & 63) : tile * kGemmTileM + tr;
             const bool m_ok = m < g.n_rows;
             const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * buf_cols);
             uint32_t row_id = (uint32_t)m;
@@ -320,20 +311,26 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
                         if (r < g.R && m_ok) g.partial[((size_t)split * g.R + r) * g.ldp + m] = v[2 * j] + v[2 * j + 1];
                     }
                 } else if (g.epi == EPI_SWIGLU) {
-                    float u[32];
-                    tmem_ld32(t0 + acc_cols + c0, u);
+                    if (warp >= 2) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int r = (c0 >> 1) + j;
-                        if (r < g.R && m_ok) {
-                            const float gv = v[2 * j] + v[2 * j + 1], uv = u[2 * j] + u[2 * j + 1];
-                            const float act = gv / (1.0f + expf(-gv)) * uv;
-                            uint16_t hi, lo;
-                            split_bf16(act, hi, lo);
-                            g.xop_out[(size_t)(2 * r) * g.ld_out + m] = hi;
-                            g.xop_out[(size_t)(2 * r + 1) * g.ld_out + m] = lo;
+                        for (int j = 0; j < 16; ++j) sm->exch[tr - 64][j] = v[2 * j] + v[2 * j + 1];
+                    }
+                    bar_sync(1, 128);
+                    if (warp < 2) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int r = (c0 >> 1) + j;
+                            if (r < g.R && m_ok) {
+                                const float gv = v[2 * j] + v[2 * j + 1], uv = sm->exch[tr][j];
+                                const float act = gv / (1.0f + expf(-gv)) * uv;
+                                uint16_t hi, lo;
+                                split_bf16(act, hi, lo);
+                                g.xop_out[(size_t)(2 * r) * g.ld_out + m] = hi;
+                                g.xop_out[(size_t)(2 * r + 1) * g.ld_out + m] = lo;
+                            }
                         }
                     }
+                    bar_sync(1, 128);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
@@ -379,15 +376,20 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
 // Launches the GEMM on `stream` with one CTA per SM (fewer when there are fewer work items).
 // Returns the cudaError_t of the launch.
 inline int skinny_gemm_launch(GemmArgs g, int n_sm, int smem_optin, cudaStream_t stream) {
-    const bool dual = g.epi == EPI_SWIGLU;
-    g.n_stages = gemm_pick_stages(g.NB, dual, smem_optin);
-    if (g.n_stages < 4) return (int)cudaErrorInvalidConfiguration;
-    const size_t smem = gemm_smem_bytes(g.NB, dual, g.n_stages);
-    const int n_items = ((g.n_rows + kGemmTileM - 1) / kGemmTileM) * g.splits;
+    const int avail = smem_optin - 1024 - (int)sizeof(GemmSmem);
+    const int kbb = gemm_kblock_bytes(g.NB);
+    // blocks per stage: as many as still leave a ring of three stages
+    int ka = g.force_ka > 0 ? g.force_ka : (avail / (4 * kbb) >= 3 ? 4 : avail / (2 * kbb) >= 3 ? 2 : 1);
+    int stages = avail / (ka * kbb);
+    if (stages > kGemmMaxStages) stages = kGemmMaxStages;
+    if (stages < 3) return (int)cudaErrorInvalidConfiguration;
+    g.n_stages = stages;
+    const size_t smem = 1024 + (size_t)stages * ka * kbb + sizeof(GemmSmem);
+    const int tile_rows = gemm_tile_rows(g.epi);
+    const int n_items = ((g.n_rows + tile_rows - 1) / tile_rows) * g.splits;
     const int grid = n_items < n_sm ? n_items : n_sm;
-    // the ring must be at least two stages deeper than the copy groups a thread keeps in flight
-    void (*kern)(const GemmArgs) = dual ? (g.n_stages >= 5 ? skinny_gemm_kernel<true, 3> : skinny_gemm_kernel<true, 2>)
-                                        : (g.n_stages >= 5 ? skinny_gemm_kernel<false, 3> : skinny_gemm_kernel<false, 2>);
+    void (*kern)(const GemmArgs) = ka == 4 ? skinny_gemm_kernel<4> : ka == 2 ? skinny_gemm_kernel<2> : skinny_gemm_kernel<1>;
+    if (ka != 1 && ka != 2 && ka != 4) return (int)cudaErrorInvalidConfiguration;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
     kern<<<grid, kGemmThreads, smem, stream>>>(g);

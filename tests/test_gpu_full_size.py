@@ -73,6 +73,45 @@ def test_7b_draft_matches_oracle(seven_b, B, ctx_lens, subset_kind):
     print(f"7B B={B}: drafts {drafts.tolist()} near-tie exemptions {exempt}")
 
 
+def test_7b_batched_draft_matches_oracle_on_sampled_sequences(seven_b):
+    """16 sequences with ragged contexts (uniform in [512, 3000]) through the batched tensor-core path at the
+    7B shape; three of them (first, last, the longest context) are recomputed by the oracle."""
+    from paper_2509_18362_b200 import binding as Bd
+    shape, W, dW = seven_b
+    B, K, N, seed = 16, 3, 32768, 77
+    ctx_lens = [int(x) for x in I.context_lengths(B, 512, 3000, seed)]
+    kv = I.paged_kv(shape, ctx_lens, K + 1, seed + 1)
+    h = I.hidden_bf16(seed + 2, (B, shape.d))
+    tok = I.token_ids(seed + 3, (B,), shape.vocab)
+    ids = I.subset_zipf(shape.vocab, N, seed + 4)
+    ctx = Bd.Context(shape, max_rows=B, max_K=8, max_ctx=max(ctx_lens) + K + 1)
+    dkv = Bd.to_device(copy_kv(kv))
+    out_d = torch.full((B, K), -1, dtype=torch.int32, device="cuda")
+    out_h = torch.zeros((B, K, shape.d), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx.fastmtp_draft(Bd.mtp_w(dW), Bd.bf16_tensor(h), torch.from_numpy(tok).cuda(), Bd.kv(dkv), B, K,
+                      torch.from_numpy(ids).cuda(), out_d, out_h, None, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    drafts, hout = out_d.cpu().numpy(), out_h.float().cpu().numpy()
+    gk = Bd.bf16_bits(dkv["k_pages"])
+    sel = sorted({0, B - 1, int(np.argmax(ctx_lens))})
+    okv = copy_kv(kv)
+    okv["block_table"], okv["seq_lens"] = okv["block_table"][sel], okv["seq_lens"][sel]
+    ref = O.draft(shape, W, h[sel], tok[sel], okv, K, ids, forced=drafts[sel])
+    exempt = ids_match(drafts[sel], ref["drafts"], ref["gap"], "7B batched drafts")
+    close(hout[sel], ref["h_out"], "7B batched h_out")
+    for i, b in enumerate(sel):
+        for k in range(K):
+            pos = ctx_lens[b] + k
+            page = int(kv["block_table"][b, pos // shape.page_size])
+            close(O.bf16_to_f64(gk[page, :, pos % shape.page_size]),
+                  O.bf16_to_f64(okv["k_pages"][page, :, pos % shape.page_size]), "7B batched K append")
+    ctx.close()
+    O.clear_weight_memo()
+    print(f"7B batched B={B}: near-tie exemptions {exempt}")
+
+
 def test_verify_accept_full_size():
     """[64, 4, 152064] bf16 logits with planted prefix lengths: exact recovery, equal to the oracle."""
     from paper_2509_18362_b200 import binding as Bd
