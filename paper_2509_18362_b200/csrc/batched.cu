@@ -267,19 +267,29 @@ __global__ void __launch_bounds__(kAttnThreads) attn_chunk_kernel(const AttnArgs
     const int32_t *bt = a.kv.block_table + (size_t)r * a.kv.max_pages;
 
     // ---- K/V copies: thread copies 16-byte pieces; a 64-token block of K or V is 64 x DH*2 bytes
+    // (all addresses of a block are formed before the first copy is issued, each in registers of its own)
     auto issue = [&](int blk) {
         unsigned char *st = smem + (size_t)(blk % kAttnStages) * STAGE;
         constexpr int PIECES = DH / 8;                      // 16-byte pieces per row
-        for (int i = tid; i < kAttnBlk * PIECES; i += kAttnThreads) {
-            const int t = i / PIECES, pc = i - t * PIECES;
-            int pos = t0 + blk * kAttnBlk + t;
-            const uint32_t ok = pos < n_ctx ? 16u : 0u;
+        constexpr int NIT = kAttnBlk * PIECES / kAttnThreads;
+        constexpr int TSTEP = kAttnThreads / PIECES;        // tokens between a thread's consecutive pieces
+        const int pc = tid % PIECES, tl = tid / PIECES;
+        size_t off[NIT];
+        uint32_t ok[NIT];
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            int pos = t0 + blk * kAttnBlk + tl + it * TSTEP;
+            ok[it] = pos < n_ctx ? 16u : 0u;
             if (pos >= n_ctx) pos = n_ctx - 1;
             int page = bt[pos / a.page];
             if ((unsigned)page >= (unsigned)a.kv.num_pages) { atomicOr(a.status, kDevBadPage); page = 0; }
-            const size_t off = (((size_t)page * a.Hkv + kvh) * a.page + (pos % a.page)) * DH + pc * 8;
-            cp_async16_off<0>(smem_u32(st + t * ROWB + pc * 16), a.kv.k_pages + off, ok);
-            cp_async16_off<0>(smem_u32(st + kAttnBlk * ROWB + t * ROWB + pc * 16), a.kv.v_pages + off, ok);
+            off[it] = (((size_t)page * a.Hkv + kvh) * a.page + (pos % a.page)) * DH + pc * 8;
+        }
+        const uint32_t d0 = smem_u32(st + tl * ROWB + pc * 16);
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            cp_async16_off<0>(d0 + it * TSTEP * ROWB, a.kv.k_pages + off[it], ok[it]);
+            cp_async16_off<0>(d0 + kAttnBlk * ROWB + it * TSTEP * ROWB, a.kv.v_pages + off[it], ok[it]);
         }
         cp_async_commit();
     };
@@ -419,16 +429,41 @@ struct MergeArgs {
 };
 
 __global__ void attn_merge_kernel(const MergeArgs a) {
+    __shared__ float red[8];
     const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x;
     const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
     const int n_ctx = min(a.kv.seq_lens[r] + a.step, max_tokens - 1) + 1;
     const int n_chunks = (n_ctx + kBatchAttnChunk - 1) / kBatchAttnChunk;
-    const float *base = a.att_part + ((size_t)r * a.Hq + head) * a.max_chunks * (a.dh + 2);
+    const int stride = a.dh + 2;
+    const float *base = a.att_part + ((size_t)r * a.Hq + head) * a.max_chunks * stride;
+    // the chunks' maxima: each thread reads some, then a block-wide maximum (exact, order-free)
     float m = -INFINITY;
-    for (int c = 0; c < n_chunks; ++c) m = fmaxf(m, base[(size_t)c * (a.dh + 2) + a.dh]);
+    for (int c = j; c < n_chunks; c += blockDim.x) m = fmaxf(m, base[(size_t)c * stride + a.dh]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((j & 31) == 0) red[j >> 5] = m;
+    __syncthreads();
+    m = red[0];
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) m = fmaxf(m, red[w]);
+    // weighted sums in ascending chunk order
     float acc = 0.f, l = 0.f;
-    for (int c = 0; c < n_chunks; ++c) {
-        const float *src = base + (size_t)c * (a.dh + 2);
+    int c = 0;
+    for (; c + 4 <= n_chunks; c += 4) {
+        float mv[4], lv[4], ov[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float *src = base + (size_t)(c + u) * stride;
+            mv[u] = src[a.dh]; lv[u] = src[a.dh + 1]; ov[u] = src[j];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float f = expf(mv[u] - m);
+            acc += ov[u] * f;
+            l += lv[u] * f;
+        }
+    }
+    for (; c < n_chunks; ++c) {
+        const float *src = base + (size_t)c * stride;
         const float f = expf(src[a.dh] - m);
         acc += src[j] * f;
         l += src[a.dh + 1] * f;
