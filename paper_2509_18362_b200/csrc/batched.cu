@@ -471,6 +471,55 @@ __global__ void attn_merge_kernel(const MergeArgs a) {
     store_hilo(a.xop, a.ld, r, head * a.dh + j, acc / l);
 }
 
+// ---- the subset in ascending id order. The argmax over the subset does not depend on the order of
+// its rows, and gathering head rows in address order keeps the 128 rows of a GEMM tile within a few
+// memory pages (an unsorted subset spreads them over the whole matrix and the address translation
+// misses cost ~25 % of the head's stream rate). Membership bitmap, then a one-block compaction.
+__global__ void ids_mark_kernel(const int32_t *ids, int N, int V, uint32_t *bitmap, uint32_t *status) {
+    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < N; j += gridDim.x * blockDim.x) {
+        int id = ids[j];
+        if ((unsigned)id >= (unsigned)V) { atomicOr(status, kDevBadToken); id = 0; }
+        atomicOr(&bitmap[id >> 5], 1u << (id & 31));
+    }
+}
+
+__global__ void __launch_bounds__(1024) ids_compact_kernel(const uint32_t *bitmap, int n_words, int32_t *sorted, int N) {
+    __shared__ int warp_tot[32];
+    __shared__ int s_total, s_last;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per = (n_words + 1023) / 1024;
+    const int w0 = tid * per, w1 = min(w0 + per, n_words);
+    int cnt = 0;
+    for (int w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    int base = 0;
+    for (int w = 0; w < warp; ++w) base += warp_tot[w];
+    if (tid == 1023) s_total = base + incl;
+    int pos = base + incl - cnt;
+    for (int w = w0; w < w1; ++w) {
+        uint32_t bits = bitmap[w];
+        while (bits) {
+            const int b = __ffs(bits) - 1;
+            bits &= bits - 1;
+            if (pos < N) sorted[pos] = w * 32 + b;
+            ++pos;
+        }
+    }
+    __syncthreads();
+    // duplicates in the caller's array leave fewer distinct ids than N: repeat the last one
+    const int total = min(s_total, N);
+    if (tid == 0) s_last = sorted[total - 1];
+    __syncthreads();
+    for (int j = total + tid; j < N; j += 1024) sorted[j] = s_last;
+}
+
 int pick_splits(int n_tiles, int n_kb, int n_sm) {
     int best = 1;
     double best_eff = 0.0;
@@ -512,6 +561,8 @@ size_t batched_layout(BatchedWs &ws, unsigned char *base, const BatchedShape &sh
     ws.att_part = reinterpret_cast<float *>(take((size_t)rows * sh.Hq * ws.max_chunks * (sh.dh + 2) * 4));
     ws.keys_bytes = (size_t)(sh.max_K > 1 ? sh.max_K : 1) * kBatchRows * 8 + 256;
     ws.keys = reinterpret_cast<unsigned long long *>(take(ws.keys_bytes));
+    ws.id_bitmap = reinterpret_cast<uint32_t *>(take((size_t)((sh.V + 31) / 32) * 4));
+    ws.sorted_ids = reinterpret_cast<int32_t *>(take((size_t)sh.V * 4));
     ws.status = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned char *>(ws.keys) + ws.keys_bytes - 256);
     if (!base) ws.status = nullptr;
     return align_up(off, 256);
@@ -525,6 +576,19 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
     const int NB = (2 * B + 15) / 16 * 16;
     cudaError_t e = cudaMemsetAsync(ws.keys, 0, ws.keys_bytes, st);     // argmax keys and the status word
     if (e != cudaSuccess) return (int)e;
+
+    // head rows in ascending id order (the debug logits keep the caller's order, so they skip this)
+    const int32_t *head_ids = c.ids;
+    if (c.ids && !c.out_logits) {
+        const int n_words = (sh.V + 31) / 32;
+        e = cudaMemsetAsync(ws.id_bitmap, 0, (size_t)n_words * 4, st);
+        if (e != cudaSuccess) return (int)e;
+        ids_mark_kernel<<<(c.N + 255) / 256 < 1024 ? (c.N + 255) / 256 : 1024, 256, 0, st>>>(c.ids, c.N, sh.V, ws.id_bitmap, ws.status);
+        ids_compact_kernel<<<1, 1024, 0, st>>>(ws.id_bitmap, n_words, ws.sorted_ids, c.N);
+        *launches += 2;
+        if ((e = cudaGetLastError()) != cudaSuccess) return (int)e;
+        head_ids = ws.sorted_ids;
+    }
 
     auto gemm = [&](GemmArgs &g, int n_rows, int Kdim, int lda, const bf16_t *x, int ldx) -> int {
         g.n_rows = n_rows; g.K = Kdim; g.lda = lda; g.x = x; g.ldx = ldx; g.NB = NB; g.R = B;
@@ -617,7 +681,7 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
         // compressed head + argmax (Eq. 3)
         g = GemmArgs{};
         g.a[0] = c.lm_head; g.a_rows[0] = c.N; g.n_seg = 1; g.epi = EPI_ARGMAX;
-        g.row_ids = c.ids; g.V = sh.V;
+        g.row_ids = head_ids; g.V = sh.V;
         g.keys = ws.keys + (size_t)step * kBatchRows;
         g.logits = c.out_logits ? c.out_logits + (size_t)step * c.N : nullptr;
         g.logits_stride = (long long)K * c.N;

@@ -19,6 +19,8 @@ struct BatchedWs {
     float *q;                     // [rows][qdim] rotated queries
     float *att_part;              // [rows][Hq][max_chunks][dh + 2]  (o, m, l) per context chunk
     unsigned long long *keys;     // [max_K][kBatchRows] argmax keys
+    uint32_t *id_bitmap;          // [ceil(V/32)] membership bits of the subset
+    int32_t *sorted_ids;          // [V] the subset in ascending id order
     uint32_t *status;
     int ld0, ldF, ldp, max_chunks, rows;
     size_t keys_bytes;

@@ -109,6 +109,36 @@ def test_batched_path_matches_oracle(B, lo, hi, K, N, subset):
         for k in range(K):
             lg = O.head_logits(ref["h_out"][b, k], ref["W"]["lm_head"], ref["ids"])
             close(got["logits"][b, k], lg, f"tiny batched logits b={b} step {k}")
+    # the production call (no debug logits) gathers the head rows in ascending id order: same results
+    prod, _ = run_draft_case(I.TINY, 800 + B, B, L, K, N, subset=subset, max_ctx=hi + K + 2, want_logits=False)
+    assert np.array_equal(prod["drafts"], got["drafts"]) and np.array_equal(prod["h_out"], got["h_out"])
+
+
+def test_batched_path_subset_with_repeated_ids():
+    """A subset array that repeats ids (outside the contract, but harmless): same drafts as the distinct subset."""
+    Bd = _binding()
+    shape = I.TINY
+    W = I.mtp_weights(shape, 31)
+    L = [int(x) for x in I.context_lengths(10, 0, 50, 32)]
+    kv = I.paged_kv(shape, L, 3, 33)
+    h = I.hidden_bf16(34, (10, shape.d))
+    tok = I.token_ids(35, (10,), shape.vocab)
+    ids = I.subset_uniform(shape.vocab, 300, 36)
+    rep = np.concatenate([ids, ids[:77], ids[5:6]]).astype(np.int32)
+    dW = Bd.to_device(W)
+    outs = []
+    for arr in (ids, rep):
+        ctx = Bd.Context(shape, max_rows=16, max_K=8, max_ctx=64)
+        dkv = Bd.to_device(copy_kv(kv))
+        out_d = torch.zeros((10, 2), dtype=torch.int32, device="cuda")
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        ctx.fastmtp_draft(Bd.mtp_w(dW), Bd.bf16_tensor(h), torch.from_numpy(tok).cuda(), Bd.kv(dkv), 10, 2,
+                          torch.from_numpy(arr).cuda(), out_d, None, None, st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        outs.append(out_d.cpu().numpy())
+        ctx.close()
+    assert np.array_equal(outs[0], outs[1])
 
 
 def test_batched_path_odd_geometry():
