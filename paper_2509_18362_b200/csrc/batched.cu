@@ -232,58 +232,143 @@ __global__ void qkv_finish_kernel(const QkvArgs a) {
     dst[e + half] = f32_bf16bits(hi);
 }
 
-// ---- attention over one 256-token chunk of one (sequence, KV head): the Hq/Hkv query heads of
-// the group share the K/V stream. Scores and the weighted sum run on mma.sync.m16n8k16 with the
-// query (and the probabilities) as the A operand, rows 0-7 the high bf16 parts of the heads and
-// rows 8-15 the low parts, so both products carry fp32-accurate inputs. Each warp owns 16 tokens of
-// every 64-token block and keeps its own running (max, sum, output); the four warps merge in
-// fixed order at the end. Output: unnormalised o, running max m and sum l per head and chunk.
+// ---- attention. A work item is one 256-token chunk of one (sequence, KV head); the Hq/Hkv query
+// heads of the group share the K/V stream. One persistent CTA per SM walks its items (item index =
+// CTA, CTA + grid, ...) as one continuous stream of 64-token blocks through a shared-memory ring,
+// so the copies of the next items are in flight while the current one is computed. Scores and the
+// weighted sum run on mma.sync.m16n8k16 with the query (and the probabilities) as the A operand,
+// rows 0-7 the high bf16 parts of the heads and rows 8-15 the low parts, so both products carry
+// fp32-accurate inputs. Each warp owns 16 tokens of every block and keeps its own running
+// (max, sum, output); the four warps merge in fixed order at the end of the item.
+// Output per item: unnormalised o, running max m and sum l per head.
 struct AttnArgs {
-    int Hq, Hkv, dh, page, max_ctx, step, max_chunks;
+    int Hq, Hkv, dh, page, page_shift, max_ctx, step, max_chunks, B;
     const float *q;              // [rows][Hq*dh]
     KvPtrs kv;
     float *att_part;             // [rows][Hq][max_chunks][dh+2]
     uint32_t *status;
 };
 
-constexpr int kAttnBlk = 64;                 // tokens per pipeline stage
-constexpr int kAttnStages = 3;
-constexpr int kAttnThreads = 128;
+constexpr int kAttnBlk = 64;                 // tokens per ring stage
+constexpr int kAttnStages = 5;
+constexpr int kAttnThreads = 128;            // compute threads (warps 0-3); warps 4-7 only issue the copies
+constexpr unsigned long long kAttnWaitNs = 2000000000ull;
+
+struct AttnItem {                            // one (sequence, KV head, chunk), CTA-uniform
+    int r, kvh, chunk, t0, n_ctx, n_blk;
+    const int32_t *bt;
+};
 
 template <int DH>
-__global__ void __launch_bounds__(kAttnThreads) attn_chunk_kernel(const AttnArgs a) {
-    constexpr int ROWB = DH * 2 + 16;                       // padded row: conflict-free fragment loads
-    constexpr int STAGE = 2 * kAttnBlk * ROWB;              // K block then V block
-    extern __shared__ __align__(16) unsigned char smem[];
-    const int chunk = blockIdx.x, kvh = blockIdx.y, r = blockIdx.z;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
-    const int n_ctx = min(a.kv.seq_lens[r] + a.step, max_tokens - 1) + 1;     // visible positions 0 .. n_ctx-1
-    const int t0 = chunk * kBatchAttnChunk;
-    if (t0 >= n_ctx) return;
-    const int n_tok = min(kBatchAttnChunk, n_ctx - t0);
-    const int n_blk = (n_tok + kAttnBlk - 1) / kAttnBlk;
-    const int gq = a.Hq / a.Hkv;
-    const int32_t *bt = a.kv.block_table + (size_t)r * a.kv.max_pages;
+struct AttnSmem {
+    static constexpr int ROWB = DH * 2 + 16;                     // padded row: conflict-free fragment loads
+    static constexpr int QB = 8 * DH * 4;                        // the group's query vectors (fp32)
+    static constexpr int STAGE = 2 * kAttnBlk * ROWB + QB;       // K block, V block, queries (first block of an item)
+    static constexpr int MERGE = 4 * 8 * (DH + 2) * 4;
+    static constexpr int TOTAL = kAttnStages * STAGE + MERGE + (kBatchRows + 1) * 4 + kBatchRows * 4 + (2 * kAttnStages + 1) * 8;
+};
 
-    // ---- K/V copies: thread copies 16-byte pieces; a 64-token block of K or V is 64 x DH*2 bytes
-    // (all addresses of a block are formed before the first copy is issued, each in registers of its own)
-    auto issue = [&](int blk) {
-        unsigned char *st = smem + (size_t)(blk % kAttnStages) * STAGE;
-        constexpr int PIECES = DH / 8;                      // 16-byte pieces per row
-        constexpr int NIT = kAttnBlk * PIECES / kAttnThreads;
-        constexpr int TSTEP = kAttnThreads / PIECES;        // tokens between a thread's consecutive pieces
-        const int pc = tid % PIECES, tl = tid / PIECES;
+template <int DH>
+__global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArgs a) {
+    using L = AttnSmem<DH>;
+    constexpr int ROWB = L::ROWB, STAGE = L::STAGE;
+    extern __shared__ __align__(16) unsigned char smem[];
+    float *mo = reinterpret_cast<float *>(smem + kAttnStages * STAGE);                    // [4][8][DH + 2]
+    // 8-byte barriers first (STAGE and MERGE are multiples of 16), then the 4-byte tables
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + kAttnStages * STAGE + L::MERGE);  // [stages] copies landed
+    uint64_t *empty = full + kAttnStages;                                                  // [stages] stage consumed
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(empty + kAttnStages);
+    int *prefix = reinterpret_cast<int *>(empty + kAttnStages + 1);                        // [B + 1] chunks before sequence r
+    int *nctx = prefix + kBatchRows + 1;
+    const bool producer = threadIdx.x >= kAttnThreads;
+    const int tid = threadIdx.x & (kAttnThreads - 1), warp = tid >> 5, lane = tid & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kAttnStages; ++s) { mbar_init(&full[s], kAttnThreads); mbar_init(&empty[s], kAttnThreads); }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    // a wait that gives up after two seconds (or when another thread has), so a logic error cannot hang the device
+    auto wait = [&](uint64_t *bar, uint32_t parity) -> bool {
+        if (mbar_try_wait(bar, parity)) return true;
+        const unsigned long long t_begin = global_timer_ns();
+        uint32_t polls = 0;
+        while (!mbar_try_wait(bar, parity)) {
+            if ((++polls & 63u) == 0) {
+                if (*abort_flag) return false;
+                if (global_timer_ns() - t_begin > kAttnWaitNs) { *abort_flag = 1u; return false; }
+            }
+        }
+        return true;
+    };
+    const int gq = a.Hq / a.Hkv;
+    const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
+    if (threadIdx.x < a.B) nctx[threadIdx.x] = min(a.kv.seq_lens[threadIdx.x] + a.step, max_tokens - 1) + 1;     // visible positions 0 .. n-1
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        for (int r = 0; r < a.B; ++r) { prefix[r] = acc; acc += (nctx[r] + kBatchAttnChunk - 1) / kBatchAttnChunk; }
+        prefix[a.B] = acc;
+    }
+    __syncthreads();
+    const int n_items = prefix[a.B] * a.Hkv;
+
+    auto load_item = [&](AttnItem &it, int item) {
+        const int cidx = item / a.Hkv;
+        it.kvh = item - cidx * a.Hkv;
+        int r = 0;
+        while (prefix[r + 1] <= cidx) ++r;
+        it.r = r;
+        it.chunk = cidx - prefix[r];
+        it.t0 = it.chunk * kBatchAttnChunk;
+        it.n_ctx = nctx[r];
+        it.n_blk = (min(kBatchAttnChunk, it.n_ctx - it.t0) + kAttnBlk - 1) / kAttnBlk;
+        it.bt = a.kv.block_table + (size_t)r * a.kv.max_pages;
+    };
+
+    if (producer) {
+    // ---- copy warps: block fb of item fc goes into stage fi % kAttnStages once its previous reader is done.
+    // The block-table entries of a block are loaded one block ahead, so their latency is off the issue path.
+    constexpr int PIECES = DH / 8;                      // 16-byte pieces per row
+    constexpr int NIT = kAttnBlk * PIECES / kAttnThreads;
+    constexpr int TSTEP = kAttnThreads / PIECES;        // tokens between a thread's consecutive pieces
+    const int pc = tid % PIECES, tl = tid / PIECES;
+    auto load_pages = [&](const AttnItem &it_, int blk, int (&pg)[NIT]) {
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            int pos = it_.t0 + blk * kAttnBlk + tl + it * TSTEP;
+            if (pos >= it_.n_ctx) pos = it_.n_ctx - 1;
+            pg[it] = it_.bt[a.page_shift >= 0 ? pos >> a.page_shift : pos / a.page];
+        }
+    };
+    AttnItem fc, fn;
+    int f_item = blockIdx.x, fb = 0, fi = 0;
+    int pg_cur[NIT], pg_next[NIT];
+    if (f_item < n_items) { load_item(fc, f_item); load_pages(fc, 0, pg_cur); }
+    while (f_item < n_items) {
+        // where the next block is, and its block-table entries
+        int n_item = f_item, nb = fb + 1;
+        fn = fc;
+        if (nb == fc.n_blk) {
+            nb = 0;
+            n_item += gridDim.x;
+            if (n_item < n_items) load_item(fn, n_item);
+        }
+        if (n_item < n_items) load_pages(fn, nb, pg_next);
+        const int stage = fi % kAttnStages;
+        if (!wait(&empty[stage], ((fi / kAttnStages) & 1) ^ 1)) break;
+        unsigned char *st = smem + (size_t)stage * STAGE;
         size_t off[NIT];
         uint32_t ok[NIT];
 #pragma unroll
         for (int it = 0; it < NIT; ++it) {
-            int pos = t0 + blk * kAttnBlk + tl + it * TSTEP;
-            ok[it] = pos < n_ctx ? 16u : 0u;
-            if (pos >= n_ctx) pos = n_ctx - 1;
-            int page = bt[pos / a.page];
+            int pos = fc.t0 + fb * kAttnBlk + tl + it * TSTEP;
+            ok[it] = pos < fc.n_ctx ? 16u : 0u;
+            if (pos >= fc.n_ctx) pos = fc.n_ctx - 1;
+            const int pgi = a.page_shift >= 0 ? pos >> a.page_shift : pos / a.page;
+            const int in_page = pos - pgi * a.page;
+            int page = pg_cur[it];
             if ((unsigned)page >= (unsigned)a.kv.num_pages) { atomicOr(a.status, kDevBadPage); page = 0; }
-            off[it] = (((size_t)page * a.Hkv + kvh) * a.page + (pos % a.page)) * DH + pc * 8;
+            off[it] = (((size_t)page * a.Hkv + fc.kvh) * a.page + in_page) * DH + pc * 8;
         }
         const uint32_t d0 = smem_u32(st + tl * ROWB + pc * 16);
 #pragma unroll
@@ -291,58 +376,72 @@ __global__ void __launch_bounds__(kAttnThreads) attn_chunk_kernel(const AttnArgs
             cp_async16_off<0>(d0 + it * TSTEP * ROWB, a.kv.k_pages + off[it], ok[it]);
             cp_async16_off<0>(d0 + kAttnBlk * ROWB + it * TSTEP * ROWB, a.kv.v_pages + off[it], ok[it]);
         }
-        cp_async_commit();
-    };
-    issue(0);
-    if (n_blk > 1) issue(1); else cp_async_commit();
-
-    // ---- query fragments: A rows 0-7 = hi parts of heads 0..gq-1, rows 8-15 = lo parts
-    const int hrow = lane >> 2, kq = (lane & 3) * 2;
-    const float scale = rsqrtf((float)DH);
-    uint32_t qa[DH / 16][4];
-    {
-        const float *qh = a.q + ((size_t)r * a.Hq + (size_t)kvh * gq + hrow) * DH;
-#pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks) {
-            float v0 = 0.f, v1 = 0.f, v2 = 0.f, v3 = 0.f;
-            if (hrow < gq) {
-                v0 = qh[ks * 16 + kq] * scale; v1 = qh[ks * 16 + kq + 1] * scale;
-                v2 = qh[ks * 16 + kq + 8] * scale; v3 = qh[ks * 16 + kq + 9] * scale;
-            }
-            uint16_t h0, l0, h1, l1, h2, l2, h3, l3;
-            split_bf16(v0, h0, l0); split_bf16(v1, h1, l1); split_bf16(v2, h2, l2); split_bf16(v3, h3, l3);
-            qa[ks][0] = (uint32_t)h0 | ((uint32_t)h1 << 16);      // row hrow,     k = kq, kq+1
-            qa[ks][1] = (uint32_t)l0 | ((uint32_t)l1 << 16);      // row hrow + 8
-            qa[ks][2] = (uint32_t)h2 | ((uint32_t)h3 << 16);      // row hrow,     k = kq+8, kq+9
-            qa[ks][3] = (uint32_t)l2 | ((uint32_t)l3 << 16);
+        if (fb == 0) {     // the item's query vectors ride with its first block
+            const float *qsrc = a.q + ((size_t)fc.r * a.Hq + (size_t)fc.kvh * gq) * DH;
+            for (int i = tid; i < gq * DH / 4; i += kAttnThreads)
+                cp_async16_off<0>(smem_u32(st + 2 * kAttnBlk * ROWB + i * 16), qsrc + i * 4, 16u);
         }
+        cp_async_arrive(&full[stage]);      // this thread's arrival fires when its copies above have landed
+        ++fi;
+        fc = fn; f_item = n_item; fb = nb;
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) pg_cur[it] = pg_next[it];
     }
-    float m_run = -INFINITY, l_run = 0.f;       // of head hrow, this warp's tokens (replicated on the 4 lanes of a row)
-    float o[DH / 8][2];                          // o[nt][j]: head hrow, dim nt*8 + kq + j
-#pragma unroll
-    for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = 0.f;
+    cp_async_wait_all();
+    } else {
 
-    for (int blk = 0; blk < n_blk; ++blk) {
-        if (blk + 2 < n_blk) issue(blk + 2); else cp_async_commit();
-        cp_async_wait_group<2>();
-        __syncthreads();
-        const unsigned char *sk = smem + (size_t)(blk % kAttnStages) * STAGE;
+    // ---- compute side
+    const int hrow = lane >> 2, kq = (lane & 3) * 2;
+    const float scale = rsqrtf((float)DH) * 1.4426950408889634f;    // scores in units of log2(e): probabilities by exp2
+    AttnItem cc;
+    int c_item = blockIdx.x, cb = 0, ci = 0;
+    if (c_item < n_items) load_item(cc, c_item);
+    uint32_t qa[DH / 16][4];
+    float m_run = -INFINITY, l_run = 0.f;       // of head hrow, this warp's tokens (replicated on the 4 lanes of a row)
+    float o[DH / 8][4];                          // MMA accumulators: [0],[1] the hi-part products, [2],[3] the lo-part ones
+    while (c_item < n_items) {
+        const int stage = ci % kAttnStages;
+        // the 128 compute threads agree on the outcome of the wait before any of them moves on
+        if (epi_any(!wait(&full[stage], (ci / kAttnStages) & 1))) break;
+        const unsigned char *sk = smem + (size_t)stage * STAGE;
         const unsigned char *sv = sk + kAttnBlk * ROWB;
-        const int tw = warp * 16;                              // this warp's tokens inside the block
-        const int tbase = t0 + blk * kAttnBlk + tw;
-        if (tbase < n_ctx) {
-            // scores: two n-tiles of 8 tokens
-            float s[2][4];
+        if (cb == 0) {
+            // query fragments: A rows 0-7 = hi parts of heads 0..gq-1, rows 8-15 = lo parts
+            const float *qh = reinterpret_cast<const float *>(sv + kAttnBlk * ROWB) + hrow * DH;
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt) {
-                s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-                const unsigned char *krow = sk + (size_t)(tw + nt * 8 + hrow) * ROWB;     // B column n = token lane/4
-#pragma unroll
-                for (int ks = 0; ks < DH / 16; ++ks) {
-                    const uint32_t b0 = *reinterpret_cast<const uint32_t *>(krow + (ks * 16 + kq) * 2);
-                    const uint32_t b1 = *reinterpret_cast<const uint32_t *>(krow + (ks * 16 + kq + 8) * 2);
-                    mma_bf16(s[nt], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+            for (int ks = 0; ks < DH / 16; ++ks) {
+                float v0 = 0.f, v1 = 0.f, v2 = 0.f, v3 = 0.f;
+                if (hrow < gq) {
+                    const float2 lo2 = *reinterpret_cast<const float2 *>(qh + ks * 16 + kq);
+                    const float2 hi2 = *reinterpret_cast<const float2 *>(qh + ks * 16 + kq + 8);
+                    v0 = lo2.x * scale; v1 = lo2.y * scale; v2 = hi2.x * scale; v3 = hi2.y * scale;
                 }
+                uint16_t h0, l0, h1, l1, h2, l2, h3, l3;
+                split_bf16(v0, h0, l0); split_bf16(v1, h1, l1); split_bf16(v2, h2, l2); split_bf16(v3, h3, l3);
+                qa[ks][0] = (uint32_t)h0 | ((uint32_t)h1 << 16);      // row hrow,     k = kq, kq+1
+                qa[ks][1] = (uint32_t)l0 | ((uint32_t)l1 << 16);      // row hrow + 8
+                qa[ks][2] = (uint32_t)h2 | ((uint32_t)h3 << 16);      // row hrow,     k = kq+8, kq+9
+                qa[ks][3] = (uint32_t)l2 | ((uint32_t)l3 << 16);
+            }
+            m_run = -INFINITY; l_run = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+        }
+        const int tw = warp * 16;                              // this warp's tokens inside the block
+        const int tbase = cc.t0 + cb * kAttnBlk + tw;
+        if (tbase < cc.n_ctx) {
+            // scores: two n-tiles of 8 tokens; one ldmatrix.x4 brings both tiles' K fragments of a 16-wide slice
+            float s[2][4];
+            s[0][0] = s[0][1] = s[0][2] = s[0][3] = 0.f;
+            s[1][0] = s[1][1] = s[1][2] = s[1][3] = 0.f;
+            const uint32_t kaddr = smem_u32(sk) + (uint32_t)((tw + (lane & 7) + ((lane >> 4) << 3)) * ROWB + ((lane >> 3) & 1) * 16);
+#pragma unroll
+            for (int ks = 0; ks < DH / 16; ++ks) {
+                uint32_t b00, b01, b10, b11;
+                asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(b00), "=r"(b01), "=r"(b10), "=r"(b11) : "r"(kaddr + ks * 32));
+                mma_bf16(s[0], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b00, b01);
+                mma_bf16(s[1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b10, b11);
             }
             // thread holds, for head hrow: tokens tw + nt*8 + kq + {0,1}: hi part in [0],[1], lo part in [2],[3]
             float sc[4];
@@ -352,20 +451,20 @@ __global__ void __launch_bounds__(kAttnThreads) attn_chunk_kernel(const AttnArgs
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
                     float v = s[nt][j] + s[nt][j + 2];
-                    if (tbase + nt * 8 + kq + j >= n_ctx) v = -INFINITY;
+                    if (tbase + nt * 8 + kq + j >= cc.n_ctx) v = -INFINITY;
                     sc[nt * 2 + j] = v;
                     mx = fmaxf(mx, v);
                 }
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
             const float m_new = fmaxf(m_run, mx);                 // finite: the warp's first token is visible
-            const float corr = expf(m_run - m_new);               // 0 on the first block (m_run = -inf)
+            const float corr = exp2f(m_run - m_new);              // 0 on the item's first block (m_run = -inf)
             float psum = 0.f;
             uint32_t pa[4];
             {
                 float pr[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) { pr[i] = expf(sc[i] - m_new); psum += pr[i]; }
+                for (int i = 0; i < 4; ++i) { pr[i] = exp2f(sc[i] - m_new); psum += pr[i]; }
                 uint16_t h0, l0, h1, l1, h2, l2, h3, l3;
                 split_bf16(pr[0], h0, l0); split_bf16(pr[1], h1, l1); split_bf16(pr[2], h2, l2); split_bf16(pr[3], h3, l3);
                 pa[0] = (uint32_t)h0 | ((uint32_t)h1 << 16);      // row hrow,   tokens kq, kq+1
@@ -377,47 +476,55 @@ __global__ void __launch_bounds__(kAttnThreads) attn_chunk_kernel(const AttnArgs
             psum += __shfl_xor_sync(0xffffffffu, psum, 2);
             l_run = l_run * corr + psum;
             m_run = m_new;
-            // weighted sum: B[k = token][n = dim] read with a transposing ldmatrix from V[token][dim]
+            // weighted sum, accumulated in the MMA: rescale the running output only when some row's maximum moved
+            if (__any_sync(0xffffffffu, corr != 1.0f)) {
 #pragma unroll
-            for (int nt = 0; nt < DH / 8; ++nt) {
-                uint32_t b0, b1;
-                const unsigned char *vrow = sv + (size_t)(tw + (lane & 15)) * ROWB + nt * 16;
-                asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];"
-                             : "=r"(b0), "=r"(b1) : "r"(smem_u32(vrow)));
-                float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                mma_bf16(acc, pa[0], pa[1], pa[2], pa[3], b0, b1);
-                o[nt][0] = o[nt][0] * corr + acc[0] + acc[2];
-                o[nt][1] = o[nt][1] * corr + acc[1] + acc[3];
+                for (int nt = 0; nt < DH / 8; ++nt) { o[nt][0] *= corr; o[nt][1] *= corr; o[nt][2] *= corr; o[nt][3] *= corr; }
+            }
+            // B[k = token][n = dim] read with a transposing ldmatrix from V[token][dim], two n-tiles per load
+            const uint32_t vaddr = smem_u32(sv) + (uint32_t)((tw + (lane & 7) + ((lane >> 3) & 1) * 8) * ROWB + (lane >> 4) * 16);
+#pragma unroll
+            for (int nt = 0; nt < DH / 8; nt += 2) {
+                uint32_t b00, b01, b10, b11;
+                asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(b00), "=r"(b01), "=r"(b10), "=r"(b11) : "r"(vaddr + nt * 16));
+                mma_bf16(o[nt], pa[0], pa[1], pa[2], pa[3], b00, b01);
+                mma_bf16(o[nt + 1], pa[0], pa[1], pa[2], pa[3], b10, b11);
             }
         }
-        __syncthreads();
-    }
-    cp_async_wait_group<0>();
-    // ---- merge the four warps (fixed order) and write the chunk's partial
-    float *mo = reinterpret_cast<float *>(smem);                 // [4][8][DH + 2]
-    __syncthreads();
-    {
-        float *dst = mo + ((size_t)warp * 8 + hrow) * (DH + 2);
+        mbar_arrive(&empty[stage]);        // this thread has read all it needs from the stage
+        ++ci;
+        if (++cb == cc.n_blk) {
+            // ---- end of the item: merge the four warps (fixed order) and write the chunk's partial
+            float *dst = mo + ((size_t)warp * 8 + hrow) * (DH + 2);
 #pragma unroll
-        for (int nt = 0; nt < DH / 8; ++nt) { dst[nt * 8 + kq] = o[nt][0]; dst[nt * 8 + kq + 1] = o[nt][1]; }
-        if ((lane & 3) == 0) { dst[DH] = m_run; dst[DH + 1] = l_run; }
+            for (int nt = 0; nt < DH / 8; ++nt) { dst[nt * 8 + kq] = o[nt][0] + o[nt][2]; dst[nt * 8 + kq + 1] = o[nt][1] + o[nt][3]; }
+            if ((lane & 3) == 0) { dst[DH] = m_run; dst[DH + 1] = l_run; }
+            bar_sync(1, kAttnThreads);
+            for (int i = tid; i < gq * DH; i += kAttnThreads) {
+                const int h = i / DH, j = i - h * DH;
+                float m = -INFINITY;
+                for (int w = 0; w < 4; ++w) m = fmaxf(m, mo[((size_t)w * 8 + h) * (DH + 2) + DH]);
+                float acc = 0.f, l = 0.f;
+                for (int w = 0; w < 4; ++w) {
+                    const float *src = mo + ((size_t)w * 8 + h) * (DH + 2);
+                    const float f = src[DH] == -INFINITY ? 0.f : exp2f(src[DH] - m);
+                    acc += src[j] * f;
+                    l += src[DH + 1] * f;
+                }
+                float *out = a.att_part + (((size_t)cc.r * a.Hq + (size_t)cc.kvh * gq + h) * a.max_chunks + cc.chunk) * (DH + 2);
+                out[j] = acc;
+                if (j == 0) { out[DH] = m * 0.6931471805599453f; out[DH + 1] = l; }     // the chunk maximum in natural-log units
+            }
+            bar_sync(1, kAttnThreads);     // merge buffer free for the next item
+            cb = 0;
+            c_item += gridDim.x;
+            if (c_item < n_items) load_item(cc, c_item);
+        }
+    }
     }
     __syncthreads();
-    for (int i = tid; i < gq * DH; i += kAttnThreads) {
-        const int h = i / DH, j = i - h * DH;
-        float m = -INFINITY;
-        for (int w = 0; w < 4; ++w) m = fmaxf(m, mo[((size_t)w * 8 + h) * (DH + 2) + DH]);
-        float acc = 0.f, l = 0.f;
-        for (int w = 0; w < 4; ++w) {
-            const float *src = mo + ((size_t)w * 8 + h) * (DH + 2);
-            const float f = src[DH] == -INFINITY ? 0.f : expf(src[DH] - m);
-            acc += src[j] * f;
-            l += src[DH + 1] * f;
-        }
-        float *out = a.att_part + (((size_t)r * a.Hq + (size_t)kvh * gq + h) * a.max_chunks + chunk) * (DH + 2);
-        out[j] = acc;
-        if (j == 0) { out[DH] = m; out[DH + 1] = l; }
-    }
+    if (threadIdx.x == 0 && *abort_flag) atomicOr(a.status, 0x8u);
 }
 
 // ---- combine a head's chunk partials in ascending order; write the O-projection's operand.
@@ -611,10 +718,12 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
         return (int)cudaGetLastError();
     };
     int rc = 0;
-    const size_t attn_smem = (size_t)kAttnStages * 2 * kAttnBlk * (sh.dh * 2 + 16);
-    if (sh.dh == 128) e = cudaFuncSetAttribute(attn_chunk_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
-    else e = cudaFuncSetAttribute(attn_chunk_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
+    const size_t attn_smem = sh.dh == 128 ? AttnSmem<128>::TOTAL : AttnSmem<64>::TOTAL;
+    if (sh.dh == 128) e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
+    else e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
     if (e != cudaSuccess) return (int)e;
+    int page_shift = -1;
+    for (int b = 0; b < 31; ++b) if ((1 << b) == sh.page) page_shift = b;
 
     for (int step = 0; step <= K; ++step) {
         PrologueArgs pa{};
@@ -651,9 +760,9 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
             AttnArgs a{};
             a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.dh = sh.dh; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = step;
             a.max_chunks = ws.max_chunks; a.q = ws.q; a.kv = c.kv; a.att_part = ws.att_part; a.status = ws.status;
-            const dim3 grid(ws.max_chunks, sh.Hkv, B);
-            if (sh.dh == 128) attn_chunk_kernel<128><<<grid, kAttnThreads, attn_smem, st>>>(a);
-            else attn_chunk_kernel<64><<<grid, kAttnThreads, attn_smem, st>>>(a);
+            a.page_shift = page_shift; a.B = B;
+            if (sh.dh == 128) attn_kernel<128><<<c.n_sm, 2 * kAttnThreads, attn_smem, st>>>(a);
+            else attn_kernel<64><<<c.n_sm, 2 * kAttnThreads, attn_smem, st>>>(a);
             ++*launches;
             if ((rc = (int)cudaGetLastError())) return rc;
             MergeArgs m{};
