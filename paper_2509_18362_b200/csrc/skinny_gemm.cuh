@@ -120,7 +120,13 @@ __device__ __forceinline__ void produce_kblock(const GemmArgs &g, const GemmProd
     const bool kvalid = (kb + J) * kGemmBK + pr.c * 8 < g.K;
     const uint32_t dst = pr.dst0 + (uint32_t)pr.stage * pr.stage_bytes + (uint32_t)J * pr.kblock_bytes;
     const uint32_t dx = dst + 16384;
-    if (kvalid) {
+    if (kvalid && (aok[0] & aok[1] & aok[2] & aok[3]) != 0u) {      // the common case: plain 16-byte copies
+#pragma unroll
+        for (int i = 0; i < 4; ++i) cp_async16_full<J * 128>(dst + i * 4096, ap[i]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (xok[i]) cp_async16_full<J * 128>(dx + i * 4096, xp[i]);
+    } else if (kvalid) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) cp_async16_off<J * 128>(dst + i * 4096, ap[i], aok[i]);
 #pragma unroll

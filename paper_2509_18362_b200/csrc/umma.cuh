@@ -84,6 +84,11 @@ __device__ __forceinline__ void cp_async16_off(uint32_t dst_smem, const void *sr
     asm volatile("cp.async.cg.shared.global [%0], [%1+%2], 16, %3;" ::"r"(dst_smem), "l"(src), "n"(OFF), "r"(src_bytes)
                  : "memory");
 }
+// The same copy without the source-size operand (always 16 bytes).
+template <int OFF>
+__device__ __forceinline__ void cp_async16_full(uint32_t dst_smem, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1+%2], 16;" ::"r"(dst_smem), "l"(src), "n"(OFF) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait_group() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
