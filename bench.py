@@ -121,7 +121,7 @@ class ClockSampler:
 # DRAM traffic of one mega_kernel launch on the default workload, from the ncu capture summarised in
 # profiles/mega_kernel_7b_batch1_ncu.md (dram__bytes_read.sum + dram__bytes_write.sum). It is only
 # reported while the kernel sources are the ones the counters were taken from.
-NCU_TRAFFIC = {"bytes_per_launch": 2270662000 + 7515904, "sources_sha256": "2b761a5f5efaed197cc413cc7643acb0e54af2e860f4d6aed152b630f9d5da5e"}
+NCU_TRAFFIC = {"bytes_per_launch": 2270711040 + 5550080, "sources_sha256": "c9f7b65262f333ce2e10af16a8bd44d1fca9651f0a339a8002c53df6f0c8089a"}
 KERNEL_SOURCES = ["megakernel.cu", "mega.cuh", "ptx.cuh", "api.cu"]
 
 
@@ -347,6 +347,12 @@ def run_ours(a):
     bytes_launch = sum(algorithmic_bytes_per_draft_step(s, B, N, ctx_lens, k) for k in range(K))
     peak, peak_kind = load_peaks()
     achieved = bytes_launch / (draft_ms * 1e-3) / 1e9
+    # which path the draft call took: one persistent launch per group of sequences, or (more sequences than one
+    # launch takes) the batched path, a sequence of tensor-core GEMM and row-wise kernels per step
+    per_call = (launches / a.steps) - 1                      # kernels of one fastmtp_draft call (verify is the other one)
+    kernel_name = ("mega_kernel (fastmtp_draft, K steps per launch)" if per_call <= 2 else
+                   "batched path: all %d kernels of one fastmtp_draft call (skinny_gemm_kernel x %d, attn_kernel, row-wise)"
+                   % (per_call, 6 * K))
     out = {
         "metric": "draft_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": a.steps,
         "warmup": max(a.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -361,7 +367,7 @@ def run_ours(a):
                 "h2d_bytes_per_step": int(hh.numel() * 2 + htok.numel() * 4 + hlog.numel() * 2 + hdv.numel() * 4),
                 "d2h_bytes_per_step": int(hout.numel() * 4 + hacc.numel() * 4 + hbon.numel() * 4 + 8),
                 "steps": n_e2e},
-        "roofline": {"bound": "hbm", "kernel": "mega_kernel (fastmtp_draft, K steps per launch)",
+        "roofline": {"bound": "hbm", "kernel": kernel_name,
                      "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / 8000.0,
                      "algorithmic_bytes_per_launch": int(bytes_launch), "launch_ms": draft_ms,
@@ -379,7 +385,7 @@ def run_ours(a):
 
 
 def run_sweep(a):
-    """Subset size {8192 .. full} (Zipf-weighted draws) x batch {1, 4, 16, 32} x K {1, 3, 5} on the 7B-class head at
+    """Subset size {8192 .. full} (Zipf-weighted draws) x batch {1, 4, 16, 32, 64} x K {1, 3, 5} on the 7B-class head at
     context 2048: device-timed draft calls only, one JSON line per point."""
     import torch
     import __graft_entry__ as G
@@ -393,7 +399,7 @@ def run_sweep(a):
     w = Bd.mtp_w(dW)
     peak, peak_kind = load_peaks()
     sizes = [8192, 16384, 32768, 65536, s.vocab] if a.shape == "7b" else [256, 1024, s.vocab]
-    for B in (1, 4, 16, 32):
+    for B in (1, 4, 16, 32, 64):
         ctx_lens = [a.ctx] * B
         kv = I.paged_kv(s, ctx_lens, 6, a.seed + 1)
         dkv = Bd.to_device(kv)
