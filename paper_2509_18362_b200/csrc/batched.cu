@@ -73,6 +73,8 @@ __device__ __forceinline__ void load_f32x8(const float *p, float (&v)[8]) {
 
 // Each thread owns eight consecutive columns per pass (d % 64 == 0), so every load and store is 16 bytes.
 __global__ void __launch_bounds__(kRowThreads) prologue_kernel(const PrologueArgs a) {
+    chain_release();
+    chain_wait();
     __shared__ float red[32];
     __shared__ int s_tok;
     const int r = blockIdx.x, tid = threadIdx.x;
@@ -138,6 +140,8 @@ struct PostArgs {
 };
 
 __global__ void __launch_bounds__(kRowThreads) post_kernel(const PostArgs a) {
+    chain_release();
+    chain_wait();
     __shared__ float red[32];
     const int r = blockIdx.x, tid = threadIdx.x;
     float ss = 0.f;
@@ -197,6 +201,8 @@ struct QkvArgs {
 };
 
 __global__ void qkv_finish_kernel(const QkvArgs a) {
+    chain_release();
+    chain_wait();
     const int head = blockIdx.x, r = blockIdx.y, e = threadIdx.x, half = a.dh >> 1;
     const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
     const int pos_true = a.kv.seq_lens[r] + a.step;
@@ -270,6 +276,8 @@ struct AttnSmem {
 
 template <int DH>
 __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArgs a) {
+    chain_release();
+    chain_wait();
     using L = AttnSmem<DH>;
     constexpr int ROWB = L::ROWB, STAGE = L::STAGE;
     extern __shared__ __align__(16) unsigned char smem[];
@@ -536,6 +544,8 @@ struct MergeArgs {
 };
 
 __global__ void attn_merge_kernel(const MergeArgs a) {
+    chain_release();
+    chain_wait();
     __shared__ float red[8];
     const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x;
     const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
@@ -583,6 +593,8 @@ __global__ void attn_merge_kernel(const MergeArgs a) {
 // memory pages (an unsorted subset spreads them over the whole matrix and the address translation
 // misses cost ~25 % of the head's stream rate). Membership bitmap, then a one-block compaction.
 __global__ void ids_mark_kernel(const int32_t *ids, int N, int V, uint32_t *bitmap, uint32_t *status) {
+    chain_release();
+    chain_wait();
     for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < N; j += gridDim.x * blockDim.x) {
         int id = ids[j];
         if ((unsigned)id >= (unsigned)V) { atomicOr(status, kDevBadToken); id = 0; }
@@ -591,6 +603,8 @@ __global__ void ids_mark_kernel(const int32_t *ids, int N, int V, uint32_t *bitm
 }
 
 __global__ void __launch_bounds__(1024) ids_compact_kernel(const uint32_t *bitmap, int n_words, int32_t *sorted, int N) {
+    chain_release();
+    chain_wait();
     __shared__ int warp_tot[32];
     __shared__ int s_total, s_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -690,10 +704,11 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
         const int n_words = (sh.V + 31) / 32;
         e = cudaMemsetAsync(ws.id_bitmap, 0, (size_t)n_words * 4, st);
         if (e != cudaSuccess) return (int)e;
-        ids_mark_kernel<<<(c.N + 255) / 256 < 1024 ? (c.N + 255) / 256 : 1024, 256, 0, st>>>(c.ids, c.N, sh.V, ws.id_bitmap, ws.status);
-        ids_compact_kernel<<<1, 1024, 0, st>>>(ws.id_bitmap, n_words, ws.sorted_ids, c.N);
+        e = launch_chained(ids_mark_kernel, dim3((c.N + 255) / 256 < 1024 ? (c.N + 255) / 256 : 1024), dim3(256), 0, st, c.ids, c.N, sh.V,
+                           ws.id_bitmap, ws.status);
+        if (e == cudaSuccess) e = launch_chained(ids_compact_kernel, dim3(1), dim3(1024), 0, st, ws.id_bitmap, n_words, ws.sorted_ids, c.N);
         *launches += 2;
-        if ((e = cudaGetLastError()) != cudaSuccess) return (int)e;
+        if (e != cudaSuccess) return (int)e;
         head_ids = ws.sorted_ids;
     }
 
@@ -713,9 +728,8 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
         a.d = d; a.splits = splits; a.rows = B; a.ldp = ws.ldp; a.ld = ws.ld0; a.residual = residual; a.final = final;
         a.K = K; a.step = step; a.eps = sh.eps; a.partial = ws.partial; a.x = ws.x; a.hout = ws.hout;
         a.out_h = c.out_h; a.gain = gain; a.xop = ws.xop0;
-        post_kernel<<<B, kRowThreads, 0, st>>>(a);
         ++*launches;
-        return (int)cudaGetLastError();
+        return (int)launch_chained(post_kernel, dim3(B), dim3(kRowThreads), 0, st, a);
     };
     int rc = 0;
     const size_t attn_smem = sh.dh == 128 ? AttnSmem<128>::TOTAL : AttnSmem<64>::TOTAL;
@@ -732,9 +746,8 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
         pa.keys_prev = step > 0 ? ws.keys + (size_t)(step - 1) * kBatchRows : nullptr;
         pa.out_drafts = c.out_drafts; pa.embed = c.embed; pa.g_h = c.g_hnorm; pa.g_e = c.g_enorm;
         pa.xop = ws.xop0; pa.status = ws.status; pa.user_status = c.user_status;
-        prologue_kernel<<<B, kRowThreads, 0, st>>>(pa);
         ++*launches;
-        if ((rc = (int)cudaGetLastError())) return rc;
+        if ((rc = (int)launch_chained(prologue_kernel, dim3(B), dim3(kRowThreads), 0, st, pa))) return rc;
         if (step == K) break;
 
         GemmArgs g{};
@@ -752,25 +765,23 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
             a.qdim = qdim; a.kvdim = kvdim; a.dh = sh.dh; a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.splits = g.splits; a.rows = B;
             a.ldp = ws.ldp; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = step; a.partial = ws.partial; a.q = ws.q;
             a.kv = c.kv; a.rope_cos = c.rope_cos; a.rope_sin = c.rope_sin; a.status = ws.status;
-            qkv_finish_kernel<<<dim3(sh.Hq + 2 * sh.Hkv, B), sh.dh / 2, 0, st>>>(a);
             ++*launches;
-            if ((rc = (int)cudaGetLastError())) return rc;
+            if ((rc = (int)launch_chained(qkv_finish_kernel, dim3(sh.Hq + 2 * sh.Hkv, B), dim3(sh.dh / 2), 0, st, a))) return rc;
         }
         {
             AttnArgs a{};
             a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.dh = sh.dh; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = step;
             a.max_chunks = ws.max_chunks; a.q = ws.q; a.kv = c.kv; a.att_part = ws.att_part; a.status = ws.status;
             a.page_shift = page_shift; a.B = B;
-            if (sh.dh == 128) attn_kernel<128><<<c.n_sm, 2 * kAttnThreads, attn_smem, st>>>(a);
-            else attn_kernel<64><<<c.n_sm, 2 * kAttnThreads, attn_smem, st>>>(a);
             ++*launches;
-            if ((rc = (int)cudaGetLastError())) return rc;
+            if (sh.dh == 128) rc = (int)launch_chained(attn_kernel<128>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
+            else rc = (int)launch_chained(attn_kernel<64>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
+            if (rc) return rc;
             MergeArgs m{};
             m.Hq = sh.Hq; m.dh = sh.dh; m.page = sh.page; m.max_ctx = sh.max_ctx; m.step = step; m.max_chunks = ws.max_chunks;
             m.ld = ws.ld0; m.kv = c.kv; m.att_part = ws.att_part; m.xop = ws.xop0;
-            attn_merge_kernel<<<dim3(sh.Hq, B), sh.dh, 0, st>>>(m);
             ++*launches;
-            if ((rc = (int)cudaGetLastError())) return rc;
+            if ((rc = (int)launch_chained(attn_merge_kernel, dim3(sh.Hq, B), dim3(sh.dh), 0, st, m))) return rc;
         }
         // x += W_o o
         g = GemmArgs{};

@@ -169,6 +169,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
         tmem_relinquish();
         tc_fence_before_sync();
     }
+    chain_release();
+    chain_wait();            // set-up above overlaps the previous kernel's tail; its outputs are read below
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&sm->tmem_base);
@@ -398,8 +400,8 @@ inline int skinny_gemm_launch(GemmArgs g, int n_sm, int smem_optin, cudaStream_t
     if (ka != 1 && ka != 2 && ka != 4) return (int)cudaErrorInvalidConfiguration;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
-    kern<<<grid, kGemmThreads, smem, stream>>>(g);
-    return (int)cudaGetLastError();
+    e = launch_chained(kern, dim3(grid), dim3(kGemmThreads), smem, stream, g);
+    return (int)e;
 }
 
 }  // namespace fmtp
