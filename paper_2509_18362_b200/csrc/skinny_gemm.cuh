@@ -112,7 +112,8 @@ struct GemmProducer {
 // Copies this thread's share of K block kb + J (if it is inside the item) into block J of the
 // current stage. Source addresses are the per-row pointers plus the immediate J * 128 bytes, so
 // all blocks of a stage go out before a pointer register is rewritten.
-template <int J>
+// PART: 1 = the weight rows only, 2 = the activation rows only, 3 = both.
+template <int J, int PART>
 __device__ __forceinline__ void produce_kblock(const GemmArgs &g, const GemmProducer &pr, int kb, int kb1,
                                                const bf16_t *(&ap)[4], const bf16_t *(&xp)[4],
                                                const uint32_t (&aok)[4], const uint32_t (&xok)[4]) {
@@ -121,23 +122,47 @@ __device__ __forceinline__ void produce_kblock(const GemmArgs &g, const GemmProd
     const uint32_t dst = pr.dst0 + (uint32_t)pr.stage * pr.stage_bytes + (uint32_t)J * pr.kblock_bytes;
     const uint32_t dx = dst + 16384;
     if (kvalid && (aok[0] & aok[1] & aok[2] & aok[3]) != 0u) {      // the common case: plain 16-byte copies
+        if (PART & 1) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) cp_async16_full<J * 128>(dst + i * 4096, ap[i]);
+            for (int i = 0; i < 4; ++i) cp_async16_full<J * 128>(dst + i * 4096, ap[i]);
+        }
+        if (PART & 2) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (xok[i]) cp_async16_full<J * 128>(dx + i * 4096, xp[i]);
+            for (int i = 0; i < 4; ++i)
+                if (xok[i]) cp_async16_full<J * 128>(dx + i * 4096, xp[i]);
+        }
     } else if (kvalid) {
+        if (PART & 1) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) cp_async16_off<J * 128>(dst + i * 4096, ap[i], aok[i]);
+            for (int i = 0; i < 4; ++i) cp_async16_off<J * 128>(dst + i * 4096, ap[i], aok[i]);
+        }
+        if (PART & 2) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (xok[i]) cp_async16_off<J * 128>(dx + i * 4096, xp[i], 16u);
+            for (int i = 0; i < 4; ++i)
+                if (xok[i]) cp_async16_off<J * 128>(dx + i * 4096, xp[i], 16u);
+        }
     } else {   // this chunk column lies beyond K: zeros, nothing is read
+        if (PART & 1) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) cp_async16_off<0>(dst + i * 4096, g.a[0], 0u);
+            for (int i = 0; i < 4; ++i) cp_async16_off<0>(dst + i * 4096, g.a[0], 0u);
+        }
+        if (PART & 2) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (xok[i]) cp_async16_off<0>(dx + i * 4096, g.a[0], 0u);
+            for (int i = 0; i < 4; ++i)
+                if (xok[i]) cp_async16_off<0>(dx + i * 4096, g.a[0], 0u);
+        }
+    }
+}
+
+template <int KA, int PART>
+__device__ __forceinline__ void produce_stage(const GemmArgs &g, const GemmProducer &pr, int kb, int kb1,
+                                              const bf16_t *(&ap)[4], const bf16_t *(&xp)[4],
+                                              const uint32_t (&aok)[4], const uint32_t (&xok)[4]) {
+    produce_kblock<0, PART>(g, pr, kb, kb1, ap, xp, aok, xok);
+    if constexpr (KA > 1) produce_kblock<1, PART>(g, pr, kb, kb1, ap, xp, aok, xok);
+    if constexpr (KA > 2) {
+        produce_kblock<2, PART>(g, pr, kb, kb1, ap, xp, aok, xok);
+        produce_kblock<3, PART>(g, pr, kb, kb1, ap, xp, aok, xok);
     }
 }
 
@@ -169,8 +194,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
         tmem_relinquish();
         tc_fence_before_sync();
     }
-    chain_release();
-    chain_wait();            // set-up above overlaps the previous kernel's tail; its outputs are read below
+    chain_release();         // the next kernel of the stream may start its own set-up
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&sm->tmem_base);
@@ -189,13 +213,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
         pr.stage_bytes = stage_bytes; pr.kblock_bytes = kblock_bytes; pr.S = S; pr.c = c;
         pr.stage = 0; pr.phase = 0;
         bool ok_run = true;
-        for (int item = blockIdx.x; item < n_items && ok_run; item += gridDim.x) {
+        const bf16_t *ap[4];
+        const bf16_t *xp[4];
+        uint32_t aok[4], xok[4];
+        int kb0 = 0, kb1 = 0;
+        auto setup_item = [&](int item) {
             const int tile = item / g.splits, split = item - tile * g.splits;
-            const int kb0 = split * g.kb_per_split;
-            int kb1 = kb0 + g.kb_per_split;
+            kb0 = split * g.kb_per_split;
+            kb1 = kb0 + g.kb_per_split;
             if (kb1 > n_kb) kb1 = n_kb;
-            const bf16_t *ap[4];
-            uint32_t aok[4], xok[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int tr = r0 + 32 * i;
@@ -223,7 +249,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
                 }
                 ap[i] = base + (size_t)row * g.lda + (size_t)kb0 * kGemmBK + c * 8;
             }
-            const bf16_t *xp[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 int n = r0 + 32 * i;
@@ -231,24 +256,42 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
                 if (n >= g.NB) n = g.NB - 1;
                 xp[i] = g.x + (size_t)n * g.ldx + (size_t)kb0 * kGemmBK + c * 8;
             }
+        };
+        // The weights (and the row ids, written several kernels ago) do not depend on the predecessor in the
+        // stream: the weight part of the first item's first stages goes out before waiting for it.
+        setup_item(blockIdx.x);
+        int pre = 0;
+        for (int kb = kb0; kb < kb1 && pre < S; kb += KA, ++pre) {
+            pr.stage = pre;
+            produce_stage<KA, 1>(g, pr, kb, kb1, ap, xp, aok, xok);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) ap[i] += KA * kGemmBK;
+        }
+        pr.stage = 0;
+        chain_wait();
+        for (int item = blockIdx.x; item < n_items && ok_run; item += gridDim.x) {
+            if (item != (int)blockIdx.x) setup_item(item);
             for (int kb = kb0; kb < kb1; kb += KA) {
                 if (!gemm_wait(sm, &sm->empty[pr.stage], pr.phase ^ 1u)) { ok_run = false; break; }
-                produce_kblock<0>(g, pr, kb, kb1, ap, xp, aok, xok);
-                if constexpr (KA > 1) produce_kblock<1>(g, pr, kb, kb1, ap, xp, aok, xok);
-                if constexpr (KA > 2) {
-                    produce_kblock<2>(g, pr, kb, kb1, ap, xp, aok, xok);
-                    produce_kblock<3>(g, pr, kb, kb1, ap, xp, aok, xok);
+                if (pre > 0) {      // weight part already in flight: add the activation part
+                    --pre;
+                    produce_stage<KA, 2>(g, pr, kb, kb1, ap, xp, aok, xok);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) xp[i] += KA * kGemmBK;
+                } else {
+                    produce_stage<KA, 3>(g, pr, kb, kb1, ap, xp, aok, xok);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) { ap[i] += KA * kGemmBK; xp[i] += KA * kGemmBK; }
                 }
                 // this thread's arrival on the stage's barrier fires when its copies above have landed
                 cp_async_arrive(&sm->full[pr.stage]);
                 if (++pr.stage == S) { pr.stage = 0; pr.phase ^= 1u; }
-#pragma unroll
-                for (int i = 0; i < 4; ++i) { ap[i] += KA * kGemmBK; xp[i] += KA * kGemmBK; }
             }
         }
         cp_async_wait_all();
     } else if (warp == 4) {
         // ================= MMA issue: one thread
+        chain_wait();
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(g.NB);
             int stage = 0;
@@ -293,6 +336,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
         __syncwarp();
     } else {
         // ================= epilogue: thread = one row of the tile (TMEM lane 32*warp + lane)
+        chain_wait();
         uint32_t tphase[2] = {0, 0};
         int buf = 0;
         for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
