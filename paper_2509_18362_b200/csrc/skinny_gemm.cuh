@@ -7,8 +7,10 @@
 // the high part of activation row r and n = 2r + 1 the low part, so the pair carries an fp32
 // value) is small and re-read from L2 for every tile. One CTA per SM walks a static list of work
 // items (tile, K range). Roles: warps 0-3 epilogue (TMEM -> registers -> global), warp 4 issues
-// the MMAs, warps 5-12 copy A and X into a shared-memory ring with 16-byte cp.async, laid out as
-// the MMA's 128-byte-swizzled K-major tiles (64 K elements wide). A ring stage holds KA such
+// the MMAs, warps 5-12 copy A into a shared-memory ring with 16-byte cp.async, laid out as
+// the MMA's 128-byte-swizzled K-major tiles (64 K elements wide); the X block of a stage comes by
+// one TMA tile copy (same swizzle) through the copy engine, which leaves the load/store path's
+// ~64 GB/s per SM to the weights: with 64 rows the X bytes equal the weight bytes. A ring stage holds KA such
 // 64-wide blocks that are requested back to back, so a weight row is read in pieces of KA x 128
 // contiguous bytes. Accumulators are double buffered in TMEM so the epilogue of one item overlaps
 // the MMAs of the next.
@@ -19,6 +21,7 @@
 // Every wait is time-bounded; on expiry the CTA raises the timeout flag, drains and returns.
 #pragma once
 #include "umma.cuh"
+#include <cuda.h>
 
 namespace fmtp {
 
@@ -101,12 +104,25 @@ __device__ __forceinline__ bool epi_any(bool flag) {
     return out != 0;
 }
 
+// One TMA tile copy global -> shared (2-D tensor map, element coordinates x, y); its bytes are counted on `bar`.
+// x * element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst_smem), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
 // State of one producer thread's walk over the ring.
 struct GemmProducer {
     uint32_t dst0;            // shared address of this thread's chunk in row r0 of stage 0
     int stage_bytes, kblock_bytes, S, c;
     int stage;
     uint32_t phase;
+    bool tma_thread;          // the one producer thread that issues the X tile copies
+    uint32_t dst_x;           // shared address of the X tile in block 0 of stage 0
+    const CUtensorMap *xmap;
+    uint64_t *full;
 };
 
 // Copies this thread's share of K block kb + J (if it is inside the item) into block J of the
@@ -115,60 +131,40 @@ struct GemmProducer {
 // PART: 1 = the weight rows only, 2 = the activation rows only, 3 = both.
 template <int J, int PART>
 __device__ __forceinline__ void produce_kblock(const GemmArgs &g, const GemmProducer &pr, int kb, int kb1,
-                                               const bf16_t *(&ap)[4], const bf16_t *(&xp)[4],
-                                               const uint32_t (&aok)[4], const uint32_t (&xok)[4]) {
+                                               const bf16_t *(&ap)[4], const uint32_t (&aok)[4]) {
     if (kb + J >= kb1) return;
+    if ((PART & 2) && pr.tma_thread)
+        tma_load_2d(pr.dst_x + (uint32_t)pr.stage * pr.stage_bytes + (uint32_t)J * pr.kblock_bytes, pr.xmap, (kb + J) * kGemmBK, 0,
+                    pr.full + pr.stage);
+    if (!(PART & 1)) return;
     const bool kvalid = (kb + J) * kGemmBK + pr.c * 8 < g.K;
     const uint32_t dst = pr.dst0 + (uint32_t)pr.stage * pr.stage_bytes + (uint32_t)J * pr.kblock_bytes;
-    const uint32_t dx = dst + 16384;
     if (kvalid && (aok[0] & aok[1] & aok[2] & aok[3]) != 0u) {      // the common case: plain 16-byte copies
-        if (PART & 1) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) cp_async16_full<J * 128>(dst + i * 4096, ap[i]);
-        }
-        if (PART & 2) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (xok[i]) cp_async16_full<J * 128>(dx + i * 4096, xp[i]);
-        }
+        for (int i = 0; i < 4; ++i) cp_async16_full<J * 128>(dst + i * 4096, ap[i]);
     } else if (kvalid) {
-        if (PART & 1) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) cp_async16_off<J * 128>(dst + i * 4096, ap[i], aok[i]);
-        }
-        if (PART & 2) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (xok[i]) cp_async16_off<J * 128>(dx + i * 4096, xp[i], 16u);
-        }
+        for (int i = 0; i < 4; ++i) cp_async16_off<J * 128>(dst + i * 4096, ap[i], aok[i]);
     } else {   // this chunk column lies beyond K: zeros, nothing is read
-        if (PART & 1) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) cp_async16_off<0>(dst + i * 4096, g.a[0], 0u);
-        }
-        if (PART & 2) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (xok[i]) cp_async16_off<0>(dx + i * 4096, g.a[0], 0u);
-        }
+        for (int i = 0; i < 4; ++i) cp_async16_off<0>(dst + i * 4096, g.a[0], 0u);
     }
 }
 
 template <int KA, int PART>
 __device__ __forceinline__ void produce_stage(const GemmArgs &g, const GemmProducer &pr, int kb, int kb1,
-                                              const bf16_t *(&ap)[4], const bf16_t *(&xp)[4],
-                                              const uint32_t (&aok)[4], const uint32_t (&xok)[4]) {
-    produce_kblock<0, PART>(g, pr, kb, kb1, ap, xp, aok, xok);
-    if constexpr (KA > 1) produce_kblock<1, PART>(g, pr, kb, kb1, ap, xp, aok, xok);
+                                              const bf16_t *(&ap)[4], const uint32_t (&aok)[4]) {
+    produce_kblock<0, PART>(g, pr, kb, kb1, ap, aok);
+    if constexpr (KA > 1) produce_kblock<1, PART>(g, pr, kb, kb1, ap, aok);
     if constexpr (KA > 2) {
-        produce_kblock<2, PART>(g, pr, kb, kb1, ap, xp, aok, xok);
-        produce_kblock<3, PART>(g, pr, kb, kb1, ap, xp, aok, xok);
+        produce_kblock<2, PART>(g, pr, kb, kb1, ap, aok);
+        produce_kblock<3, PART>(g, pr, kb, kb1, ap, aok);
     }
 }
 
 // KA 64-wide K blocks per ring stage; every stage of the ring can be in flight.
 template <int KA>
-__global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const GemmArgs g) {
+__global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap xmap) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     unsigned char *ring = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
@@ -183,7 +179,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
     while ((int)alloc_cols < 2 * buf_cols) alloc_cols <<= 1;
 
     if (tid == 0) {
-        for (int s = 0; s < S; ++s) { mbar_init(&sm->full[s], kGemmProducers); mbar_init(&sm->empty[s], 1); }
+        for (int s = 0; s < S; ++s) { mbar_init(&sm->full[s], kGemmProducers + 1); mbar_init(&sm->empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&sm->tfull[b], 1); mbar_init(&sm->tempty[b], 128); }
         mbar_init(&sm->drain, 1);
         sm->abort_flag = 0;
@@ -212,10 +208,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
         pr.dst0 = smem_u32(ring) + (uint32_t)(r0 * 128 + ((c ^ (r0 & 7)) << 4));
         pr.stage_bytes = stage_bytes; pr.kblock_bytes = kblock_bytes; pr.S = S; pr.c = c;
         pr.stage = 0; pr.phase = 0;
+        pr.tma_thread = pt == 0; pr.dst_x = smem_u32(ring) + 16384; pr.xmap = &xmap; pr.full = sm->full;
         bool ok_run = true;
         const bf16_t *ap[4];
-        const bf16_t *xp[4];
-        uint32_t aok[4], xok[4];
+        uint32_t aok[4];
         int kb0 = 0, kb1 = 0;
         auto setup_item = [&](int item) {
             const int tile = item / g.splits, split = item - tile * g.splits;
@@ -249,13 +245,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
                 }
                 ap[i] = base + (size_t)row * g.lda + (size_t)kb0 * kGemmBK + c * 8;
             }
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                int n = r0 + 32 * i;
-                xok[i] = n < g.NB ? 1u : 0u;
-                if (n >= g.NB) n = g.NB - 1;
-                xp[i] = g.x + (size_t)n * g.ldx + (size_t)kb0 * kGemmBK + c * 8;
-            }
         };
         // The weights (and the row ids, written several kernels ago) do not depend on the predecessor in the
         // stream: the weight part of the first item's first stages goes out before waiting for it.
@@ -263,7 +252,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
         int pre = 0;
         for (int kb = kb0; kb < kb1 && pre < S; kb += KA, ++pre) {
             pr.stage = pre;
-            produce_stage<KA, 1>(g, pr, kb, kb1, ap, xp, aok, xok);
+            produce_stage<KA, 1>(g, pr, kb, kb1, ap, aok);
 #pragma unroll
             for (int i = 0; i < 4; ++i) ap[i] += KA * kGemmBK;
         }
@@ -273,15 +262,17 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
             if (item != (int)blockIdx.x) setup_item(item);
             for (int kb = kb0; kb < kb1; kb += KA) {
                 if (!gemm_wait(sm, &sm->empty[pr.stage], pr.phase ^ 1u)) { ok_run = false; break; }
+                if (pr.tma_thread) {   // the X tiles of this stage: their bytes are expected on the stage's barrier
+                    const int nv = kb1 - kb < KA ? kb1 - kb : KA;
+                    mbar_arrive_expect_tx(&sm->full[pr.stage], (uint32_t)(nv * g.NB * 128));
+                }
                 if (pre > 0) {      // weight part already in flight: add the activation part
                     --pre;
-                    produce_stage<KA, 2>(g, pr, kb, kb1, ap, xp, aok, xok);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) xp[i] += KA * kGemmBK;
+                    produce_stage<KA, 2>(g, pr, kb, kb1, ap, aok);
                 } else {
-                    produce_stage<KA, 3>(g, pr, kb, kb1, ap, xp, aok, xok);
+                    produce_stage<KA, 3>(g, pr, kb, kb1, ap, aok);
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) { ap[i] += KA * kGemmBK; xp[i] += KA * kGemmBK; }
+                    for (int i = 0; i < 4; ++i) ap[i] += KA * kGemmBK;
                 }
                 // this thread's arrival on the stage's barrier fires when its copies above have landed
                 cp_async_arrive(&sm->full[pr.stage]);
@@ -425,6 +416,31 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
     }
 }
 
+// Tensor map of the activation operand X [NB][ldx] (bf16): tiles of 64 K elements x NB rows, 128-byte
+// swizzle (the layout the MMA reads), zeros beyond K. Returns 0 or a cudaError_t.
+inline int gemm_encode_xmap(CUtensorMap *map, const bf16_t *x, int ldx, int K, int NB) {
+    typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static encode_fn encode = nullptr;
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr);
+        if (e != cudaSuccess) return (int)e;
+        if (!fn || qr != cudaDriverEntryPointSuccess) return (int)cudaErrorNotSupported;
+        encode = reinterpret_cast<encode_fn>(fn);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)NB};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldx * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kGemmBK, (cuuint32_t)NB};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<bf16_t *>(x), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : (int)cudaErrorInvalidValue;
+}
+
 // Launches the GEMM on `stream` with one CTA per SM (fewer when there are fewer work items).
 // Returns the cudaError_t of the launch.
 inline int skinny_gemm_launch(GemmArgs g, int n_sm, int smem_optin, cudaStream_t stream) {
@@ -440,11 +456,14 @@ inline int skinny_gemm_launch(GemmArgs g, int n_sm, int smem_optin, cudaStream_t
     const int tile_rows = gemm_tile_rows(g.epi);
     const int n_items = ((g.n_rows + tile_rows - 1) / tile_rows) * g.splits;
     const int grid = n_items < n_sm ? n_items : n_sm;
-    void (*kern)(const GemmArgs) = ka == 4 ? skinny_gemm_kernel<4> : ka == 2 ? skinny_gemm_kernel<2> : skinny_gemm_kernel<1>;
+    void (*kern)(const GemmArgs, const CUtensorMap) = ka == 4 ? skinny_gemm_kernel<4> : ka == 2 ? skinny_gemm_kernel<2> : skinny_gemm_kernel<1>;
     if (ka != 1 && ka != 2 && ka != 4) return (int)cudaErrorInvalidConfiguration;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
-    e = launch_chained(kern, dim3(grid), dim3(kGemmThreads), smem, stream, g);
+    CUtensorMap xmap;
+    int rc = gemm_encode_xmap(&xmap, g.x, g.ldx, g.K, g.NB);
+    if (rc) return rc;
+    e = launch_chained(kern, dim3(grid), dim3(kGemmThreads), smem, stream, g, xmap);
     return (int)e;
 }
 
