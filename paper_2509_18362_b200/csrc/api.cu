@@ -503,10 +503,44 @@ int fastmtp_target_step(fmtp_ctx *c, const fmtp_target_w *w, const int32_t *toke
     if (!w->embed || !w->lm_head || !w->g_final || !w->layers) return FMTP_EINVAL;
     if (!aligned16(w->embed) || !aligned16(w->lm_head) || !aligned16(w->g_final)) return FMTP_EINVAL;
     for (int l = 0; l < nl; ++l) if (!layer_ok(w->layers[l]) || !kv_ok(kvs[l])) return FMTP_EINVAL;
+    const int V = c->shape.vocab, d = c->shape.d;
+    if ((long long)B * M >= c->batched_min && M <= kBatchRows) {
+        // more rows than one launch of the persistent kernel takes: groups of whole sequences, up to 64 rows each,
+        // every layer's weights streamed once per group by the tensor-core GEMM path
+        if ((out_h && !aligned16(out_h))) return FMTP_EINVAL;
+        const int Gs = kBatchRows / M;
+        std::vector<LayerPtrs> layers(nl);
+        std::vector<KvPtrs> lkv(nl);
+        for (int b0 = 0; b0 < B; b0 += Gs) {
+            const int Bg = (B - b0 < Gs) ? B - b0 : Gs;
+            BatchedTargetCall tc;
+            std::memset(&tc, 0, sizeof(tc));
+            tc.sh = c->bsh; tc.ws = c->bws;
+            tc.rope_cos = c->s.rope_cos; tc.rope_sin = c->s.rope_sin;
+            tc.n_sm = c->n_sm; tc.smem_optin = c->smem_optin;
+            tc.B = Bg; tc.M = M; tc.n_layers = nl;
+            tc.tokens = tokens + (size_t)b0 * M;
+            tc.out_h = out_h ? out_h + (size_t)b0 * M * d : nullptr;
+            tc.out_logits = out_logits ? out_logits + (size_t)b0 * M * V : nullptr;
+            tc.out_argmax = out_argmax ? out_argmax + (size_t)b0 * M : nullptr;
+            tc.user_status = dev_status;
+            tc.embed = w->embed; tc.lm_head = w->lm_head; tc.g_final = w->g_final;
+            for (int l = 0; l < nl; ++l) {
+                set_layer(layers[l], w->layers[l]);
+                set_kv(lkv[l], kvs[l]);
+                lkv[l].block_table += (size_t)b0 * kvs[l].max_pages_per_seq;
+                lkv[l].seq_lens += b0;
+            }
+            tc.layers = layers.data();
+            tc.kvs = lkv.data();
+            int err = batched_target(tc, static_cast<cudaStream_t>(stream), &c->launches);
+            if (err) return cuda_fail(c, (cudaError_t)err);
+        }
+        return FMTP_OK;
+    }
     if (M > kMaxRows) return FMTP_ESHAPE;                // the rows of one sequence share a launch
     const int G = group_size(c, 1, B, M);
     if (G < 1) return FMTP_ESHAPE;
-    const int V = c->shape.vocab, d = c->shape.d;
     for (int b0 = 0; b0 < B; b0 += G) {
         const int Bg = (B - b0 < G) ? B - b0 : G;
         MegaParams p;

@@ -82,10 +82,13 @@ __global__ void __launch_bounds__(kRowThreads) prologue_kernel(const PrologueArg
         int tok;
         if (a.step == 0) tok = a.tok_last[r];
         else {
-            const unsigned long long key = a.keys_prev[r];
-            if ((key >> 32) == 0ull) atomicOr(a.status, kDevAllNan);
-            tok = (int)argmax_key_id(key);
-            a.out_drafts[(size_t)r * a.K + (a.step - 1)] = tok;
+            tok = 0;
+            if (a.out_drafts) {
+                const unsigned long long key = a.keys_prev[r];
+                if ((key >> 32) == 0ull) atomicOr(a.status, kDevAllNan);
+                tok = (int)argmax_key_id(key);
+                a.out_drafts[(size_t)r * a.K + (a.step - 1)] = tok;
+            }
         }
         if ((unsigned)tok >= (unsigned)a.V) { atomicOr(a.status, kDevBadToken); tok = 0; }
         s_tok = tok;
@@ -193,6 +196,7 @@ __global__ void __launch_bounds__(kRowThreads) post_kernel(const PostArgs a) {
 // append k and v (rounded to bf16) to the paged cache. Block = (head, sequence), dh/2 threads.
 struct QkvArgs {
     int qdim, kvdim, dh, Hq, Hkv, splits, rows, ldp, page, max_ctx, step;
+    int M;                       // rows per sequence: row r is sequence r / M at position seq_len + step + r % M
     const float *partial;
     float *q;
     KvPtrs kv;
@@ -205,7 +209,8 @@ __global__ void qkv_finish_kernel(const QkvArgs a) {
     chain_wait();
     const int head = blockIdx.x, r = blockIdx.y, e = threadIdx.x, half = a.dh >> 1;
     const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
-    const int pos_true = a.kv.seq_lens[r] + a.step;
+    const int seq = r / a.M;
+    const int pos_true = a.kv.seq_lens[seq] + a.step + (r - seq * a.M);
     const int pos = min(pos_true, max_tokens - 1);
     const int col = head * a.dh;              // q heads, then k heads, then v heads: the GEMM's row order
     float lo = 0.f, hi = 0.f;
@@ -231,7 +236,7 @@ __global__ void qkv_finish_kernel(const QkvArgs a) {
     }
     const bool is_k = head < a.Hq + a.Hkv;
     const int kvh = is_k ? head - a.Hq : head - a.Hq - a.Hkv;
-    int page = a.kv.block_table[(size_t)r * a.kv.max_pages + pos / a.page];
+    int page = a.kv.block_table[(size_t)seq * a.kv.max_pages + pos / a.page];
     if ((unsigned)page >= (unsigned)a.kv.num_pages) { atomicOr(a.status, kDevBadPage); page = 0; }
     bf16_t *dst = (is_k ? a.kv.k_pages : a.kv.v_pages) + (((size_t)page * a.Hkv + kvh) * a.page + (pos % a.page)) * a.dh;
     dst[e] = f32_bf16bits(lo);
@@ -248,7 +253,8 @@ __global__ void qkv_finish_kernel(const QkvArgs a) {
 // (max, sum, output); the four warps merge in fixed order at the end of the item.
 // Output per item: unnormalised o, running max m and sum l per head.
 struct AttnArgs {
-    int Hq, Hkv, dh, page, page_shift, max_ctx, step, max_chunks, B;
+    int Hq, Hkv, dh, page, page_shift, max_ctx, step, max_chunks, B;    // B: rows
+    int M;                       // rows per sequence (row r: sequence r / M, r % M further positions visible)
     const float *q;              // [rows][Hq*dh]
     KvPtrs kv;
     float *att_part;             // [rows][Hq][max_chunks][dh+2]
@@ -310,7 +316,10 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
     };
     const int gq = a.Hq / a.Hkv;
     const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
-    if (threadIdx.x < a.B) nctx[threadIdx.x] = min(a.kv.seq_lens[threadIdx.x] + a.step, max_tokens - 1) + 1;     // visible positions 0 .. n-1
+    if (threadIdx.x < a.B) {     // visible positions 0 .. n-1 of every row
+        const int seq = threadIdx.x / a.M;
+        nctx[threadIdx.x] = min(a.kv.seq_lens[seq] + a.step + ((int)threadIdx.x - seq * a.M), max_tokens - 1) + 1;
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
         int acc = 0;
@@ -330,7 +339,7 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
         it.t0 = it.chunk * kBatchAttnChunk;
         it.n_ctx = nctx[r];
         it.n_blk = (min(kBatchAttnChunk, it.n_ctx - it.t0) + kAttnBlk - 1) / kAttnBlk;
-        it.bt = a.kv.block_table + (size_t)r * a.kv.max_pages;
+        it.bt = a.kv.block_table + (size_t)(r / a.M) * a.kv.max_pages;
     };
 
     if (producer) {
@@ -537,7 +546,7 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
 
 // ---- combine a head's chunk partials in ascending order; write the O-projection's operand.
 struct MergeArgs {
-    int Hq, dh, page, max_ctx, step, max_chunks, ld;
+    int Hq, dh, page, max_ctx, step, max_chunks, ld, M;
     KvPtrs kv;
     const float *att_part;
     bf16_t *xop;
@@ -549,7 +558,8 @@ __global__ void attn_merge_kernel(const MergeArgs a) {
     __shared__ float red[8];
     const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x;
     const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
-    const int n_ctx = min(a.kv.seq_lens[r] + a.step, max_tokens - 1) + 1;
+    const int seq = r / a.M;
+    const int n_ctx = min(a.kv.seq_lens[seq] + a.step + (r - seq * a.M), max_tokens - 1) + 1;
     const int n_chunks = (n_ctx + kBatchAttnChunk - 1) / kBatchAttnChunk;
     const int stride = a.dh + 2;
     const float *base = a.att_part + ((size_t)r * a.Hq + head) * a.max_chunks * stride;
@@ -586,6 +596,23 @@ __global__ void attn_merge_kernel(const MergeArgs a) {
         l += src[a.dh + 1] * f;
     }
     store_hilo(a.xop, a.ld, r, head * a.dh + j, acc / l);
+}
+
+// ---- target step input: x = Emb(token) per row (fp32 residual stream). One block per row.
+__global__ void __launch_bounds__(kRowThreads) embed_kernel(const int32_t *tokens, const bf16_t *embed, int d, int V, float *x,
+                                                            uint32_t *status) {
+    chain_release();
+    chain_wait();
+    const int r = blockIdx.x;
+    int tok = tokens[r];
+    if ((unsigned)tok >= (unsigned)V) { if (threadIdx.x == 0) atomicOr(status, kDevBadToken); tok = 0; }
+    const bf16_t *erow = embed + (size_t)tok * d;
+    for (int j = threadIdx.x * 8; j < d; j += kRowThreads * 8) {
+        float e[8];
+        unpack_bf16x8(*reinterpret_cast<const uint4 *>(erow + j), e);
+        *reinterpret_cast<float4 *>(x + (size_t)r * d + j) = make_float4(e[0], e[1], e[2], e[3]);
+        *reinterpret_cast<float4 *>(x + (size_t)r * d + j + 4) = make_float4(e[4], e[5], e[6], e[7]);
+    }
 }
 
 // ---- the subset in ascending id order. The argmax over the subset does not depend on the order of
@@ -764,7 +791,7 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
             QkvArgs a{};
             a.qdim = qdim; a.kvdim = kvdim; a.dh = sh.dh; a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.splits = g.splits; a.rows = B;
             a.ldp = ws.ldp; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = step; a.partial = ws.partial; a.q = ws.q;
-            a.kv = c.kv; a.rope_cos = c.rope_cos; a.rope_sin = c.rope_sin; a.status = ws.status;
+            a.kv = c.kv; a.rope_cos = c.rope_cos; a.rope_sin = c.rope_sin; a.status = ws.status; a.M = 1;
             ++*launches;
             if ((rc = (int)launch_chained(qkv_finish_kernel, dim3(sh.Hq + 2 * sh.Hkv, B), dim3(sh.dh / 2), 0, st, a))) return rc;
         }
@@ -772,14 +799,14 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
             AttnArgs a{};
             a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.dh = sh.dh; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = step;
             a.max_chunks = ws.max_chunks; a.q = ws.q; a.kv = c.kv; a.att_part = ws.att_part; a.status = ws.status;
-            a.page_shift = page_shift; a.B = B;
+            a.page_shift = page_shift; a.B = B; a.M = 1;
             ++*launches;
             if (sh.dh == 128) rc = (int)launch_chained(attn_kernel<128>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
             else rc = (int)launch_chained(attn_kernel<64>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
             if (rc) return rc;
             MergeArgs m{};
             m.Hq = sh.Hq; m.dh = sh.dh; m.page = sh.page; m.max_ctx = sh.max_ctx; m.step = step; m.max_chunks = ws.max_chunks;
-            m.ld = ws.ld0; m.kv = c.kv; m.att_part = ws.att_part; m.xop = ws.xop0;
+            m.ld = ws.ld0; m.kv = c.kv; m.att_part = ws.att_part; m.xop = ws.xop0; m.M = 1;
             ++*launches;
             if ((rc = (int)launch_chained(attn_merge_kernel, dim3(sh.Hq, B), dim3(sh.dh), 0, st, m))) return rc;
         }
@@ -808,6 +835,105 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
         if ((rc = gemm(g, c.N, d, d, ws.xop0, ws.ld0))) return rc;
     }
     return 0;
+}
+
+int batched_target(const BatchedTargetCall &c, cudaStream_t st, long long *launches) {
+    const BatchedShape &sh = c.sh;
+    const BatchedWs &ws = c.ws;
+    const int R = c.B * c.M, d = sh.d;
+    const int qdim = sh.Hq * sh.dh, kvdim = sh.Hkv * sh.dh;
+    const int NB = (2 * R + 15) / 16 * 16;
+    cudaError_t e = cudaMemsetAsync(ws.keys, 0, ws.keys_bytes, st);     // argmax keys and the status word
+    if (e != cudaSuccess) return (int)e;
+    auto gemm = [&](GemmArgs &g, int n_rows, int Kdim, int lda, const bf16_t *x, int ldx) -> int {
+        g.n_rows = n_rows; g.K = Kdim; g.lda = lda; g.x = x; g.ldx = ldx; g.NB = NB; g.R = R;
+        g.status = ws.status;
+        const int n_tiles = (n_rows + kGemmTileM - 1) / kGemmTileM, n_kb = (Kdim + kGemmBK - 1) / kGemmBK;
+        g.splits = g.epi == EPI_PARTIAL ? pick_splits(n_tiles, n_kb, c.n_sm) : 1;
+        g.kb_per_split = (n_kb + g.splits - 1) / g.splits;
+        g.splits = (n_kb + g.kb_per_split - 1) / g.kb_per_split;
+        g.partial = ws.partial; g.ldp = ws.ldp;
+        ++*launches;
+        return skinny_gemm_launch(g, c.n_sm, c.smem_optin, st);
+    };
+    auto post = [&](int splits, int final, const bf16_t *gain) -> int {
+        PostArgs a{};
+        a.d = d; a.splits = splits; a.rows = R; a.ldp = ws.ldp; a.ld = ws.ld0; a.residual = 1; a.final = final;
+        a.K = 1; a.step = 0; a.eps = sh.eps; a.partial = ws.partial; a.x = ws.x; a.hout = ws.hout;
+        a.out_h = c.out_h; a.gain = gain; a.xop = ws.xop0;
+        ++*launches;
+        return (int)launch_chained(post_kernel, dim3(R), dim3(kRowThreads), 0, st, a);
+    };
+    int rc = 0;
+    const size_t attn_smem = sh.dh == 128 ? AttnSmem<128>::TOTAL : AttnSmem<64>::TOTAL;
+    if (sh.dh == 128) e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
+    else e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
+    if (e != cudaSuccess) return (int)e;
+    int page_shift = -1;
+    for (int b = 0; b < 31; ++b) if ((1 << b) == sh.page) page_shift = b;
+
+    // x = Emb(tokens); operand of the first layer = rms(x; g_in)
+    ++*launches;
+    if ((rc = (int)launch_chained(embed_kernel, dim3(R), dim3(kRowThreads), 0, st, c.tokens, c.embed, d, sh.V, ws.x, ws.status))) return rc;
+    if ((rc = post(0, 0, c.layers[0].g_in))) return rc;
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerPtrs &L = c.layers[l];
+        const KvPtrs &kv = c.kvs[l];
+        GemmArgs g{};
+        g.a[0] = L.wq; g.a[1] = L.wk; g.a[2] = L.wv;
+        g.a_rows[0] = qdim; g.a_rows[1] = kvdim; g.a_rows[2] = kvdim; g.n_seg = 3; g.epi = EPI_PARTIAL;
+        if ((rc = gemm(g, qdim + 2 * kvdim, d, d, ws.xop0, ws.ld0))) return rc;
+        {
+            QkvArgs a{};
+            a.qdim = qdim; a.kvdim = kvdim; a.dh = sh.dh; a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.splits = g.splits; a.rows = R;
+            a.ldp = ws.ldp; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = 0; a.M = c.M; a.partial = ws.partial; a.q = ws.q;
+            a.kv = kv; a.rope_cos = c.rope_cos; a.rope_sin = c.rope_sin; a.status = ws.status;
+            ++*launches;
+            if ((rc = (int)launch_chained(qkv_finish_kernel, dim3(sh.Hq + 2 * sh.Hkv, R), dim3(sh.dh / 2), 0, st, a))) return rc;
+        }
+        {
+            AttnArgs a{};
+            a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.dh = sh.dh; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = 0;
+            a.max_chunks = ws.max_chunks; a.q = ws.q; a.kv = kv; a.att_part = ws.att_part; a.status = ws.status;
+            a.page_shift = page_shift; a.B = R; a.M = c.M;
+            ++*launches;
+            if (sh.dh == 128) rc = (int)launch_chained(attn_kernel<128>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
+            else rc = (int)launch_chained(attn_kernel<64>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
+            if (rc) return rc;
+            MergeArgs m{};
+            m.Hq = sh.Hq; m.dh = sh.dh; m.page = sh.page; m.max_ctx = sh.max_ctx; m.step = 0; m.max_chunks = ws.max_chunks;
+            m.ld = ws.ld0; m.kv = kv; m.att_part = ws.att_part; m.xop = ws.xop0; m.M = c.M;
+            ++*launches;
+            if ((rc = (int)launch_chained(attn_merge_kernel, dim3(sh.Hq, R), dim3(sh.dh), 0, st, m))) return rc;
+        }
+        g = GemmArgs{};
+        g.a[0] = L.wo; g.a_rows[0] = d; g.n_seg = 1; g.epi = EPI_PARTIAL;
+        if ((rc = gemm(g, d, qdim, qdim, ws.xop0, ws.ld0))) return rc;
+        if ((rc = post(g.splits, 0, L.g_post))) return rc;
+        g = GemmArgs{};
+        g.a[0] = L.w_gate; g.a_up = L.w_up; g.a_rows[0] = sh.F; g.n_seg = 1; g.epi = EPI_SWIGLU;
+        g.xop_out = ws.xopF; g.ld_out = ws.ldF;
+        if ((rc = gemm(g, sh.F, d, d, ws.xop0, ws.ld0))) return rc;
+        g = GemmArgs{};
+        g.a[0] = L.w_down; g.a_rows[0] = d; g.n_seg = 1; g.epi = EPI_PARTIAL;
+        if ((rc = gemm(g, d, sh.F, sh.F, ws.xopF, ws.ldF))) return rc;
+        const bool last = l + 1 == c.n_layers;
+        if ((rc = post(g.splits, last ? 1 : 0, last ? c.g_final : c.layers[l + 1].g_in))) return rc;
+    }
+    if (c.out_logits || c.out_argmax) {
+        // full output head; the greedy choice is made on the bf16-rounded logits a caller would see
+        GemmArgs g{};
+        g.a[0] = c.lm_head; g.a_rows[0] = sh.V; g.n_seg = 1; g.epi = EPI_ARGMAX; g.V = sh.V;
+        g.keys = c.out_argmax ? ws.keys : nullptr;
+        g.round_bf16 = 1; g.logits_bf16 = c.out_logits; g.logits_stride = sh.V;
+        if ((rc = gemm(g, sh.V, d, d, ws.xop0, ws.ld0))) return rc;
+    }
+    // argmax keys -> token ids (if asked for), status word -> caller
+    PrologueArgs pa{};
+    pa.step = 1; pa.K = 1; pa.d = d; pa.V = sh.V; pa.ld = ws.ld0; pa.only_tokens = 1; pa.eps = sh.eps;
+    pa.keys_prev = ws.keys; pa.out_drafts = c.out_argmax; pa.status = ws.status; pa.user_status = c.user_status;
+    ++*launches;
+    return (int)launch_chained(prologue_kernel, dim3(R), dim3(kRowThreads), 0, st, pa);
 }
 
 }  // namespace fmtp

@@ -52,6 +52,25 @@ struct BatchedCall {
     KvPtrs kv;
 };
 
+struct BatchedTargetCall {
+    BatchedShape sh;
+    BatchedWs ws;
+    const float *rope_cos, *rope_sin;
+    int n_sm, smem_optin;
+    int B, M, n_layers;                   // B * M <= kBatchRows rows
+    const int32_t *tokens;                // [B][M]
+    bf16_t *out_h;                        // [B][M][d] or NULL
+    bf16_t *out_logits;                   // [B][M][V] or NULL
+    int32_t *out_argmax;                  // [B][M] or NULL
+    uint32_t *user_status;
+    const bf16_t *embed, *lm_head, *g_final;
+    const LayerPtrs *layers;              // host array [n_layers]
+    const KvPtrs *kvs;                    // host array [n_layers]
+};
+
+// Enqueues one target-decoder step (all layers, final norm, full output head) for B sequences of M rows.
+int batched_target(const BatchedTargetCall &c, cudaStream_t stream, long long *launches);
+
 // Enqueues all K steps for one group of B <= kBatchRows sequences. Returns a cudaError_t (0 = ok)
 // and adds the kernels launched to *launches.
 int batched_draft(const BatchedCall &c, cudaStream_t stream, long long *launches);

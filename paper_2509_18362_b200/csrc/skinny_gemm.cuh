@@ -58,6 +58,8 @@ struct GemmArgs {
     unsigned long long *keys;    // EPI_ARGMAX: [R]
     float *logits;               // EPI_ARGMAX, optional: row r at logits + r*logits_stride, column m
     long long logits_stride;
+    bf16_t *logits_bf16;         // EPI_ARGMAX with round_bf16, optional: the logits as bf16, same indexing
+    int round_bf16;              // 1: the argmax is decided on the logits rounded to bf16 (the values a caller sees)
     uint32_t *status;
     int n_stages;
     int force_ka;                // 0: pick the blocks per stage from the shared memory available
@@ -379,8 +381,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
                     for (int j = 0; j < 16; ++j) {
                         const int r = (c0 >> 1) + j;           // warp-uniform
                         if (r < g.R) {
-                            const float logit = v[2 * j] + v[2 * j + 1];
+                            float logit = v[2 * j] + v[2 * j + 1];
                             if (g.logits && m_ok) g.logits[(size_t)r * g.logits_stride + m] = logit;
+                            if (g.round_bf16) {
+                                const uint16_t b = f32_bf16bits(logit);
+                                if (g.logits_bf16 && m_ok) g.logits_bf16[(size_t)r * g.logits_stride + m] = b;
+                                logit = bf16bits_f32(b);
+                            }
                             unsigned long long key = m_ok ? argmax_key(logit, row_id) : 0ull;
 #pragma unroll
                             for (int o = 16; o > 0; o >>= 1) {
@@ -398,7 +405,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
             buf ^= 1;
             if (g.epi == EPI_ARGMAX) {
                 bar_sync(1, 128);
-                if (tid < g.R) {
+                if (tid < g.R && g.keys) {
                     unsigned long long k = sm->kmax[0][tid];
 #pragma unroll
                     for (int w = 1; w < 4; ++w) k = sm->kmax[w][tid] > k ? sm->kmax[w][tid] : k;

@@ -109,7 +109,9 @@ def test_target_step_prefill_decode_verify(n_layers):
 
 
 def test_target_step_more_rows_than_one_launch():
-    """5 sequences x 4 rows = 20 rows: the call runs groups of two sequences (8 rows) per launch."""
+    """5 sequences x 4 rows = 20 rows, more than one persistent launch takes: the batched tensor-core path (every
+    layer's weights streamed once for all rows). Hidden states, logits, the kernel's own argmax and the K/V appended
+    by both layers against the oracle, over two consecutive calls."""
     shape = I.TINY.with_layers(2)
     Wt = I.target_weights(shape, 611)
     B, M = 5, 4
@@ -125,11 +127,47 @@ def test_target_step_more_rows_than_one_launch():
         rh, rl = O.target_forward(shape, Wt, t, okvs)
         close(h.float().cpu().numpy(), rh, "target h 20 rows")
         close(l.float().cpu().numpy(), rl, "target logits 20 rows")
+        rt, gap = _gaps(rl)
+        ids_match(a, rt, gap, "target argmax 20 rows")
+        own = [O.argmax_token(O.bf16_to_f64(row))[0] for row in Bd.bf16_bits(l).reshape(-1, shape.vocab)]
+        assert np.array_equal(a.ravel(), np.array(own))      # decided on the bf16 logits it wrote
         gpu.advance(M)
         for kv in okvs:
             kv["seq_lens"] += M
-    assert gpu.ctx.launch_count == 6
+    assert gpu.ctx.launch_count > 6                            # a sequence of kernels per layer, not grouped launches
+    for l in range(2):
+        close(O.bf16_to_f64(Bd.bf16_bits(gpu.dkvs[l]["k_pages"])), O.bf16_to_f64(okvs[l]["k_pages"]), f"layer {l} K cache")
+        close(O.bf16_to_f64(Bd.bf16_bits(gpu.dkvs[l]["v_pages"])), O.bf16_to_f64(okvs[l]["v_pages"]), f"layer {l} V cache")
     gpu.close()
+
+
+def test_batched_target_rows_do_not_depend_on_the_batch():
+    """On the batched path too, a row's hidden state and logits are the same bits whether its sequence is scored
+    with 2 or with 11 other sequences, and with or without the logits being written."""
+    shape = I.TINY.with_layers(2)
+    Wt = I.target_weights(shape, 711)
+    B, M = 12, 3
+    Bd = _binding()
+    L = [int(x) for x in I.context_lengths(B, 0, 300, 712)]
+    kvs = [I.paged_kv(shape, L, M + 1, 720 + l, tag="t%d" % l) for l in range(2)]
+    t = I.token_ids(730, (B, M), shape.vocab)
+    big = GpuTarget(shape, Wt, kvs, max(L) + M + 2)
+    big.ctx.close()
+    big.ctx = Bd.Context(shape, max_rows=64, max_K=8, max_ctx=max(L) + M + 2)
+    h12, l12, a12 = big.step(t)
+    big.close()
+    sub = [dict(kv) for kv in kvs]
+    for kv in sub:
+        kv["block_table"] = kv["block_table"][:3].copy()
+        kv["seq_lens"] = kv["seq_lens"][:3].copy()
+    small = GpuTarget(shape, Wt, sub, max(L) + M + 2)
+    small.ctx.close()
+    small.ctx = Bd.Context(shape, max_rows=64, max_K=8, max_ctx=max(L) + M + 2)
+    h3, l3, a3 = small.step(t[:3])
+    h3b, _, a3b = small.step(t[:3], want_logits=False)       # K/V slots are rewritten with the same values
+    small.close()
+    assert torch.equal(h3, h12[:3]) and torch.equal(l3, l12[:3]) and np.array_equal(a3, a12[:3])
+    assert torch.equal(h3b, h3) and np.array_equal(a3b, a3)
 
 
 def test_rows_do_not_depend_on_rows_per_call():
