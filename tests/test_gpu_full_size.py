@@ -7,7 +7,7 @@ import torch
 
 from oracle import fastmtp_oracle as O
 from paper_2509_18362_b200 import inputs as I
-from tests.gpu_util import close, copy_kv, ids_match
+from tests.gpu_util import GAP_TOL as GAP, close, copy_kv, ids_match
 
 pytestmark = pytest.mark.gpu
 
@@ -137,3 +137,40 @@ def test_speculative_loop_at_7b_width_is_lossless():
     ref, out, accepted = speculative_vs_greedy(I.QWEN7B.with_layers(2), 7001, K, n_new, 24, 32768, 128, 4)
     assert out[:n_new] == ref[:n_new]
     assert max(accepted) >= 2 and min(accepted) == 0
+
+
+def test_7b_width_batched_target_step_matches_oracle_on_sampled_sequences():
+    """8 sequences x 4 rows (verification-shaped, 32 rows) through a 2-layer target at the 7B width on the batched
+    path; two of the sequences are recomputed by the oracle: hidden states, sampled logits, argmax."""
+    from paper_2509_18362_b200 import binding as Bd
+    from tests.test_gpu_target import GpuTarget, _bf16_gap
+    shape = I.QWEN7B.with_layers(2)
+    Wt = I.target_weights(shape, 9001)
+    B, M = 8, 4
+    L = [int(x) for x in I.context_lengths(B, 100, 700, 9002)]
+    kvs = [I.paged_kv(shape, L, M + 1, 9010 + l, tag="t7b%d" % l) for l in range(2)]
+    t = I.token_ids(9020, (B, M), shape.vocab)
+    gpu = GpuTarget(shape, Wt, kvs, max(L) + M + 2)
+    gpu.ctx.close()
+    gpu.ctx = Bd.Context(shape, max_rows=B * M, max_K=8, max_ctx=max(L) + M + 2)
+    h, l, a = gpu.step(t)
+    assert gpu.ctx.launch_count > 10
+    sel = [0, B - 1]
+    okvs = [copy_kv(kv) for kv in kvs]
+    for kv in okvs:
+        kv["block_table"], kv["seq_lens"] = kv["block_table"][sel], kv["seq_lens"][sel]
+    rh, rl = O.target_forward(shape, Wt, t[sel], okvs)
+    close(h.float().cpu().numpy()[sel], rh, "7B-width batched target h")
+    lg = l.float().cpu().numpy()[sel]
+    g = I.rng(11, "tlogit-sample")
+    cols = g.choice(shape.vocab, size=4096, replace=False)
+    close(lg[:, :, cols], rl[:, :, cols], "7B-width batched target logits (sampled columns)")
+    for i, b in enumerate(sel):
+        for m in range(M):
+            tok, _ = O.argmax_token(O.round_bf16(rl[i, m]))
+            if a[b, m] != tok:
+                assert _bf16_gap(rl[i, m]) < GAP, f"argmax mismatch outside a near tie at b={b} m={m}"
+    own = [O.argmax_token(O.bf16_to_f64(row))[0] for row in Bd.bf16_bits(l)[sel].reshape(-1, shape.vocab)]
+    assert np.array_equal(a[sel].ravel(), np.array(own))
+    gpu.close()
+    O.clear_weight_memo()
