@@ -109,12 +109,12 @@ def test_target_step_prefill_decode_verify(n_layers):
 
 
 def test_target_step_more_rows_than_one_launch():
-    """5 sequences x 4 rows = 20 rows, more than one persistent launch takes: the batched tensor-core path (every
+    """10 sequences x 3 rows = 30 rows, more sequences than one persistent launch takes: the batched tensor-core path (every
     layer's weights streamed once for all rows). Hidden states, logits, the kernel's own argmax and the K/V appended
     by both layers against the oracle, over two consecutive calls."""
     shape = I.TINY.with_layers(2)
     Wt = I.target_weights(shape, 611)
-    B, M = 5, 4
+    B, M = 10, 3
     kvs = [I.empty_paged_kv(shape, B, 32, 620 + l) for l in range(2)]
     okvs = [copy_kv(kv) for kv in kvs]
     Bd = _binding()
@@ -125,10 +125,10 @@ def test_target_step_more_rows_than_one_launch():
         t = I.token_ids(630 + it, (B, M), shape.vocab)
         h, l, a = gpu.step(t)
         rh, rl = O.target_forward(shape, Wt, t, okvs)
-        close(h.float().cpu().numpy(), rh, "target h 20 rows")
-        close(l.float().cpu().numpy(), rl, "target logits 20 rows")
+        close(h.float().cpu().numpy(), rh, "target h 30 rows")
+        close(l.float().cpu().numpy(), rl, "target logits 30 rows")
         rt, gap = _gaps(rl)
-        ids_match(a, rt, gap, "target argmax 20 rows")
+        ids_match(a, rt, gap, "target argmax 30 rows")
         own = [O.argmax_token(O.bf16_to_f64(row))[0] for row in Bd.bf16_bits(l).reshape(-1, shape.vocab)]
         assert np.array_equal(a.ravel(), np.array(own))      # decided on the bf16 logits it wrote
         gpu.advance(M)
@@ -143,7 +143,7 @@ def test_target_step_more_rows_than_one_launch():
 
 def test_batched_target_rows_do_not_depend_on_the_batch():
     """On the batched path too, a row's hidden state and logits are the same bits whether its sequence is scored
-    with 2 or with 11 other sequences, and with or without the logits being written."""
+    with 8 or with 11 other sequences, and with or without the logits being written."""
     shape = I.TINY.with_layers(2)
     Wt = I.target_weights(shape, 711)
     B, M = 12, 3
@@ -158,15 +158,15 @@ def test_batched_target_rows_do_not_depend_on_the_batch():
     big.close()
     sub = [dict(kv) for kv in kvs]
     for kv in sub:
-        kv["block_table"] = kv["block_table"][:3].copy()
-        kv["seq_lens"] = kv["seq_lens"][:3].copy()
+        kv["block_table"] = kv["block_table"][:9].copy()
+        kv["seq_lens"] = kv["seq_lens"][:9].copy()
     small = GpuTarget(shape, Wt, sub, max(L) + M + 2)
     small.ctx.close()
     small.ctx = Bd.Context(shape, max_rows=64, max_K=8, max_ctx=max(L) + M + 2)
-    h3, l3, a3 = small.step(t[:3])
-    h3b, _, a3b = small.step(t[:3], want_logits=False)       # K/V slots are rewritten with the same values
+    h3, l3, a3 = small.step(t[:9])
+    h3b, _, a3b = small.step(t[:9], want_logits=False)       # K/V slots are rewritten with the same values
     small.close()
-    assert torch.equal(h3, h12[:3]) and torch.equal(l3, l12[:3]) and np.array_equal(a3, a12[:3])
+    assert torch.equal(h3, h12[:9]) and torch.equal(l3, l12[:9]) and np.array_equal(a3, a12[:9])
     assert torch.equal(h3b, h3) and np.array_equal(a3b, a3)
 
 
