@@ -121,7 +121,7 @@ class ClockSampler:
 # DRAM traffic of one mega_kernel launch on the default workload, from the ncu capture summarised in
 # profiles/mega_kernel_7b_batch1_ncu.md (dram__bytes_read.sum + dram__bytes_write.sum). It is only
 # reported while the kernel sources are the ones the counters were taken from.
-NCU_TRAFFIC = {"bytes_per_launch": 2270711040 + 5550080, "sources_sha256": "c9f7b65262f333ce2e10af16a8bd44d1fca9651f0a339a8002c53df6f0c8089a"}
+NCU_TRAFFIC = {"bytes_per_launch": 2270611456 + 5941760, "sources_sha256": "710410f76df4f7b31c86753f4ce4c7b2a23e0b635b391ec48d4b028b368a91d1"}
 KERNEL_SOURCES = ["megakernel.cu", "mega.cuh", "ptx.cuh", "api.cu"]
 
 
