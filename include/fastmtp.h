@@ -58,10 +58,19 @@ typedef enum {
 /* Model geometry and capacity limits (fixed for the life of a context).
  * Supported: head_dim in {64, 128}; d, n_q_heads*head_dim and ffn multiples of 16 with
  * d a multiple of 64; n_q_heads a multiple of n_kv_heads with at most 8 query heads per
- * KV head; max_rows <= 4096 (rows = batch x rows-per-sequence handled in one call). A call with
- * more rows than one launch takes (8, fewer when the input vectors of that many rows do not fit
- * in shared memory) runs as consecutive launches over groups of whole sequences on the same
- * stream; a sequence's results do not depend on how the batch is grouped. */
+ * KV head; max_rows <= 4096 (rows = batch x rows-per-sequence handled in one call).
+ *
+ * Two kernel paths sit behind the draft and target calls, chosen by the call's number of
+ * sequences B alone (never by rows per sequence, so a position scored as one of 1 or of K+1 rows
+ * gives the same bits):
+ *   - few sequences (as many as fit one launch: up to 8 rows; at most 2 sequences for models that
+ *     stream >= 256 MB of layer weights per step): one persistent kernel launch per call, or per
+ *     group of whole sequences when the rows exceed one launch;
+ *   - more sequences: groups of up to 64 rows, each step a sequence of kernels on the caller's
+ *     stream that read every weight once per group (tensor-core GEMMs).
+ * Within a path a sequence's results do not depend on the batch it is in; between the two paths
+ * results agree within the documented tolerances, not bit for bit (different summation order).
+ * The environment variable FMTP_BATCHED_MIN (read at fmtp_create) overrides the switch point. */
 typedef struct {
     int32_t d, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
     int32_t n_layers;      /* target decoder depth (fastmtp_target_step); the MTP head has 1 */
@@ -149,7 +158,8 @@ int fmtp_selftest_wait_timeout(uint32_t *dev_status, int limit_ms, unsigned long
  * of the output head restricted to rows `vocab_subset` (Eq. 3) -- ties go to the lowest
  * token id; no logits are written. Step k >= 2 consumes the head's own previous output
  * hidden state (kept in fp32) and the previous draft at position L_b + k - 1.
- * All K steps run inside one kernel launch without returning to the host.
+ * All K steps are enqueued without returning to the host (one kernel launch on the persistent
+ * path, a fixed sequence of launches on the batched path).
  *
  *   h_last        dev [B, d] bf16          tok_last     dev [B] int32
  *   vocab_subset  dev [N] int32 distinct ids in [0, vocab), any order; NULL => full vocab (N ignored)
@@ -236,7 +246,8 @@ int fastmtp_verify_accept_static(const fmtp_bf16 *target_logits, const int32_t *
  *   out_logits  dev [B, M, V] bf16 full-vocabulary logits or NULL
  *   out_argmax  dev [B, M] int32 greedy token of every row (decided on the bf16-rounded
  *               logits, ties to the lowest id) or NULL
- * Requires B*M <= max_rows. A row's results do not depend on B or M.
+ * Requires B*M <= max_rows (and M <= 8 on the persistent path, M <= 64 on the batched one). Within a path a
+ * row's results do not depend on B or M.
  */
 int fastmtp_target_step(fmtp_ctx *ctx, const fmtp_target_w *w, const int32_t *tokens,
                         const fmtp_kv *layer_kvs, int B, int M,
