@@ -276,7 +276,7 @@ struct AttnSmem {
     static constexpr int ROWB = DH * 2 + 16;                     // padded row: conflict-free fragment loads
     static constexpr int QB = 8 * DH * 4;                        // the group's query vectors (fp32)
     static constexpr int STAGE = 2 * kAttnBlk * ROWB + QB;       // K block, V block, queries (first block of an item)
-    static constexpr int MERGE = 4 * 8 * (DH + 2) * 4;
+    static constexpr int MERGE = 4 * 8 * (DH + 2) * 4 + 64 * 4;  // per-warp (o, m, l) of 8 heads, then 4 x 8 weights, 8 maxima, 8 sums
     static constexpr int TOTAL = kAttnStages * STAGE + MERGE + (kBatchRows + 1) * 4 + kBatchRows * 4 + (2 * kAttnStages + 1) * 8;
 };
 
@@ -332,7 +332,7 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
     auto load_item = [&](AttnItem &it, int item) {
         const int cidx = item / a.Hkv;
         it.kvh = item - cidx * a.Hkv;
-        int r = 0;
+        int r = it.r;                        // a CTA's items come in ascending order: search on from the last one
         while (prefix[r + 1] <= cidx) ++r;
         it.r = r;
         it.chunk = cidx - prefix[r];
@@ -358,6 +358,7 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
         }
     };
     AttnItem fc, fn;
+    fc.r = 0;
     int f_item = blockIdx.x, fb = 0, fi = 0;
     int pg_cur[NIT], pg_next[NIT];
     if (f_item < n_items) { load_item(fc, f_item); load_pages(fc, 0, pg_cur); }
@@ -411,6 +412,7 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
     const int hrow = lane >> 2, kq = (lane & 3) * 2;
     const float scale = rsqrtf((float)DH) * 1.4426950408889634f;    // scores in units of log2(e): probabilities by exp2
     AttnItem cc;
+    cc.r = 0;
     int c_item = blockIdx.x, cb = 0, ci = 0;
     if (c_item < n_items) load_item(cc, c_item);
     uint32_t qa[DH / 16][4];
@@ -518,20 +520,32 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
             for (int nt = 0; nt < DH / 8; ++nt) { dst[nt * 8 + kq] = o[nt][0] + o[nt][2]; dst[nt * 8 + kq + 1] = o[nt][1] + o[nt][3]; }
             if ((lane & 3) == 0) { dst[DH] = m_run; dst[DH + 1] = l_run; }
             bar_sync(1, kAttnThreads);
+            float *wgt = mo + 4 * 8 * (DH + 2);          // [4][8] weights, [8] maxima, [8] sums
+            if (tid < 32) {                               // thread = (head tid >> 2, warp tid & 3)
+                const int h = tid >> 2, w = tid & 3;
+                float m = -INFINITY;
+                for (int u = 0; u < 4; ++u) m = fmaxf(m, mo[((size_t)u * 8 + h) * (DH + 2) + DH]);
+                const float mw = mo[((size_t)w * 8 + h) * (DH + 2) + DH];
+                wgt[w * 8 + h] = mw == -INFINITY ? 0.f : exp2f(mw - m);
+                if (w == 0) {
+                    float l = 0.f;
+                    for (int u = 0; u < 4; ++u) {         // ascending warp order
+                        const float mu = mo[((size_t)u * 8 + h) * (DH + 2) + DH];
+                        l += mo[((size_t)u * 8 + h) * (DH + 2) + DH + 1] * (mu == -INFINITY ? 0.f : exp2f(mu - m));
+                    }
+                    wgt[32 + h] = m;
+                    wgt[40 + h] = l;
+                }
+            }
+            bar_sync(1, kAttnThreads);
             for (int i = tid; i < gq * DH; i += kAttnThreads) {
                 const int h = i / DH, j = i - h * DH;
-                float m = -INFINITY;
-                for (int w = 0; w < 4; ++w) m = fmaxf(m, mo[((size_t)w * 8 + h) * (DH + 2) + DH]);
-                float acc = 0.f, l = 0.f;
-                for (int w = 0; w < 4; ++w) {
-                    const float *src = mo + ((size_t)w * 8 + h) * (DH + 2);
-                    const float f = src[DH] == -INFINITY ? 0.f : exp2f(src[DH] - m);
-                    acc += src[j] * f;
-                    l += src[DH + 1] * f;
-                }
+                float acc = 0.f;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) acc += mo[((size_t)w * 8 + h) * (DH + 2) + j] * wgt[w * 8 + h];
                 float *out = a.att_part + (((size_t)cc.r * a.Hq + (size_t)cc.kvh * gq + h) * a.max_chunks + cc.chunk) * (DH + 2);
                 out[j] = acc;
-                if (j == 0) { out[DH] = m * 0.6931471805599453f; out[DH + 1] = l; }     // the chunk maximum in natural-log units
+                if (j == 0) { out[DH] = wgt[32 + h] * 0.6931471805599453f; out[DH + 1] = wgt[40 + h]; }     // the chunk maximum in natural-log units
             }
             bar_sync(1, kAttnThreads);     // merge buffer free for the next item
             cb = 0;
