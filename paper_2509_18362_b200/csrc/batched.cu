@@ -589,15 +589,29 @@ __global__ void attn_merge_kernel(const MergeArgs a) {
     // weighted sums in ascending chunk order
     float acc = 0.f, l = 0.f;
     int c = 0;
-    for (; c + 4 <= n_chunks; c += 4) {
-        float mv[4], lv[4], ov[4];
+    for (; c + 8 <= n_chunks; c += 8) {          // eight chunks' loads in flight, added in ascending order
+        float mv[8], lv[8], ov[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
             const float *src = base + (size_t)(c + u) * stride;
             mv[u] = src[a.dh]; lv[u] = src[a.dh + 1]; ov[u] = src[j];
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
+            const float f = expf(mv[u] - m);
+            acc += ov[u] * f;
+            l += lv[u] * f;
+        }
+    }
+    for (; c + 2 <= n_chunks; c += 2) {
+        float mv[2], lv[2], ov[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const float *src = base + (size_t)(c + u) * stride;
+            mv[u] = src[a.dh]; lv[u] = src[a.dh + 1]; ov[u] = src[j];
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
             const float f = expf(mv[u] - m);
             acc += ov[u] * f;
             l += lv[u] * f;
