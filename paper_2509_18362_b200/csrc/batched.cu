@@ -226,8 +226,15 @@ __global__ void qkv_finish_kernel(const QkvArgs a) {
         hi = y * cs + x * sn;
     }
     if (head < a.Hq) {
-        a.q[(size_t)r * a.qdim + col + e] = lo;
-        a.q[(size_t)r * a.qdim + col + e + half] = hi;
+        // stored ready for the attention MMA: scaled by log2(e) / sqrt(dh), each value as its two bf16 parts
+        // (hi in the low half-word, lo in the high one)
+        const float sc = (1.0f / sqrtf((float)a.dh)) * 1.4426950408889634f;
+        uint32_t *qq = reinterpret_cast<uint32_t *>(a.q);
+        uint16_t h0, l0, h1, l1;
+        split_bf16(lo * sc, h0, l0);
+        split_bf16(hi * sc, h1, l1);
+        qq[(size_t)r * a.qdim + col + e] = (uint32_t)h0 | ((uint32_t)l0 << 16);
+        qq[(size_t)r * a.qdim + col + e + half] = (uint32_t)h1 | ((uint32_t)l1 << 16);
         return;
     }
     if (pos_true >= max_tokens) {             // no slot for this position: flagged, nothing written
@@ -255,7 +262,7 @@ __global__ void qkv_finish_kernel(const QkvArgs a) {
 struct AttnArgs {
     int Hq, Hkv, dh, page, page_shift, max_ctx, step, max_chunks, B;    // B: rows
     int M;                       // rows per sequence (row r: sequence r / M, r % M further positions visible)
-    const float *q;              // [rows][Hq*dh]
+    const float *q;              // [rows][Hq*dh] words: the scaled query values as {hi, lo} bf16 pairs
     KvPtrs kv;
     float *att_part;             // [rows][Hq][max_chunks][dh+2]
     uint32_t *status;
@@ -395,7 +402,7 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
             cp_async16_off<0>(d0 + kAttnBlk * ROWB + it * TSTEP * ROWB, a.kv.v_pages + off[it], ok[it]);
         }
         if (fb == 0) {     // the item's query vectors ride with its first block
-            const float *qsrc = a.q + ((size_t)fc.r * a.Hq + (size_t)fc.kvh * gq) * DH;
+            const float *qsrc = a.q + ((size_t)fc.r * a.Hq + (size_t)fc.kvh * gq) * DH;    // packed {hi, lo} words
             for (int i = tid; i < gq * DH / 4; i += kAttnThreads)
                 cp_async16_off<0>(smem_u32(st + 2 * kAttnBlk * ROWB + i * 16), qsrc + i * 4, 16u);
         }
@@ -410,7 +417,6 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
 
     // ---- compute side
     const int hrow = lane >> 2, kq = (lane & 3) * 2;
-    const float scale = rsqrtf((float)DH) * 1.4426950408889634f;    // scores in units of log2(e): probabilities by exp2
     AttnItem cc;
     cc.r = 0;
     int c_item = blockIdx.x, cb = 0, ci = 0;
@@ -426,21 +432,19 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
         const unsigned char *sv = sk + kAttnBlk * ROWB;
         if (cb == 0) {
             // query fragments: A rows 0-7 = hi parts of heads 0..gq-1, rows 8-15 = lo parts
-            const float *qh = reinterpret_cast<const float *>(sv + kAttnBlk * ROWB) + hrow * DH;
+            // (the rotary kernel stored every query value as {hi, lo} bf16 halves of one word, already scaled)
+            const uint32_t *qh = reinterpret_cast<const uint32_t *>(sv + kAttnBlk * ROWB) + hrow * DH;
 #pragma unroll
             for (int ks = 0; ks < DH / 16; ++ks) {
-                float v0 = 0.f, v1 = 0.f, v2 = 0.f, v3 = 0.f;
+                uint2 w0 = make_uint2(0u, 0u), w1 = make_uint2(0u, 0u);
                 if (hrow < gq) {
-                    const float2 lo2 = *reinterpret_cast<const float2 *>(qh + ks * 16 + kq);
-                    const float2 hi2 = *reinterpret_cast<const float2 *>(qh + ks * 16 + kq + 8);
-                    v0 = lo2.x * scale; v1 = lo2.y * scale; v2 = hi2.x * scale; v3 = hi2.y * scale;
+                    w0 = *reinterpret_cast<const uint2 *>(qh + ks * 16 + kq);
+                    w1 = *reinterpret_cast<const uint2 *>(qh + ks * 16 + kq + 8);
                 }
-                uint16_t h0, l0, h1, l1, h2, l2, h3, l3;
-                split_bf16(v0, h0, l0); split_bf16(v1, h1, l1); split_bf16(v2, h2, l2); split_bf16(v3, h3, l3);
-                qa[ks][0] = (uint32_t)h0 | ((uint32_t)h1 << 16);      // row hrow,     k = kq, kq+1
-                qa[ks][1] = (uint32_t)l0 | ((uint32_t)l1 << 16);      // row hrow + 8
-                qa[ks][2] = (uint32_t)h2 | ((uint32_t)h3 << 16);      // row hrow,     k = kq+8, kq+9
-                qa[ks][3] = (uint32_t)l2 | ((uint32_t)l3 << 16);
+                qa[ks][0] = __byte_perm(w0.x, w0.y, 0x5410);      // row hrow (hi parts), k = kq, kq+1
+                qa[ks][1] = __byte_perm(w0.x, w0.y, 0x7632);      // row hrow + 8 (lo parts)
+                qa[ks][2] = __byte_perm(w1.x, w1.y, 0x5410);      // row hrow,     k = kq+8, kq+9
+                qa[ks][3] = __byte_perm(w1.x, w1.y, 0x7632);
             }
             m_run = -INFINITY; l_run = 0.f;
 #pragma unroll
