@@ -327,6 +327,46 @@ def target_forward(shp, W: dict, tokens: np.ndarray, kvs: list, want_logits: boo
     return h, logits
 
 
+def target_forward_block(shp, W: dict, tokens, kvs: list, logit_rows=()):
+    """target_forward for ONE sequence (batch index 0) with the work grouped by layer instead of by row.
+
+    Same definition, same order of operations per row: the M new tokens sit at cache positions
+    L .. L+M-1, each layer normalises, projects (q, k, v), rotates, appends K/V (rounded to bf16)
+    and attends causally, adds the output projection, then the SwiGLU MLP. The only difference is
+    that a layer's projections are evaluated for all M rows at once -- one matrix product (a
+    library matmul) per weight matrix -- so that a layer's weights are widened once per call and
+    not once per row; a long prompt through a deep target is otherwise out of reach. Attention,
+    rotary embedding and cache writes run row by row exactly as in decoder_layer. Pinned against
+    target_forward on the small shape.
+
+    Returns h [M, d] (post final norm, float64) and {row: full-vocabulary logits} for logit_rows."""
+    tokens = [int(t) for t in np.asarray(tokens).ravel()]
+    M = len(tokens)
+    Hq, Hkv, dh = shp.n_q_heads, shp.n_kv_heads, shp.head_dim
+    L = int(kvs[0]["seq_lens"][0])
+    x = bf16_to_f64(W["embed"][tokens])                                   # [M, d]
+    for l, lw in enumerate(W["layers"]):
+        n = rmsnorm(x, lw["g_in"], shp.rms_eps)
+        q = (n @ bf16_to_f64(lw["wq"]).T).reshape(M, Hq, dh)
+        k = (n @ bf16_to_f64(lw["wk"]).T).reshape(M, Hkv, dh)
+        v = (n @ bf16_to_f64(lw["wv"]).T).reshape(M, Hkv, dh)
+        o = np.empty((M, Hq * dh))
+        for m in range(M):
+            pos = L + m
+            qm = rope(q[m], pos, shp.rope_theta)
+            km = rope(k[m], pos, shp.rope_theta)
+            kv_write(kvs[l], 0, pos, km, v[m], shp.page_size)
+            Kc, Vc = kv_read(kvs[l], 0, pos + 1, shp.page_size)
+            o[m] = gqa_attention(qm, Kc, Vc).reshape(Hq * dh)
+        x = x + o @ bf16_to_f64(lw["wo"]).T
+        n = rmsnorm(x, lw["g_post"], shp.rms_eps)
+        act = silu(n @ bf16_to_f64(lw["w_gate"]).T) * (n @ bf16_to_f64(lw["w_up"]).T)
+        x = x + act @ bf16_to_f64(lw["w_down"]).T
+    h = rmsnorm(x, W["g_final"], shp.rms_eps)
+    logits = {int(r): head_logits(h[int(r)], W["lm_head"]) for r in logit_rows}
+    return h, logits
+
+
 def _boundary_logits(row: np.ndarray) -> np.ndarray:
     """Target logits cross the library boundary as bf16 before any argmax reads them."""
     return bf16_to_f64(f64_to_bf16(row))

@@ -502,3 +502,24 @@ def test_tiny_config_draft_runs_and_is_deterministic():
     b = O.draft(shape, W, h, tok, _copy_kv(kv), 3, ids)
     assert np.array_equal(a["drafts"], b["drafts"]) and a["drafts"].shape == (1, 3)
     assert np.all(np.abs(np.sqrt((a["h_out"] ** 2).mean(-1)) - 1.0) < 0.1)      # post-norm rms ~ gains ~ 1
+
+
+def test_layer_grouped_target_forward_equals_the_row_by_row_one():
+    """target_forward_block (a layer's projections as one matrix product over all rows) computes what target_forward
+    computes row by row: hidden states, logits and both layers' caches, on a prompt that crosses pages and with rows
+    appended to a non-empty cache."""
+    shp = I.TINY.with_layers(3)
+    Wt = I.target_weights(shp, 71)
+    toks = I.token_ids(72, (1, 37), shp.vocab)
+    a = [I.empty_paged_kv(shp, 1, 64, 80 + l) for l in range(3)]
+    b = [{k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in kv.items()} for kv in a]
+    for lo, hi in ((0, 29), (29, 37)):                      # a prefill, then more rows on top of it
+        h1, l1 = O.target_forward(shp, Wt, toks[:, lo:hi], a)
+        h2, l2 = O.target_forward_block(shp, Wt, toks[0, lo:hi], b, logit_rows=(0, hi - lo - 1))
+        assert np.max(np.abs(h1[0] - h2)) <= 1e-12 * max(1.0, np.max(np.abs(h1)))
+        for r, lg in l2.items():
+            assert np.max(np.abs(l1[0, r] - lg)) <= 1e-12 * max(1.0, np.max(np.abs(lg)))
+        for kv in a + b:
+            kv["seq_lens"][0] += hi - lo
+    for x, y in zip(a, b):
+        assert np.array_equal(x["k_pages"], y["k_pages"]) and np.array_equal(x["v_pages"], y["v_pages"])
