@@ -149,43 +149,53 @@ int fmtp_selftest_wait_timeout(uint32_t *dev_status, int limit_ms, unsigned long
 
 /* Recursive K-step draft for B sequences.
  *
- * Step 1 consumes, per sequence b, the pair (h_last[b], tok_last[b]): the target's last
- * hidden state (the post-final-norm vector that feeds the target's output head) and the
- * newest verified token. The pair occupies MTP-cache position L_b = mtp_kv->seq_lens[b].
- * Each step embeds the token, RMS-normalises hidden state and embedding, projects their
- * concatenation 2d -> d, runs one decoder layer (appending this position's K/V to the MTP
- * cache and attending over positions 0..pos), applies the final norm, and takes the argmax
- * of the output head restricted to rows `vocab_subset` (Eq. 3) -- ties go to the lowest
- * token id; no logits are written. Step k >= 2 consumes the head's own previous output
- * hidden state (kept in fp32) and the previous draft at position L_b + k - 1.
- * All K steps are enqueued without returning to the host (one kernel launch on the persistent
- * path, a fixed sequence of launches on the batched path).
+ * Extend rows. Since its last draft call sequence b has committed n = n_ext[b] new positions (n = accepted
+ * drafts + 1 after a verification, the prompt after a prefill). For each of them the caller passes the pair
+ * (h_last[b][m], tok_last[b][m]): the target's hidden state at that position (the post-final-norm vector
+ * that feeds the target's output head) and the token that follows it. The pairs take MTP-cache positions
+ * L_b .. L_b + n - 1 (L_b = mtp_kv->seq_lens[b]) and run through the MTP module in ONE pass over its
+ * weights, causal among themselves: this is step k = 1 of the paper, which runs the head over the shifted
+ * sequence with the target's hidden states. Only the last pair feeds the output head and gives draft 1.
+ * max_ext = 1 with n_ext = NULL is the plain form: one pair (h_last[b], tok_last[b]) per sequence.
  *
- *   h_last        dev [B, d] bf16          tok_last     dev [B] int32
+ * Each step embeds the token, RMS-normalises hidden state and embedding, projects their concatenation
+ * 2d -> d, runs one decoder layer (appending this position's K/V to the MTP cache and attending over
+ * positions 0..pos), applies the final norm, and takes the argmax of the output head restricted to rows
+ * `vocab_subset` (Eq. 3) -- ties go to the lowest token id; no logits are written. Step k >= 2 consumes the
+ * head's own previous output hidden state (kept in fp32) and the previous draft at position
+ * L_b + n - 1 + (k - 1). All K steps are enqueued without returning to the host (one kernel launch on the
+ * persistent path, a fixed sequence of launches on the batched path).
+ *
+ *   h_last        dev [B, max_ext, d] bf16   tok_last     dev [B, max_ext] int32
+ *   n_ext         dev [B] int32 in [1, max_ext] (values outside are clamped), or NULL: every sequence has
+ *                 max_ext pairs. Rows m >= n_ext[b] of h_last / tok_last are padding and are never used.
  *   vocab_subset  dev [N] int32 distinct ids in [0, vocab), any order; NULL => full vocab (N ignored)
- *   out_drafts    dev [B, K] int32         out_h        dev [B, K, d] bf16 or NULL (post-final-norm)
+ *   out_drafts    dev [B, K] int32           out_h        dev [B, K, d] bf16 or NULL (post-final-norm)
  *   out_logits    dev [B, K, N] fp32 or NULL: debug copy of the subset logits (defeats the
  *                 "no logits written" property; leave NULL in production)
  *   dev_status    dev 1 word, OR-ed with FMTP_DEV_* flags; may be NULL
  *
- * The call writes MTP-cache slots L_b .. L_b+K-1 and does not change seq_lens; the caller
- * commits by advancing seq_lens (normally by 1: slot L_b was computed from the target's
- * hidden state, later slots are speculative and are overwritten by the next round).
- * Requires B <= max_rows, K <= max_K, L_b + K <= max_ctx.
+ * The call writes MTP-cache slots L_b .. L_b + n + K - 2 and does not change seq_lens; the caller commits
+ * by advancing seq_lens by n (the extend rows are final; the K - 1 slots after them are speculative and
+ * are overwritten by the next call). Extending in one call gives the same bits as n calls with one pair
+ * each on the persistent path, and agrees within the tolerances on the batched path.
+ * Requires B * max_ext <= max_rows, max_ext <= 64, K <= max_K, L_b + n + K - 1 <= max_ctx. The persistent
+ * kernel takes the call when B is below the switch point and the B * max_ext rows fit one launch (8 rows;
+ * 4 at the 7B-class width), the batched path otherwise.
  */
 int fastmtp_draft(fmtp_ctx *ctx, const fmtp_mtp_w *w,
-                  const fmtp_bf16 *h_last, const int32_t *tok_last,
+                  const fmtp_bf16 *h_last, const int32_t *tok_last, const int32_t *n_ext, int max_ext,
                   const fmtp_kv *mtp_kv, int B, int K,
                   const int32_t *vocab_subset, int N,
                   int32_t *out_drafts, fmtp_bf16 *out_h, float *out_logits,
                   uint32_t *dev_status, void *stream);
 
 /* Same operation with the per-step inputs and the result in HOST memory: h_last host
- * [B,d] bf16 and tok_last host [B] are copied to the device, the draft runs, out_drafts
- * host [B,K] is copied back and `stream` is synchronised. Weights, subset and KV cache stay
- * on the device. Returns FMTP_EBOUNDS / FMTP_ETIMEOUT if the kernels flagged a problem. */
+ * [B,max_ext,d] bf16, tok_last host [B,max_ext] and n_ext host [B] (or NULL) are copied to the device, the
+ * draft runs, out_drafts host [B,K] is copied back and `stream` is synchronised. Weights, subset and KV
+ * cache stay on the device. Returns FMTP_EBOUNDS / FMTP_ETIMEOUT if the kernels flagged a problem. */
 int fastmtp_draft_host(fmtp_ctx *ctx, const fmtp_mtp_w *w,
-                       const fmtp_bf16 *h_last_host, const int32_t *tok_last_host,
+                       const fmtp_bf16 *h_last_host, const int32_t *tok_last_host, const int32_t *n_ext_host, int max_ext,
                        const fmtp_kv *mtp_kv, int B, int K,
                        const int32_t *vocab_subset, int N,
                        int32_t *out_drafts_host, void *stream);
@@ -205,6 +215,18 @@ int fastmtp_verify_accept(fmtp_ctx *ctx, const fmtp_bf16 *target_logits, const i
                           int B, int K, int V,
                           int32_t *out_accept_len, int32_t *out_bonus, int32_t *out_argmax,
                           uint32_t *dev_status, void *stream);
+
+/* The acceptance step of Sec. 2.3 "Verification phase" on token ids: for callers whose target step already
+ * returned the greedy token of every verification row (fastmtp_target_step with out_argmax and
+ * out_logits = NULL), so that no [B, K+1, V] logits are ever written or read. Same rule and same results as
+ * fastmtp_verify_accept given g = target_argmax: accept_len[b] = number of leading drafts equal to g[b, j],
+ * bonus[b] = g[b, accept_len[b]].
+ *
+ *   target_argmax dev [B, K+1] int32       drafts dev [B, K] int32 (ignored if K == 0)
+ *   out_accept_len, out_bonus dev [B]
+ * Uses no workspace; any B. */
+int fastmtp_accept_ids(fmtp_ctx *ctx, const int32_t *target_argmax, const int32_t *drafts, int B, int K,
+                       int32_t *out_accept_len, int32_t *out_bonus, void *stream);
 
 /* Host-buffer form: logits and drafts are copied in, accept_len / bonus copied out. */
 int fastmtp_verify_accept_host(fmtp_ctx *ctx, const fmtp_bf16 *target_logits_host,
@@ -226,6 +248,8 @@ int fastmtp_verify_accept_host(fmtp_ctx *ctx, const fmtp_bf16 *target_logits_hos
  *   device current); make that first call outside any stream capture.
  *   All calls share the one array: it is cleared on `stream` at the start of every call, and two
  *   calls whose work overlaps on the GPU (different streams, no ordering) race on it.
+ *   The looked-up address is kept for the life of the process: after a cudaDeviceReset on that device it is
+ *   stale, so a process that resets a device must not call this entry point on it again.
  * Arguments, layouts and the meaning of dev_status are those of fastmtp_verify_accept. */
 #define FMTP_STATIC_VERIFY_MAX_ROWS 1024
 int fastmtp_verify_accept_static(const fmtp_bf16 *target_logits, const int32_t *drafts,

@@ -25,7 +25,7 @@ DEV_BAD_TOKEN, DEV_BAD_PAGE, DEV_BAD_POS, DEV_TIMEOUT, DEV_ALL_NAN = 1, 2, 4, 8,
 
 EXPORTS = ["fmtp_create", "fmtp_destroy", "fmtp_workspace_bytes", "fmtp_set_workspace", "fmtp_strerror",
            "fmtp_last_cuda_error", "fmtp_launch_count", "fmtp_selftest_wait_timeout", "fastmtp_draft", "fastmtp_draft_host",
-           "fastmtp_verify_accept", "fastmtp_verify_accept_host", "fastmtp_verify_accept_static",
+           "fastmtp_verify_accept", "fastmtp_verify_accept_host", "fastmtp_verify_accept_static", "fastmtp_accept_ids",
            "fastmtp_target_step"]
 
 _p = C.c_void_p
@@ -72,16 +72,18 @@ lib.fmtp_launch_count.argtypes = [_p]
 lib.fmtp_launch_count.restype = C.c_longlong
 lib.fmtp_selftest_wait_timeout.argtypes = [_p, C.c_int, _p, _p]
 lib.fmtp_selftest_wait_timeout.restype = C.c_int
-lib.fastmtp_draft.argtypes = [_p, C.POINTER(fmtp_mtp_w), _p, _p, C.POINTER(fmtp_kv), C.c_int, C.c_int, _p, C.c_int,
-                              _p, _p, _p, _p, _p]
+lib.fastmtp_draft.argtypes = [_p, C.POINTER(fmtp_mtp_w), _p, _p, _p, C.c_int, C.POINTER(fmtp_kv), C.c_int, C.c_int, _p,
+                              C.c_int, _p, _p, _p, _p, _p]
 lib.fastmtp_draft.restype = C.c_int
-lib.fastmtp_draft_host.argtypes = [_p, C.POINTER(fmtp_mtp_w), _p, _p, C.POINTER(fmtp_kv), C.c_int, C.c_int, _p,
-                                   C.c_int, _p, _p]
+lib.fastmtp_draft_host.argtypes = [_p, C.POINTER(fmtp_mtp_w), _p, _p, _p, C.c_int, C.POINTER(fmtp_kv), C.c_int, C.c_int,
+                                   _p, C.c_int, _p, _p]
 lib.fastmtp_draft_host.restype = C.c_int
 lib.fastmtp_verify_accept.argtypes = [_p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p, _p]
 lib.fastmtp_verify_accept.restype = C.c_int
 lib.fastmtp_verify_accept_host.argtypes = [_p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p]
 lib.fastmtp_verify_accept_host.restype = C.c_int
+lib.fastmtp_accept_ids.argtypes = [_p, _p, _p, C.c_int, C.c_int, _p, _p, _p]
+lib.fastmtp_accept_ids.restype = C.c_int
 lib.fastmtp_verify_accept_static.argtypes = [_p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p, _p]
 lib.fastmtp_verify_accept_static.restype = C.c_int
 lib.fastmtp_target_step.argtypes = [_p, C.POINTER(fmtp_target_w), _p, C.POINTER(fmtp_kv), C.c_int, C.c_int,
@@ -190,24 +192,30 @@ class Context:
 
     # -- entry points (same names and argument order as the C ABI)
     def fastmtp_draft(self, w: fmtp_mtp_w, h_last, tok_last, mtp_kv: fmtp_kv, B, K, vocab_subset, out_drafts,
-                      out_h=None, out_logits=None, dev_status=None, stream=None):
+                      out_h=None, out_logits=None, dev_status=None, stream=None, n_ext=None, max_ext=1):
+        """h_last [B, max_ext, d] / tok_last [B, max_ext]; n_ext (device int32 [B]) and max_ext follow tok_last in
+        the C argument list and default to the plain one-pair-per-sequence form."""
         N = 0 if vocab_subset is None else int(vocab_subset.numel())
-        self._check(lib.fastmtp_draft(self.handle, C.byref(w), _ptr(h_last), _ptr(tok_last), C.byref(mtp_kv), B, K,
-                                      _ptr(vocab_subset), N, _ptr(out_drafts), _ptr(out_h), _ptr(out_logits),
-                                      _ptr(dev_status), _stream(stream)), "fastmtp_draft")
+        self._check(lib.fastmtp_draft(self.handle, C.byref(w), _ptr(h_last), _ptr(tok_last), _ptr(n_ext), int(max_ext),
+                                      C.byref(mtp_kv), B, K, _ptr(vocab_subset), N, _ptr(out_drafts), _ptr(out_h),
+                                      _ptr(out_logits), _ptr(dev_status), _stream(stream)), "fastmtp_draft")
 
     def fastmtp_draft_host(self, w: fmtp_mtp_w, h_last_host, tok_last_host, mtp_kv: fmtp_kv, B, K, vocab_subset,
-                           out_drafts_host, stream=None):
+                           out_drafts_host, stream=None, n_ext_host=None, max_ext=1):
         N = 0 if vocab_subset is None else int(vocab_subset.numel())
         self._check(lib.fastmtp_draft_host(self.handle, C.byref(w), _ptr(h_last_host), _ptr(tok_last_host),
-                                           C.byref(mtp_kv), B, K, _ptr(vocab_subset), N, _ptr(out_drafts_host),
-                                           _stream(stream)), "fastmtp_draft_host")
+                                           _ptr(n_ext_host), int(max_ext), C.byref(mtp_kv), B, K, _ptr(vocab_subset), N,
+                                           _ptr(out_drafts_host), _stream(stream)), "fastmtp_draft_host")
 
     def fastmtp_verify_accept(self, target_logits, drafts, B, K, V, out_accept_len, out_bonus, out_argmax=None,
                               dev_status=None, stream=None):
         self._check(lib.fastmtp_verify_accept(self.handle, _ptr(target_logits), _ptr(drafts), B, K, V,
                                               _ptr(out_accept_len), _ptr(out_bonus), _ptr(out_argmax),
                                               _ptr(dev_status), _stream(stream)), "fastmtp_verify_accept")
+
+    def fastmtp_accept_ids(self, target_argmax, drafts, B, K, out_accept_len, out_bonus, stream=None):
+        self._check(lib.fastmtp_accept_ids(self.handle, _ptr(target_argmax), _ptr(drafts), B, K, _ptr(out_accept_len),
+                                           _ptr(out_bonus), _stream(stream)), "fastmtp_accept_ids")
 
     def fastmtp_verify_accept_host(self, logits_host, drafts_host, B, K, V, out_accept_host, out_bonus_host,
                                    stream=None):

@@ -20,8 +20,6 @@ struct fmtp_ctx {
     int KC;
     int dp, qp, Fp;
     int max_chunks;
-    int stage_F_pref;          // -1 auto, 0 never, 1 whenever it fits (env FMTP_STAGE_F)
-    int stages_cap;            // upper bound on ring stages (env FMTP_STAGES)
     // workspace
     unsigned char *ws;
     size_t ws_bytes, ws_need;
@@ -31,7 +29,7 @@ struct fmtp_ctx {
     uint32_t *vcounter;
     // staging for the *_host entry points (device side inside the workspace, host side pinned)
     bf16_t *st_h;
-    int32_t *st_tok, *st_out;
+    int32_t *st_tok, *st_next, *st_out;
     uint32_t *st_status;
     void *pinned;
     size_t pinned_bytes;
@@ -43,6 +41,11 @@ struct fmtp_ctx {
     BatchedShape bsh;
     BatchedWs bws;
     int batched_min;           // calls with at least this many sequences take the batched path (env FMTP_BATCHED_MIN)
+    // answers that depend on the geometry only, kept so that the hot calls make no CUDA attribute / occupancy query:
+    struct { size_t smem; int grid; } mega_cfg[4];                 // per kernel instantiation: footprint its limit was raised to
+    struct { int mode, B, M, G; } group_memo[16];                  // sequences per launch for (mode, B, M)
+    int n_group_memo;
+    TmapCache tmaps;                                               // tensor maps of the batched path's GEMM operands
 };
 
 namespace {
@@ -92,7 +95,6 @@ size_t layout(fmtp_ctx *c, unsigned char *base) {
     c->ctrl_off = cv.off;
     int nkeys = (sh.max_K > 1 ? sh.max_K : 1) * kMaxRows;
     s.keys = cv.take<unsigned long long>((size_t)nkeys);
-    s.att_cnt = cv.take<uint32_t>((size_t)R * sh.n_kv_heads);
     s.barrier = cv.take<uint32_t>(1);
     s.abort_flag = cv.take<uint32_t>(1);
     s.status = cv.take<uint32_t>(1);
@@ -106,6 +108,7 @@ size_t layout(fmtp_ctx *c, unsigned char *base) {
     c->vcounter = cv.take<uint32_t>(1);
     c->st_h = cv.take<bf16_t>((size_t)RB * d);
     c->st_tok = cv.take<int32_t>((size_t)RB);
+    c->st_next = cv.take<int32_t>((size_t)RB);
     c->st_out = cv.take<int32_t>((size_t)RB * (sh.max_K > 1 ? sh.max_K : 1) + 2 * kVerifyMaxRows);
     c->st_status = cv.take<uint32_t>(1);
     size_t off = align_up(cv.off, 256);
@@ -131,8 +134,7 @@ int configure(fmtp_ctx *c, MegaParams &p, int mode, int B, int M) {
     p.dp = c->dp; p.qp = c->qp; p.Fp = c->Fp;
     p.eps = sh.rms_eps;
     p.KC = c->KC;
-    p.row_stride = p.KC * 2;
-    p.stage_bytes = kTileRows * p.row_stride;
+    p.stage_bytes = kTileRows * p.KC * 2;
     {   // a stage also has to hold one 64-token K/V chunk of a KV head
         int kvb = 2 * kAttnChunk * p.dh * 2;
         if (kvb > p.stage_bytes) p.stage_bytes = kvb;
@@ -153,22 +155,14 @@ int configure(fmtp_ctx *c, MegaParams &p, int mode, int B, int M) {
     size_t actq = (size_t)2 * R * act_stride(p.qdim) * 2;
     size_t base = attn > actd ? attn : actd;
     if (actq > base) base = actq;
-    size_t actF = (size_t)2 * R * act_stride(p.F) * 2;
-    size_t withF = base > actF ? base : actF;
     base = align_up(base, 128);
-    withF = align_up(withF, 128);
     size_t fixed = mega_fixed_smem(R);
     size_t avail = (size_t)c->smem_optin;
-    int st_noF = fixed + base < avail ? (int)((avail - fixed - base) / p.stage_bytes) : 0;
-    int st_F = fixed + withF < avail ? (int)((avail - fixed - withF) / p.stage_bytes) : 0;
-    // the ffn-wide input of the down projection is used once per CTA, so by default it is read from
-    // global memory (fetched one stage ahead) and the shared memory goes to a deeper ring
-    bool useF = (c->stage_F_pref == 1) && st_F >= 2;
-    p.stage_F_in_smem = useF ? 1 : 0;
-    p.scratch_smem = (int)(useF ? withF : base);
-    int ns = useF ? st_F : st_noF;
+    // the ffn-wide input of the down projection is used once per CTA: it is read from global memory (L2), one
+    // stage ahead, and the shared memory goes to a deeper ring
+    p.scratch_smem = (int)base;
+    int ns = fixed + base < avail ? (int)((avail - fixed - base) / p.stage_bytes) : 0;
     if (ns > kMaxStages) ns = kMaxStages;
-    if (ns > c->stages_cap) ns = c->stages_cap;
     if (ns < 2) return FMTP_ESHAPE;
     p.n_stages = ns;
     p.s = c->s;
@@ -198,11 +192,15 @@ int launch_mega(fmtp_ctx *c, MegaParams &p, cudaStream_t st) {
     if (e != cudaSuccess) return cuda_fail(c, e);
     int err = 0;
     size_t smem = mega_smem_bytes(p);
-    int grid = mega_max_grid(p, smem, &err);
-    if (err) return cuda_fail(c, (cudaError_t)err);
-    if (grid < 1) return FMTP_ESHAPE;
-    if (grid > c->n_sm) grid = c->n_sm;
-    err = mega_launch(p, grid, st);
+    auto &cfg = c->mega_cfg[mega_kernel_index(p)];
+    if (cfg.smem != smem || cfg.grid < 1) {       // first call with this footprint: raise the kernel's limit, ask the occupancy
+        int grid = mega_max_grid(p, smem, &err);
+        if (err) return cuda_fail(c, (cudaError_t)err);
+        if (grid < 1) return FMTP_ESHAPE;
+        cfg.smem = smem;
+        cfg.grid = grid > c->n_sm ? c->n_sm : grid;
+    }
+    err = mega_launch(p, cfg.grid, st);
     if (err) return cuda_fail(c, (cudaError_t)err);
     c->launches++;
     return FMTP_OK;
@@ -213,14 +211,21 @@ int launch_mega(fmtp_ctx *c, MegaParams &p, cudaStream_t st) {
 // one whose input vectors still leave a ring of three stages (two at worst); 0 if even one
 // sequence does not fit.
 int group_size(fmtp_ctx *c, int mode, int B, int M) {
+    for (int i = 0; i < c->n_group_memo; ++i)
+        if (c->group_memo[i].mode == mode && c->group_memo[i].B == B && c->group_memo[i].M == M) return c->group_memo[i].G;
     int gmax = kMaxRows / M;
     if (gmax > B) gmax = B;
-    for (int want = 3; want >= 2; --want)
+    int G = 0;
+    for (int want = 3; want >= 2 && G == 0; --want)
         for (int g = gmax; g >= 1; --g) {
             MegaParams tmp;
-            if (configure(c, tmp, mode, g, M) == FMTP_OK && tmp.n_stages >= want) return g;
+            if (configure(c, tmp, mode, g, M) == FMTP_OK && tmp.n_stages >= want) { G = g; break; }
         }
-    return 0;
+    if (c->n_group_memo < 16) {
+        auto &m = c->group_memo[c->n_group_memo++];
+        m.mode = mode; m.B = B; m.M = M; m.G = G;
+    }
+    return G;
 }
 
 int status_to_code(uint32_t st) {
@@ -270,18 +275,10 @@ int fmtp_create(const fmtp_shape *sh, fmtp_ctx **out) {
     c->n_sm = sms;
     c->smem_optin = optin;
     c->KC = (sh->d % 512 == 0) ? 512 : (sh->d % 256 == 0) ? 256 : (sh->d % 128 == 0) ? 128 : 64;
-    if (const char *v = std::getenv("FMTP_KC")) {
-        int kc = std::atoi(v);
-        if ((kc == 64 || kc == 128 || kc == 256 || kc == 512 || kc == 1024) && sh->d % kc == 0) c->KC = kc;
-    }
     c->dp = (sh->d + 31) & ~31;
     c->qp = (sh->n_q_heads * sh->head_dim + 31) & ~31;
     c->Fp = (sh->ffn + 31) & ~31;
     c->max_chunks = (sh->max_ctx + kAttnChunk - 1) / kAttnChunk;
-    c->stage_F_pref = -1;
-    if (const char *v = std::getenv("FMTP_STAGE_F")) c->stage_F_pref = std::atoi(v);
-    c->stages_cap = kMaxStages;
-    if (const char *v = std::getenv("FMTP_STAGES")) { int n = std::atoi(v); if (n >= 2 && n <= kMaxStages) c->stages_cap = n; }
     c->bsh.d = sh->d; c->bsh.Hq = sh->n_q_heads; c->bsh.Hkv = sh->n_kv_heads; c->bsh.dh = sh->head_dim; c->bsh.F = sh->ffn;
     c->bsh.V = sh->vocab; c->bsh.page = sh->page_size; c->bsh.max_ctx = sh->max_ctx; c->bsh.max_K = sh->max_K;
     c->bsh.max_rows = sh->max_rows; c->bsh.eps = sh->rms_eps;
@@ -299,7 +296,7 @@ int fmtp_create(const fmtp_shape *sh, fmtp_ctx **out) {
         if (layer_bytes >= 256e6 && c->batched_min > 3) c->batched_min = 3;
     }
     if (const char *v = std::getenv("FMTP_BATCHED_MIN")) { int n = std::atoi(v); if (n >= 1) c->batched_min = n; }
-    c->pinned_bytes = (size_t)sh->max_rows * sh->d * 2 + (size_t)sh->max_rows * 4 * (2 + (sh->max_K > 1 ? sh->max_K : 1)) +
+    c->pinned_bytes = (size_t)sh->max_rows * sh->d * 2 + (size_t)sh->max_rows * 4 * (3 + (sh->max_K > 1 ? sh->max_K : 1)) +
                       2 * kVerifyMaxRows * 4 + 256;
     e = cudaMallocHost(&c->pinned, c->pinned_bytes);
     if (e != cudaSuccess) { delete c; return FMTP_ECUDA; }
@@ -347,35 +344,54 @@ int fmtp_set_workspace(fmtp_ctx *c, void *dev, size_t bytes) {
     return FMTP_OK;
 }
 
-int fastmtp_draft(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_last, const int32_t *tok_last,
-                  const fmtp_kv *kv, int B, int K, const int32_t *subset, int N, int32_t *out_drafts,
-                  fmtp_bf16 *out_h, float *out_logits, uint32_t *dev_status, void *stream) {
+}  // extern "C"
+
+namespace {
+
+// Everything fastmtp_draft can check on the host, before anything is enqueued.
+int check_draft_args(const fmtp_ctx *c, const fmtp_mtp_w *w, const void *h_last, const void *tok_last, int max_ext,
+                     const fmtp_kv *kv, int B, int K, const int32_t *subset, int N, const void *out_drafts, const void *out_h) {
     if (!c || !w || !h_last || !tok_last || !kv || !out_drafts) return FMTP_EINVAL;
     if (!c->ws) return FMTP_ENOMEM;
-    if (B <= 0 || K <= 0) return FMTP_EINVAL;
-    if (B > c->shape.max_rows || K > c->shape.max_K) return FMTP_ESHAPE;
+    if (B <= 0 || K <= 0 || max_ext <= 0) return FMTP_EINVAL;
+    if ((long long)B * max_ext > c->shape.max_rows || K > c->shape.max_K || max_ext > kBatchRows) return FMTP_ESHAPE;
     if (subset && (N <= 0 || N > c->shape.vocab)) return FMTP_EINVAL;
     if (!w->embed || !w->lm_head || !w->g_hnorm || !w->g_enorm || !w->w_proj || !w->g_final) return FMTP_EINVAL;
     if (!aligned16(w->embed) || !aligned16(w->lm_head) || !aligned16(w->g_hnorm) || !aligned16(w->g_enorm) ||
         !aligned16(w->w_proj) || !aligned16(w->g_final) || !aligned16(h_last) || !layer_ok(w->layer) || !kv_ok(*kv))
         return FMTP_EINVAL;
+    if (out_h && !aligned16(out_h)) return FMTP_EINVAL;
+    return FMTP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int fastmtp_draft(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_last, const int32_t *tok_last,
+                  const int32_t *n_ext, int max_ext, const fmtp_kv *kv, int B, int K, const int32_t *subset, int N,
+                  int32_t *out_drafts, fmtp_bf16 *out_h, float *out_logits, uint32_t *dev_status, void *stream) {
+    int rc = check_draft_args(c, w, h_last, tok_last, max_ext, kv, B, K, subset, N, out_drafts, out_h);
+    if (rc) return rc;
     const int Neff = subset ? N : c->shape.vocab;
-    if (B >= c->batched_min) {
-        if (out_h && !aligned16(out_h)) return FMTP_EINVAL;
-        // more sequences than one launch of the persistent kernel takes: groups of up to 64 sequences, every
-        // weight streamed once per step and group by the tensor-core GEMM path
+    const int d = c->shape.d;
+    // the persistent kernel takes the call if its sequences are few and the extend rows of a group fit one launch
+    const int G = B < c->batched_min ? group_size(c, 0, B, max_ext) : 0;
+    if (G < 1) {
+        // groups of up to 64 sequences, every weight streamed once per step and group by the tensor-core GEMM path
         for (int b0 = 0; b0 < B; b0 += kBatchRows) {
             BatchedCall bc;
             std::memset(&bc, 0, sizeof(bc));
             bc.sh = c->bsh; bc.ws = c->bws;
             bc.rope_cos = c->s.rope_cos; bc.rope_sin = c->s.rope_sin;
-            bc.n_sm = c->n_sm; bc.smem_optin = c->smem_optin;
+            bc.n_sm = c->n_sm; bc.smem_optin = c->smem_optin; bc.cache = &c->tmaps;
             bc.B = (B - b0 < kBatchRows) ? B - b0 : kBatchRows;
             bc.K = K; bc.N = Neff; bc.ids = subset;
-            bc.h_last = h_last + (size_t)b0 * c->shape.d;
-            bc.tok_last = tok_last + b0;
+            bc.M0 = max_ext; bc.n_ext = n_ext ? n_ext + b0 : nullptr;
+            bc.h_last = h_last + (size_t)b0 * max_ext * d;
+            bc.tok_last = tok_last + (size_t)b0 * max_ext;
             bc.out_drafts = out_drafts + (size_t)b0 * K;
-            bc.out_h = out_h ? out_h + (size_t)b0 * K * c->shape.d : nullptr;
+            bc.out_h = out_h ? out_h + (size_t)b0 * K * d : nullptr;
             bc.out_logits = out_logits ? out_logits + (size_t)b0 * K * Neff : nullptr;
             bc.user_status = dev_status;
             bc.embed = w->embed; bc.lm_head = w->lm_head; bc.g_hnorm = w->g_hnorm; bc.g_enorm = w->g_enorm;
@@ -389,20 +405,19 @@ int fastmtp_draft(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_last, con
         }
         return FMTP_OK;
     }
-    const int G = group_size(c, 0, B, 1);
-    if (G < 1) return FMTP_ESHAPE;
     for (int b0 = 0; b0 < B; b0 += G) {
         const int Bg = (B - b0 < G) ? B - b0 : G;
         MegaParams p;
-        int rc = configure(c, p, 0, Bg, 1);
+        rc = configure(c, p, 0, Bg, max_ext);
         if (rc) return rc;
         p.K = K;
         p.N = Neff;
         p.ids = subset;
-        p.h_last = h_last + (size_t)b0 * c->shape.d;
-        p.tokens = tok_last + b0;
+        p.h_last = h_last + (size_t)b0 * max_ext * d;
+        p.tokens = tok_last + (size_t)b0 * max_ext;
+        p.n_ext = n_ext ? n_ext + b0 : nullptr;
         p.out_tokens = out_drafts + (size_t)b0 * K;
-        p.out_h = out_h ? out_h + (size_t)b0 * K * c->shape.d : nullptr;
+        p.out_h = out_h ? out_h + (size_t)b0 * K * d : nullptr;
         p.out_logits_f32 = out_logits ? out_logits + (size_t)b0 * K * Neff : nullptr;
         p.user_status = dev_status;
         p.embed = w->embed; p.lm_head = w->lm_head; p.g_hnorm = w->g_hnorm; p.g_enorm = w->g_enorm;
@@ -418,24 +433,29 @@ int fastmtp_draft(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_last, con
 }
 
 int fastmtp_draft_host(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_host, const int32_t *tok_host,
-                       const fmtp_kv *kv, int B, int K, const int32_t *subset, int N, int32_t *out_host,
-                       void *stream) {
-    if (!c || !h_host || !tok_host || !out_host) return FMTP_EINVAL;
-    if (!c->ws) return FMTP_ENOMEM;
-    if (B <= 0 || K <= 0) return FMTP_EINVAL;
-    if (B > c->shape.max_rows || K > c->shape.max_K) return FMTP_ESHAPE;
+                       const int32_t *n_ext_host, int max_ext, const fmtp_kv *kv, int B, int K, const int32_t *subset, int N,
+                       int32_t *out_host, void *stream) {
+    if (!c || !out_host) return FMTP_EINVAL;
+    // every check of the device call first: on a negative return nothing has been enqueued
+    int rc = check_draft_args(c, w, c->st_h, tok_host, max_ext, kv, B, K, subset, N, out_host, nullptr);
+    if (rc) return rc;
+    if (!h_host) return FMTP_EINVAL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t hb = (size_t)B * c->shape.d * 2, tb = (size_t)B * 4, ob = (size_t)B * K * 4;
+    const size_t rows = (size_t)B * max_ext;
+    const size_t hb = rows * c->shape.d * 2, tb = rows * 4, nb = n_ext_host ? (size_t)B * 4 : 0, ob = (size_t)B * K * 4;
     unsigned char *pin = static_cast<unsigned char *>(c->pinned);
     std::memcpy(pin, h_host, hb);
     std::memcpy(pin + hb, tok_host, tb);
+    if (nb) std::memcpy(pin + hb + tb, n_ext_host, nb);
     cudaError_t e = cudaMemcpyAsync(c->st_h, pin, hb, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(c->st_tok, pin + hb, tb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && nb) e = cudaMemcpyAsync(c->st_next, pin + hb + tb, nb, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->st_status, 0, 4, st);
     if (e != cudaSuccess) return cuda_fail(c, e);
-    int rc = fastmtp_draft(c, w, c->st_h, c->st_tok, kv, B, K, subset, N, c->st_out, nullptr, nullptr, c->st_status, st);
+    rc = fastmtp_draft(c, w, c->st_h, c->st_tok, nb ? c->st_next : nullptr, max_ext, kv, B, K, subset, N, c->st_out, nullptr,
+                       nullptr, c->st_status, st);
     if (rc) return rc;
-    unsigned char *po = pin + align_up(hb + tb, 16);
+    unsigned char *po = pin + align_up(hb + tb + nb, 16);
     e = cudaMemcpyAsync(po, c->st_out, ob, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(po + ob, c->st_status, 4, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
@@ -455,6 +475,16 @@ int fastmtp_verify_accept(fmtp_ctx *c, const fmtp_bf16 *logits, const int32_t *d
     if ((long long)B * (K + 1) > kVerifyMaxRows) return FMTP_ESHAPE;
     int err = verify_launch(logits, drafts, B, K, V, out_accept, out_bonus, out_argmax, c->vkeys, c->vcounter,
                             c->s.status, dev_status, c->n_sm, static_cast<cudaStream_t>(stream));
+    if (err) return cuda_fail(c, (cudaError_t)err);
+    c->launches++;
+    return FMTP_OK;
+}
+
+int fastmtp_accept_ids(fmtp_ctx *c, const int32_t *target_argmax, const int32_t *drafts, int B, int K,
+                       int32_t *out_accept, int32_t *out_bonus, void *stream) {
+    if (!c || !target_argmax || !out_accept || !out_bonus || (K > 0 && !drafts)) return FMTP_EINVAL;
+    if (B <= 0 || K < 0) return FMTP_EINVAL;
+    int err = accept_ids_launch(target_argmax, drafts, B, K, out_accept, out_bonus, static_cast<cudaStream_t>(stream));
     if (err) return cuda_fail(c, (cudaError_t)err);
     c->launches++;
     return FMTP_OK;
@@ -526,7 +556,7 @@ int fastmtp_target_step(fmtp_ctx *c, const fmtp_target_w *w, const int32_t *toke
             std::memset(&tc, 0, sizeof(tc));
             tc.sh = c->bsh; tc.ws = c->bws;
             tc.rope_cos = c->s.rope_cos; tc.rope_sin = c->s.rope_sin;
-            tc.n_sm = c->n_sm; tc.smem_optin = c->smem_optin;
+            tc.n_sm = c->n_sm; tc.smem_optin = c->smem_optin; tc.cache = &c->tmaps;
             tc.B = Bg; tc.M = M; tc.n_layers = nl;
             tc.tokens = tokens + (size_t)b0 * M;
             tc.out_h = out_h ? out_h + (size_t)b0 * M * d : nullptr;

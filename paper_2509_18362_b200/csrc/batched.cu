@@ -33,10 +33,39 @@ __device__ __forceinline__ void store_hilo(bf16_t *xop, int ld, int r, int j, fl
     xop[(size_t)(2 * r + 1) * ld + j] = lo;
 }
 
+// ---- rows of a launch. Row r belongs to sequence r / M. In a target step the M rows of a sequence sit at
+// positions L .. L+M-1. In draft step 0 they are the sequence's extend rows (Sec. 2.3 "Drafting phase":
+// the pairs of target hidden state and next token committed since the last call), n = n_ext[seq] of them
+// at positions L .. L+n-1, the last one being draft step 1; rows beyond n are padding (computed, never
+// stored or published). A later draft step has one row per sequence at position L + n - 1 + step.
+struct RowGeo {
+    int M;                   // rows per sequence in this launch
+    int M0;                  // rows per sequence of draft step 0 (the bound of n_ext); target step: M
+    int step;                // draft step (0 in a target step)
+    const int32_t *n_ext;    // [sequences] or NULL (= M0 for every sequence)
+};
+__device__ __forceinline__ int geo_next(const RowGeo &g, int seq) { return g.n_ext ? min(max(g.n_ext[seq], 1), g.M0) : g.M0; }
+// Position of row r (before clamping to the cache's capacity); *valid = false for a padding row.
+__device__ __forceinline__ int geo_pos(const RowGeo &g, const KvPtrs &kv, int r, bool *valid) {
+    const int seq = r / g.M, m = r - seq * g.M;
+    const int L = max(kv.seq_lens[seq], 0);
+    if (g.step > 0) { *valid = true; return L + geo_next(g, seq) - 1 + g.step; }
+    const int n = geo_next(g, seq);
+    *valid = m < n;
+    return L + min(m, n - 1);
+}
+// Extend step of a draft: only the last extend row of a sequence publishes its result (hidden state, head
+// operand), under the sequence's index; -1 for every other row.
+__device__ __forceinline__ int geo_out_seq(const RowGeo &g, int r) {
+    const int seq = r / g.M, m = r - seq * g.M;
+    return m == geo_next(g, seq) - 1 ? seq : -1;
+}
+
 // ---- step input: [rms(h; g_h) ; rms(Emb(tok); g_e)] as the projection's operand; also turns the
 // previous step's argmax key into its draft token. One block per sequence.
 struct PrologueArgs {
     int step, K, d, V, ld, only_tokens;
+    RowGeo geo;                  // step 0 of a draft with extend rows: which rows are padding
     float eps;
     const bf16_t *h_last;
     const int32_t *tok_last;
@@ -80,8 +109,10 @@ __global__ void __launch_bounds__(kRowThreads) prologue_kernel(const PrologueArg
     const int r = blockIdx.x, tid = threadIdx.x;
     if (tid == 0) {
         int tok;
-        if (a.step == 0) tok = a.tok_last[r];
-        else {
+        if (a.step == 0) {
+            const int seq = r / a.geo.M;                   // a padding row's token is never looked at
+            tok = (r - seq * a.geo.M < geo_next(a.geo, seq)) ? a.tok_last[r] : 0;
+        } else {
             tok = 0;
             if (a.out_drafts) {
                 const unsigned long long key = a.keys_prev[r];
@@ -134,6 +165,8 @@ __global__ void __launch_bounds__(kRowThreads) prologue_kernel(const PrologueArg
 // GEMM = rms(x; gain) as hi/lo. With `final`: the normed vector is the step's output hidden state.
 struct PostArgs {
     int d, splits, rows, ldp, ld, residual, final, K, step;
+    int map_out, seq0;           // final norm of a draft's extend step: row r publishes as sequence seq0 + geo_out_seq(r)
+    RowGeo geo;
     float eps;
     const float *partial;
     float *x, *hout;
@@ -172,21 +205,27 @@ __global__ void __launch_bounds__(kRowThreads) post_kernel(const PostArgs a) {
     }
     ss = block_sum(ss, red);
     const float rs = 1.0f / sqrtf(ss / (float)a.d + a.eps);
+    int dst = r;
+    if (a.map_out) {
+        const int o = geo_out_seq(a.geo, r);
+        if (o < 0) return;                       // an extend row that is not its sequence's last: nothing to publish
+        dst = a.seq0 + o;
+    }
     for (int j = tid * 8; j < a.d; j += kRowThreads * 8) {
         float v[8], gn[8];
         load_f32x8(a.x + (size_t)r * a.d + j, v);
         unpack_bf16x8(*reinterpret_cast<const uint4 *>(a.gain + j), gn);
 #pragma unroll
         for (int i = 0; i < 8; ++i) v[i] = v[i] * rs * gn[i];
-        store_hilo8(a.xop, a.ld, r, j, v);
+        store_hilo8(a.xop, a.ld, dst, j, v);
         if (a.final) {
-            *reinterpret_cast<float4 *>(a.hout + (size_t)r * a.d + j) = make_float4(v[0], v[1], v[2], v[3]);
-            *reinterpret_cast<float4 *>(a.hout + (size_t)r * a.d + j + 4) = make_float4(v[4], v[5], v[6], v[7]);
+            *reinterpret_cast<float4 *>(a.hout + (size_t)dst * a.d + j) = make_float4(v[0], v[1], v[2], v[3]);
+            *reinterpret_cast<float4 *>(a.hout + (size_t)dst * a.d + j + 4) = make_float4(v[4], v[5], v[6], v[7]);
             if (a.out_h) {
                 uint32_t o[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) o[i] = (uint32_t)f32_bf16bits(v[2 * i]) | ((uint32_t)f32_bf16bits(v[2 * i + 1]) << 16);
-                *reinterpret_cast<uint4 *>(a.out_h + ((size_t)r * a.K + a.step) * a.d + j) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4 *>(a.out_h + ((size_t)dst * a.K + a.step) * a.d + j) = make_uint4(o[0], o[1], o[2], o[3]);
             }
         }
     }
@@ -195,8 +234,8 @@ __global__ void __launch_bounds__(kRowThreads) post_kernel(const PostArgs a) {
 // ---- after the QKV GEMM: sum the partials, rotate q and k at the row's position, keep q in fp32,
 // append k and v (rounded to bf16) to the paged cache. Block = (head, sequence), dh/2 threads.
 struct QkvArgs {
-    int qdim, kvdim, dh, Hq, Hkv, splits, rows, ldp, page, max_ctx, step;
-    int M;                       // rows per sequence: row r is sequence r / M at position seq_len + step + r % M
+    int qdim, kvdim, dh, Hq, Hkv, splits, rows, ldp, page, max_ctx;
+    RowGeo geo;                  // which sequence and position a row has
     const float *partial;
     float *q;
     KvPtrs kv;
@@ -209,8 +248,9 @@ __global__ void qkv_finish_kernel(const QkvArgs a) {
     chain_wait();
     const int head = blockIdx.x, r = blockIdx.y, e = threadIdx.x, half = a.dh >> 1;
     const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
-    const int seq = r / a.M;
-    const int pos_true = a.kv.seq_lens[seq] + a.step + (r - seq * a.M);
+    const int seq = r / a.geo.M;
+    bool valid;
+    const int pos_true = geo_pos(a.geo, a.kv, r, &valid);
     const int pos = min(pos_true, max_tokens - 1);
     const int col = head * a.dh;              // q heads, then k heads, then v heads: the GEMM's row order
     float lo = 0.f, hi = 0.f;
@@ -237,6 +277,7 @@ __global__ void qkv_finish_kernel(const QkvArgs a) {
         qq[(size_t)r * a.qdim + col + e + half] = (uint32_t)h1 | ((uint32_t)l1 << 16);
         return;
     }
+    if (!valid) return;                       // padding row: nothing to store
     if (pos_true >= max_tokens) {             // no slot for this position: flagged, nothing written
         if (head == a.Hq && e == 0) atomicOr(a.status, kDevBadPos);
         return;
@@ -260,8 +301,8 @@ __global__ void qkv_finish_kernel(const QkvArgs a) {
 // (max, sum, output); the four warps merge in fixed order at the end of the item.
 // Output per item: unnormalised o, running max m and sum l per head.
 struct AttnArgs {
-    int Hq, Hkv, dh, page, page_shift, max_ctx, step, max_chunks, B;    // B: rows
-    int M;                       // rows per sequence (row r: sequence r / M, r % M further positions visible)
+    int Hq, Hkv, dh, page, page_shift, max_ctx, max_chunks, B;    // B: rows
+    RowGeo geo;                  // which sequence and position a row has
     const float *q;              // [rows][Hq*dh] words: the scaled query values as {hi, lo} bf16 pairs
     KvPtrs kv;
     float *att_part;             // [rows][Hq][max_chunks][dh+2]
@@ -324,8 +365,8 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
     const int gq = a.Hq / a.Hkv;
     const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
     if (threadIdx.x < a.B) {     // visible positions 0 .. n-1 of every row
-        const int seq = threadIdx.x / a.M;
-        nctx[threadIdx.x] = min(a.kv.seq_lens[seq] + a.step + ((int)threadIdx.x - seq * a.M), max_tokens - 1) + 1;
+        bool valid;
+        nctx[threadIdx.x] = min(geo_pos(a.geo, a.kv, threadIdx.x, &valid), max_tokens - 1) + 1;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -346,7 +387,7 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
         it.t0 = it.chunk * kBatchAttnChunk;
         it.n_ctx = nctx[r];
         it.n_blk = (min(kBatchAttnChunk, it.n_ctx - it.t0) + kAttnBlk - 1) / kAttnBlk;
-        it.bt = a.kv.block_table + (size_t)(r / a.M) * a.kv.max_pages;
+        it.bt = a.kv.block_table + (size_t)(r / a.geo.M) * a.kv.max_pages;
     };
 
     if (producer) {
@@ -564,7 +605,8 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
 
 // ---- combine a head's chunk partials in ascending order; write the O-projection's operand.
 struct MergeArgs {
-    int Hq, dh, page, max_ctx, step, max_chunks, ld, M;
+    int Hq, dh, page, max_ctx, max_chunks, ld;
+    RowGeo geo;
     KvPtrs kv;
     const float *att_part;
     bf16_t *xop;
@@ -576,8 +618,8 @@ __global__ void attn_merge_kernel(const MergeArgs a) {
     __shared__ float red[8];
     const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x;
     const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
-    const int seq = r / a.M;
-    const int n_ctx = min(a.kv.seq_lens[seq] + a.step + (r - seq * a.M), max_tokens - 1) + 1;
+    bool valid;
+    const int n_ctx = min(geo_pos(a.geo, a.kv, r, &valid), max_tokens - 1) + 1;
     const int n_chunks = (n_ctx + kBatchAttnChunk - 1) / kBatchAttnChunk;
     const int stride = a.dh + 2;
     const float *base = a.att_part + ((size_t)r * a.Hq + head) * a.max_chunks * stride;
@@ -734,6 +776,7 @@ size_t batched_layout(BatchedWs &ws, unsigned char *base, const BatchedShape &sh
     };
     ws.xop0 = reinterpret_cast<bf16_t *>(take((size_t)128 * ws.ld0 * 2));
     ws.xopF = reinterpret_cast<bf16_t *>(take((size_t)128 * ws.ldF * 2));
+    ws.xopH = reinterpret_cast<bf16_t *>(take((size_t)128 * ws.ld0 * 2));
     ws.partial = reinterpret_cast<float *>(take((size_t)kBatchMaxSplits * rows * ws.ldp * 4));
     ws.x = reinterpret_cast<float *>(take((size_t)rows * sh.d * 4));
     ws.hout = reinterpret_cast<float *>(take((size_t)rows * sh.d * 4));
@@ -752,8 +795,9 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
     const BatchedShape &sh = c.sh;
     const BatchedWs &ws = c.ws;
     const int B = c.B, K = c.K, d = sh.d;
+    const int M0 = c.M0 > 1 ? c.M0 : 1;
+    const bool ext = M0 > 1;                       // step 0 carries up to M0 extend rows per sequence
     const int qdim = sh.Hq * sh.dh, kvdim = sh.Hkv * sh.dh;
-    const int NB = (2 * B + 15) / 16 * 16;
     cudaError_t e = cudaMemsetAsync(ws.keys, 0, ws.keys_bytes, st);     // argmax keys and the status word
     if (e != cudaSuccess) return (int)e;
 
@@ -771,8 +815,8 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
         head_ids = ws.sorted_ids;
     }
 
-    auto gemm = [&](GemmArgs &g, int n_rows, int Kdim, int lda, const bf16_t *x, int ldx) -> int {
-        g.n_rows = n_rows; g.K = Kdim; g.lda = lda; g.x = x; g.ldx = ldx; g.NB = NB; g.R = B;
+    auto gemm = [&](GemmArgs &g, int rows, int n_rows, int Kdim, int lda, const bf16_t *x, int ldx) -> int {
+        g.n_rows = n_rows; g.K = Kdim; g.lda = lda; g.x = x; g.ldx = ldx; g.NB = (2 * rows + 15) / 16 * 16; g.R = rows;
         g.status = ws.status;
         const int n_tiles = (n_rows + kGemmTileM - 1) / kGemmTileM, n_kb = (Kdim + kGemmBK - 1) / kGemmBK;
         g.splits = g.epi == EPI_PARTIAL ? pick_splits(n_tiles, n_kb, c.n_sm) : 1;
@@ -780,93 +824,126 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
         g.splits = (n_kb + g.kb_per_split - 1) / g.kb_per_split;      // no empty range
         g.partial = ws.partial; g.ldp = ws.ldp;
         ++*launches;
-        return skinny_gemm_launch(g, c.n_sm, c.smem_optin, st);
-    };
-    auto post = [&](int splits, int residual, int final, const bf16_t *gain, int step) -> int {
-        PostArgs a{};
-        a.d = d; a.splits = splits; a.rows = B; a.ldp = ws.ldp; a.ld = ws.ld0; a.residual = residual; a.final = final;
-        a.K = K; a.step = step; a.eps = sh.eps; a.partial = ws.partial; a.x = ws.x; a.hout = ws.hout;
-        a.out_h = c.out_h; a.gain = gain; a.xop = ws.xop0;
-        ++*launches;
-        return (int)launch_chained(post_kernel, dim3(B), dim3(kRowThreads), 0, st, a);
+        return skinny_gemm_launch(g, c.n_sm, c.smem_optin, st, c.cache);
     };
     int rc = 0;
     const size_t attn_smem = sh.dh == 128 ? AttnSmem<128>::TOTAL : AttnSmem<64>::TOTAL;
-    if (sh.dh == 128) e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
-    else e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
-    if (e != cudaSuccess) return (int)e;
+    if (c.cache->attn_smem < (int)attn_smem) {
+        if (sh.dh == 128) e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
+        else e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
+        if (e != cudaSuccess) return (int)e;
+        c.cache->attn_smem = (int)attn_smem;
+    }
     int page_shift = -1;
     for (int b = 0; b < 31; ++b) if ((1 << b) == sh.page) page_shift = b;
 
-    for (int step = 0; step <= K; ++step) {
+    // One pass of the MTP module (projection, decoder layer, final norm) over `rows` activation rows of the sequences
+    // seq0 .. seq0 + rows / geo.M - 1 of the group. The final norm publishes into `xop_head` (the output head's operand),
+    // hout and out_h, under the row's own index or, in an extend pass, under its sequence's.
+    auto mtp_pass = [&](int step, int rows, int seq0, const RowGeo &geo, bf16_t *xop_head, int map_out) -> int {
+        KvPtrs kv = c.kv;
+        kv.block_table += (size_t)seq0 * kv.max_pages;
+        kv.seq_lens += seq0;
+        auto post = [&](int splits, int residual, int final, const bf16_t *gain) -> int {
+            PostArgs a{};
+            a.d = d; a.splits = splits; a.rows = rows; a.ldp = ws.ldp; a.ld = ws.ld0; a.residual = residual; a.final = final;
+            a.K = K; a.step = step; a.eps = sh.eps; a.partial = ws.partial; a.x = ws.x; a.hout = ws.hout;
+            a.out_h = c.out_h; a.gain = gain; a.xop = final ? xop_head : ws.xop0;
+            a.map_out = final ? map_out : 0; a.seq0 = seq0; a.geo = geo;
+            ++*launches;
+            return (int)launch_chained(post_kernel, dim3(rows), dim3(kRowThreads), 0, st, a);
+        };
         PrologueArgs pa{};
-        pa.step = step; pa.K = K; pa.d = d; pa.V = sh.V; pa.ld = ws.ld0; pa.only_tokens = step == K ? 1 : 0;
-        pa.eps = sh.eps; pa.h_last = c.h_last; pa.tok_last = c.tok_last; pa.hout = ws.hout;
+        pa.step = step; pa.K = K; pa.d = d; pa.V = sh.V; pa.ld = ws.ld0; pa.only_tokens = 0; pa.geo = geo;
+        pa.eps = sh.eps; pa.h_last = c.h_last + (size_t)seq0 * M0 * d; pa.tok_last = c.tok_last + (size_t)seq0 * M0; pa.hout = ws.hout;
         pa.keys_prev = step > 0 ? ws.keys + (size_t)(step - 1) * kBatchRows : nullptr;
         pa.out_drafts = c.out_drafts; pa.embed = c.embed; pa.g_h = c.g_hnorm; pa.g_e = c.g_enorm;
         pa.xop = ws.xop0; pa.status = ws.status; pa.user_status = c.user_status;
         ++*launches;
-        if ((rc = (int)launch_chained(prologue_kernel, dim3(B), dim3(kRowThreads), 0, st, pa))) return rc;
-        if (step == K) break;
-
+        int rc = 0;
+        if ((rc = (int)launch_chained(prologue_kernel, dim3(rows), dim3(kRowThreads), 0, st, pa))) return rc;
         GemmArgs g{};
         // x = W_p [rms(h); rms(e)]
         g.a[0] = c.w_proj; g.a_rows[0] = d; g.n_seg = 1; g.epi = EPI_PARTIAL;
-        if ((rc = gemm(g, d, 2 * d, 2 * d, ws.xop0, ws.ld0))) return rc;
-        if ((rc = post(g.splits, 0, 0, c.layer.g_in, step))) return rc;
+        if ((rc = gemm(g, rows, d, 2 * d, 2 * d, ws.xop0, ws.ld0))) return rc;
+        if ((rc = post(g.splits, 0, 0, c.layer.g_in))) return rc;
         // q, k, v
         g = GemmArgs{};
         g.a[0] = c.layer.wq; g.a[1] = c.layer.wk; g.a[2] = c.layer.wv;
         g.a_rows[0] = qdim; g.a_rows[1] = kvdim; g.a_rows[2] = kvdim; g.n_seg = 3; g.epi = EPI_PARTIAL;
-        if ((rc = gemm(g, qdim + 2 * kvdim, d, d, ws.xop0, ws.ld0))) return rc;
+        if ((rc = gemm(g, rows, qdim + 2 * kvdim, d, d, ws.xop0, ws.ld0))) return rc;
         {
             QkvArgs a{};
-            a.qdim = qdim; a.kvdim = kvdim; a.dh = sh.dh; a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.splits = g.splits; a.rows = B;
-            a.ldp = ws.ldp; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = step; a.partial = ws.partial; a.q = ws.q;
-            a.kv = c.kv; a.rope_cos = c.rope_cos; a.rope_sin = c.rope_sin; a.status = ws.status; a.M = 1;
+            a.qdim = qdim; a.kvdim = kvdim; a.dh = sh.dh; a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.splits = g.splits; a.rows = rows;
+            a.ldp = ws.ldp; a.page = sh.page; a.max_ctx = sh.max_ctx; a.geo = geo; a.partial = ws.partial; a.q = ws.q;
+            a.kv = kv; a.rope_cos = c.rope_cos; a.rope_sin = c.rope_sin; a.status = ws.status;
             ++*launches;
-            if ((rc = (int)launch_chained(qkv_finish_kernel, dim3(sh.Hq + 2 * sh.Hkv, B), dim3(sh.dh / 2), 0, st, a))) return rc;
+            if ((rc = (int)launch_chained(qkv_finish_kernel, dim3(sh.Hq + 2 * sh.Hkv, rows), dim3(sh.dh / 2), 0, st, a))) return rc;
         }
         {
             AttnArgs a{};
-            a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.dh = sh.dh; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = step;
-            a.max_chunks = ws.max_chunks; a.q = ws.q; a.kv = c.kv; a.att_part = ws.att_part; a.status = ws.status;
-            a.page_shift = page_shift; a.B = B; a.M = 1;
+            a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.dh = sh.dh; a.page = sh.page; a.max_ctx = sh.max_ctx; a.geo = geo;
+            a.max_chunks = ws.max_chunks; a.q = ws.q; a.kv = kv; a.att_part = ws.att_part; a.status = ws.status;
+            a.page_shift = page_shift; a.B = rows;
             ++*launches;
             if (sh.dh == 128) rc = (int)launch_chained(attn_kernel<128>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
             else rc = (int)launch_chained(attn_kernel<64>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
             if (rc) return rc;
             MergeArgs m{};
-            m.Hq = sh.Hq; m.dh = sh.dh; m.page = sh.page; m.max_ctx = sh.max_ctx; m.step = step; m.max_chunks = ws.max_chunks;
-            m.ld = ws.ld0; m.kv = c.kv; m.att_part = ws.att_part; m.xop = ws.xop0; m.M = 1;
+            m.Hq = sh.Hq; m.dh = sh.dh; m.page = sh.page; m.max_ctx = sh.max_ctx; m.geo = geo; m.max_chunks = ws.max_chunks;
+            m.ld = ws.ld0; m.kv = kv; m.att_part = ws.att_part; m.xop = ws.xop0;
             ++*launches;
-            if ((rc = (int)launch_chained(attn_merge_kernel, dim3(sh.Hq, B), dim3(sh.dh), 0, st, m))) return rc;
+            if ((rc = (int)launch_chained(attn_merge_kernel, dim3(sh.Hq, rows), dim3(sh.dh), 0, st, m))) return rc;
         }
         // x += W_o o
         g = GemmArgs{};
         g.a[0] = c.layer.wo; g.a_rows[0] = d; g.n_seg = 1; g.epi = EPI_PARTIAL;
-        if ((rc = gemm(g, d, qdim, qdim, ws.xop0, ws.ld0))) return rc;
-        if ((rc = post(g.splits, 1, 0, c.layer.g_post, step))) return rc;
+        if ((rc = gemm(g, rows, d, qdim, qdim, ws.xop0, ws.ld0))) return rc;
+        if ((rc = post(g.splits, 1, 0, c.layer.g_post))) return rc;
         // act = silu(W_gate n) * (W_up n), written as the down projection's operand
         g = GemmArgs{};
         g.a[0] = c.layer.w_gate; g.a_up = c.layer.w_up; g.a_rows[0] = sh.F; g.n_seg = 1; g.epi = EPI_SWIGLU;
         g.xop_out = ws.xopF; g.ld_out = ws.ldF;
-        if ((rc = gemm(g, sh.F, d, d, ws.xop0, ws.ld0))) return rc;
+        if ((rc = gemm(g, rows, sh.F, d, d, ws.xop0, ws.ld0))) return rc;
         // x += W_down act; h_out = rms(x; g_final)
         g = GemmArgs{};
         g.a[0] = c.layer.w_down; g.a_rows[0] = d; g.n_seg = 1; g.epi = EPI_PARTIAL;
-        if ((rc = gemm(g, d, sh.F, sh.F, ws.xopF, ws.ldF))) return rc;
-        if ((rc = post(g.splits, 1, 1, c.g_final, step))) return rc;
+        if ((rc = gemm(g, rows, d, sh.F, sh.F, ws.xopF, ws.ldF))) return rc;
+        return post(g.splits, 1, 1, c.g_final);
+    };
+
+    for (int step = 0; step < K; ++step) {
+        const bf16_t *xop_head = ws.xop0;
+        if (step == 0 && ext) {
+            // extend rows: whole sequences in passes of up to 64 rows; each pass streams the module's weights once and
+            // publishes its sequences' last rows into the head's operand, so the output head runs once for the group
+            const int Gs = kBatchRows / M0;
+            for (int s0 = 0; s0 < B; s0 += Gs) {
+                const int Bs = B - s0 < Gs ? B - s0 : Gs;
+                const RowGeo geo{M0, M0, 0, c.n_ext ? c.n_ext + s0 : nullptr};
+                if ((rc = mtp_pass(0, Bs * M0, s0, geo, ws.xopH, 1))) return rc;
+            }
+            xop_head = ws.xopH;
+        } else {
+            const RowGeo geo{1, M0, step, c.n_ext};
+            if ((rc = mtp_pass(step, B, 0, geo, ws.xop0, 0))) return rc;
+        }
         // compressed head + argmax (Eq. 3)
-        g = GemmArgs{};
+        GemmArgs g{};
         g.a[0] = c.lm_head; g.a_rows[0] = c.N; g.n_seg = 1; g.epi = EPI_ARGMAX;
         g.row_ids = head_ids; g.V = sh.V;
         g.keys = ws.keys + (size_t)step * kBatchRows;
         g.logits = c.out_logits ? c.out_logits + (size_t)step * c.N : nullptr;
         g.logits_stride = (long long)K * c.N;
-        if ((rc = gemm(g, c.N, d, d, ws.xop0, ws.ld0))) return rc;
+        if ((rc = gemm(g, B, c.N, d, d, xop_head, ws.ld0))) return rc;
     }
-    return 0;
+    // the last step's argmax keys -> draft tokens; status word -> caller
+    PrologueArgs pa{};
+    pa.step = K; pa.K = K; pa.d = d; pa.V = sh.V; pa.ld = ws.ld0; pa.only_tokens = 1; pa.geo = RowGeo{1, M0, K, c.n_ext};
+    pa.eps = sh.eps; pa.keys_prev = ws.keys + (size_t)(K - 1) * kBatchRows;
+    pa.out_drafts = c.out_drafts; pa.status = ws.status; pa.user_status = c.user_status;
+    ++*launches;
+    return (int)launch_chained(prologue_kernel, dim3(B), dim3(kRowThreads), 0, st, pa);
 }
 
 int batched_target(const BatchedTargetCall &c, cudaStream_t st, long long *launches) {
@@ -875,6 +952,7 @@ int batched_target(const BatchedTargetCall &c, cudaStream_t st, long long *launc
     const int R = c.B * c.M, d = sh.d;
     const int qdim = sh.Hq * sh.dh, kvdim = sh.Hkv * sh.dh;
     const int NB = (2 * R + 15) / 16 * 16;
+    const RowGeo geo{c.M, c.M, 0, nullptr};       // M rows per sequence at positions L .. L+M-1, all of them real
     cudaError_t e = cudaMemsetAsync(ws.keys, 0, ws.keys_bytes, st);     // argmax keys and the status word
     if (e != cudaSuccess) return (int)e;
     auto gemm = [&](GemmArgs &g, int n_rows, int Kdim, int lda, const bf16_t *x, int ldx) -> int {
@@ -886,7 +964,7 @@ int batched_target(const BatchedTargetCall &c, cudaStream_t st, long long *launc
         g.splits = (n_kb + g.kb_per_split - 1) / g.kb_per_split;
         g.partial = ws.partial; g.ldp = ws.ldp;
         ++*launches;
-        return skinny_gemm_launch(g, c.n_sm, c.smem_optin, st);
+        return skinny_gemm_launch(g, c.n_sm, c.smem_optin, st, c.cache);
     };
     auto post = [&](int splits, int final, const bf16_t *gain) -> int {
         PostArgs a{};
@@ -898,9 +976,12 @@ int batched_target(const BatchedTargetCall &c, cudaStream_t st, long long *launc
     };
     int rc = 0;
     const size_t attn_smem = sh.dh == 128 ? AttnSmem<128>::TOTAL : AttnSmem<64>::TOTAL;
-    if (sh.dh == 128) e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
-    else e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
-    if (e != cudaSuccess) return (int)e;
+    if (c.cache->attn_smem < (int)attn_smem) {
+        if (sh.dh == 128) e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
+        else e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem);
+        if (e != cudaSuccess) return (int)e;
+        c.cache->attn_smem = (int)attn_smem;
+    }
     int page_shift = -1;
     for (int b = 0; b < 31; ++b) if ((1 << b) == sh.page) page_shift = b;
 
@@ -918,23 +999,23 @@ int batched_target(const BatchedTargetCall &c, cudaStream_t st, long long *launc
         {
             QkvArgs a{};
             a.qdim = qdim; a.kvdim = kvdim; a.dh = sh.dh; a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.splits = g.splits; a.rows = R;
-            a.ldp = ws.ldp; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = 0; a.M = c.M; a.partial = ws.partial; a.q = ws.q;
+            a.ldp = ws.ldp; a.page = sh.page; a.max_ctx = sh.max_ctx; a.geo = geo; a.partial = ws.partial; a.q = ws.q;
             a.kv = kv; a.rope_cos = c.rope_cos; a.rope_sin = c.rope_sin; a.status = ws.status;
             ++*launches;
             if ((rc = (int)launch_chained(qkv_finish_kernel, dim3(sh.Hq + 2 * sh.Hkv, R), dim3(sh.dh / 2), 0, st, a))) return rc;
         }
         {
             AttnArgs a{};
-            a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.dh = sh.dh; a.page = sh.page; a.max_ctx = sh.max_ctx; a.step = 0;
+            a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.dh = sh.dh; a.page = sh.page; a.max_ctx = sh.max_ctx; a.geo = geo;
             a.max_chunks = ws.max_chunks; a.q = ws.q; a.kv = kv; a.att_part = ws.att_part; a.status = ws.status;
-            a.page_shift = page_shift; a.B = R; a.M = c.M;
+            a.page_shift = page_shift; a.B = R;
             ++*launches;
             if (sh.dh == 128) rc = (int)launch_chained(attn_kernel<128>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
             else rc = (int)launch_chained(attn_kernel<64>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
             if (rc) return rc;
             MergeArgs m{};
-            m.Hq = sh.Hq; m.dh = sh.dh; m.page = sh.page; m.max_ctx = sh.max_ctx; m.step = 0; m.max_chunks = ws.max_chunks;
-            m.ld = ws.ld0; m.kv = kv; m.att_part = ws.att_part; m.xop = ws.xop0; m.M = c.M;
+            m.Hq = sh.Hq; m.dh = sh.dh; m.page = sh.page; m.max_ctx = sh.max_ctx; m.geo = geo; m.max_chunks = ws.max_chunks;
+            m.ld = ws.ld0; m.kv = kv; m.att_part = ws.att_part; m.xop = ws.xop0;
             ++*launches;
             if ((rc = (int)launch_chained(attn_merge_kernel, dim3(sh.Hq, R), dim3(sh.dh), 0, st, m))) return rc;
         }
@@ -963,6 +1044,7 @@ int batched_target(const BatchedTargetCall &c, cudaStream_t st, long long *launc
     // argmax keys -> token ids (if asked for), status word -> caller
     PrologueArgs pa{};
     pa.step = 1; pa.K = 1; pa.d = d; pa.V = sh.V; pa.ld = ws.ld0; pa.only_tokens = 1; pa.eps = sh.eps;
+    pa.geo = geo;
     pa.keys_prev = ws.keys; pa.out_drafts = c.out_argmax; pa.status = ws.status; pa.user_status = c.user_status;
     ++*launches;
     return (int)launch_chained(prologue_kernel, dim3(R), dim3(kRowThreads), 0, st, pa);

@@ -10,9 +10,25 @@ constexpr int kBatchRows = 64;        // sequences per group (activation columns
 constexpr int kBatchAttnChunk = 256;  // context tokens per attention work item
 constexpr int kBatchMaxSplits = 8;
 
+// What the launches of the batched path would otherwise ask the driver for on every call; lives in the context
+// (one per device), filled on first use: the tensor maps of the GEMMs' activation operands, and the
+// shared-memory limits already raised on the kernels.
+struct TmapEntry {
+    const void *x;
+    int ldx, K, NB;
+    alignas(64) unsigned char map[128];      // a CUtensorMap
+};
+struct TmapCache {
+    TmapEntry e[12];
+    int n, next;
+    int gemm_smem[3];                        // limit set on skinny_gemm_kernel<1>, <2>, <4>
+    int attn_smem;                           // limit set on attn_kernel
+};
+
 struct BatchedWs {
     bf16_t *xop0;                 // [128][ld0]  hi/lo activation operand (projection, QKV, O-proj, MLP and head inputs)
     bf16_t *xopF;                 // [128][ldF]  hi/lo SwiGLU activation (input of the down projection)
+    bf16_t *xopH;                 // [128][ld0]  head operand gathered from the passes of a draft's extend step
     float *partial;               // [kBatchMaxSplits][rows][ldp] split-K partial sums
     float *x;                     // [rows][d]   residual stream
     float *hout;                  // [rows][d]   final-normed hidden state (recursed in fp32)
@@ -39,10 +55,13 @@ struct BatchedCall {
     BatchedWs ws;
     const float *rope_cos, *rope_sin;     // [max_ctx][dh/2]
     int n_sm, smem_optin;
+    TmapCache *cache;
     int B, K, N;
     const int32_t *ids;                   // subset or NULL
-    const bf16_t *h_last;                 // [B][d]
-    const int32_t *tok_last;              // [B]
+    int M0;                               // extend rows per sequence in step 0 (layout of h_last / tok_last), >= 1
+    const int32_t *n_ext;                 // [B] rows of a sequence that count (1..M0), NULL = M0 for every sequence
+    const bf16_t *h_last;                 // [B][M0][d]
+    const int32_t *tok_last;              // [B][M0]
     int32_t *out_drafts;                  // [B][K]
     bf16_t *out_h;                        // [B][K][d] or NULL
     float *out_logits;                    // [B][K][N] or NULL
@@ -57,6 +76,7 @@ struct BatchedTargetCall {
     BatchedWs ws;
     const float *rope_cos, *rope_sin;
     int n_sm, smem_optin;
+    TmapCache *cache;
     int B, M, n_layers;                   // B * M <= kBatchRows rows
     const int32_t *tokens;                // [B][M]
     bf16_t *out_h;                        // [B][M][d] or NULL

@@ -43,7 +43,6 @@ struct Scratch {
     bf16_t *actF_hi, *actF_lo;        // [R][Fp]  SwiGLU activation
     float *ssA, *ssB, *ssC, *ssD;     // [grid][8] per-CTA partial sums of squares
     float *att_part;                  // [R][Hq][max_chunks][dh + 2] (o, m, l) per context chunk
-    uint32_t *att_cnt;                // [B_max][Hkv] arrival counters
     unsigned long long *keys;         // [max_K or 1][8] argmax keys
     const float *rope_cos, *rope_sin; // [max_ctx][dh/2]
     uint32_t *barrier;                // grid barrier counter
@@ -57,20 +56,20 @@ struct MegaParams {
     int dp, qp, Fp;                   // padded row lengths of the hi/lo buffers (multiples of 32)
     float eps;
     int KC;                           // k elements per pipeline stage
-    int n_stages, stage_bytes, row_stride;  // ring geometry (bytes)
+    int n_stages, stage_bytes;        // ring geometry: stages of stage_bytes (32 weight rows x KC elements, or one K/V chunk)
     int scratch_smem;                 // bytes of the per-phase shared scratch region
-    int stage_F_in_smem;              // 1: the ffn-length activation is staged in shared memory
     int max_chunks;                   // capacity of att_part's chunk dimension
     int max_ctx;                      // rows of the rotary table
     // call
     int mode;                         // 0: MTP draft, 1: target step
-    int B, M, R;                      // sequences, rows per sequence, R = B*M
+    int B, M, R;                      // sequences, rows per sequence (draft: extend rows of step 0), R = B*M
     int K;                            // draft steps (mode 0)
     int n_layers;                     // mode 1
     int N;                            // head rows (subset size or V)
     const int32_t *ids;               // subset or NULL
-    const bf16_t *h_last;             // [B][d] (mode 0)
-    const int32_t *tokens;            // mode 0: tok_last [B]; mode 1: [B][M]
+    const bf16_t *h_last;             // [B][M][d] (mode 0)
+    const int32_t *tokens;            // mode 0: tok_last [B][M]; mode 1: [B][M]
+    const int32_t *n_ext;             // mode 0: [B] extend rows per sequence (1..M), NULL = M for every sequence
     int32_t *out_tokens;              // mode 0: drafts [B][K]; mode 1: argmax [B][M] or NULL
     bf16_t *out_h;                    // mode 0: [B][K][d]; mode 1: [B][M][d]; or NULL
     float *out_logits_f32;            // mode 0 debug [B][K][N] or NULL
@@ -87,15 +86,23 @@ struct MegaParams {
 size_t mega_smem_bytes(const MegaParams &p);
 // Shared memory used besides the per-phase scratch and the ring, for R activation rows.
 size_t mega_fixed_smem(int R);
-// Cooperative launch on `stream` with `grid` CTAs (one per SM). Returns the cudaError_t.
+// Cooperative launch on `stream` with `grid` CTAs (one per SM). The kernel's shared-memory limit must have been
+// raised to this footprint by mega_max_grid. Returns the cudaError_t.
 int mega_launch(const MegaParams &p, int grid, cudaStream_t stream);
-// Largest co-resident grid for this shared-memory footprint on the current device.
+// Raises the shared-memory limit of the kernel these parameters select and returns the largest co-resident
+// grid for this footprint on the current device. The answer depends on (kernel, footprint) only: callers cache it.
 int mega_max_grid(const MegaParams &p, size_t smem_bytes, int *err);
+// Which of the kernel's instantiations (head dimension, more than four activation rows) the parameters select: 0..3.
+int mega_kernel_index(const MegaParams &p);
 
 // Verification kernel (verify.cu).
 int verify_launch(const bf16_t *logits, const int32_t *drafts, int B, int K, int V,
                   int32_t *accept_len, int32_t *bonus, int32_t *out_argmax,
                   unsigned long long *keys, uint32_t *counter, uint32_t *status, uint32_t *user_status,
                   int n_sm, cudaStream_t stream);
+
+// Acceptance on token ids (verify.cu): accept_len / bonus from the target's per-row greedy tokens [B][K+1].
+int accept_ids_launch(const int32_t *target_argmax, const int32_t *drafts, int B, int K, int32_t *accept_len, int32_t *bonus,
+                      cudaStream_t stream);
 
 }  // namespace fmtp

@@ -19,8 +19,8 @@
 //     x^2; the consuming phase multiplies its accumulators by rsqrt(mean(x^2)+eps).
 //   * Attention splits the context into fixed 64-token chunks (work items over sequence x KV head
 //     x chunk) whose committed K/V the producers stream through the same ring, fp32 softmax per
-//     chunk, and the CTA that finishes a (sequence, KV head) group last merges its chunks in a
-//     fixed order -- no float atomics anywhere, results are reproducible.
+//     chunk; after a grid barrier a merge phase, spread over all CTAs, combines a head's chunk
+//     partials in ascending order -- no float atomics anywhere, results are reproducible.
 //   * Producers and consumers each walk the phase program from ONE loop with a runtime phase
 //     kind: the code is much larger than the instruction cache, and straight-line code that runs
 //     once per step is fetched from L2 (measured: 3-10x slower than the same code in a loop).
@@ -40,6 +40,7 @@ constexpr uint32_t kDevBadToken = 0x1u, kDevBadPage = 0x2u, kDevBadPos = 0x4u, k
                    kDevAllNan = 0x10u;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait gives up after 2 s
 
+
 enum Kind { PROJ = 0, QKV = 1, OPROJ = 2, GATEUP = 3, DOWN = 4, HEAD = 5, ATTN = 6, EMBED = 7, MERGE = 8, DONE = 9 };
 
 // The phase program of a launch. Draft: K x (PROJ, QKV, ATTN, MERGE, OPROJ, GATEUP, DOWN, HEAD).
@@ -56,6 +57,7 @@ struct Misc {   // small shared-memory block
     float colred[kTileRows][kMaxRows];
     unsigned long long keyred[kConsumerWarps][kMaxRows];
     int tok[kMaxRows];
+    int outrow[kMaxRows];   // where the head publishes activation row r (out_row), set when the head's input is staged
     unsigned long long rowptr[kProducerWarps][32];   // tile row pointers, one line per producer warp
     int flag;
     uint32_t aborted;
@@ -68,12 +70,12 @@ struct Misc {   // small shared-memory block
 constexpr int kProfMarks = 512;
 __device__ unsigned long long g_prof[160][kProfMarks];
 __device__ long long g_wait[160][8];   // consumer wait-full, consumer stage body, producer wait-empty, producer issue
-#define PROF(c) do { if ((c).tid == 0 && (c).nprof < kProfMarks) g_prof[(c).cta][(c).nprof++] = global_timer_ns(); } while (0)
+#define PROF(c, tag) do { if ((c).tid == 0 && (c).nprof < kProfMarks) g_prof[(c).cta][(c).nprof++] = ((unsigned long long)(tag) << 48) | (global_timer_ns() & 0xffffffffffffull); } while (0)
 #define PROF_T0() long long prof_t0 = clock64()
 #define PROF_ACC(c, slot, cond) do { if (cond) { long long prof_t1 = clock64(); (c).pacc[slot] += prof_t1 - prof_t0; prof_t0 = prof_t1; } } while (0)
 #define PROF_FLUSH(c, lo, hi, cond) do { if (cond) for (int q_ = lo; q_ < hi; ++q_) atomicAdd((unsigned long long *)&g_wait[(c).cta][q_], (unsigned long long)(c).pacc[q_]); } while (0)
 #else
-#define PROF(c) do { } while (0)
+#define PROF(c, tag) do { } while (0)
 #define PROF_T0() do { } while (0)
 #define PROF_ACC(c, slot, cond) do { } while (0)
 #define PROF_FLUSH(c, lo, hi, cond) do { } while (0)
@@ -93,6 +95,7 @@ struct Cta {
     unsigned char *scr;    // per-phase scratch (activation staging / attention)
     unsigned char *ring;
     int cta, grid, tid, warp, lane;
+    int R, M;              // activation rows and rows per sequence of the current step (see set_step_rows)
     int slot;              // ring slot of the next stage (same sequence in producer and consumers)
     uint32_t parity;       // mbarrier phase parity of that slot
     uint32_t bar_target;   // grid barrier generation
@@ -143,8 +146,9 @@ __device__ __forceinline__ void grid_barrier(Cta &c) {
     bar_sync(1, kConsumerThreads);
     c.bar_target += (uint32_t)c.grid;
     if (c.tid == 0) {
-        __threadfence();
-        atomicAdd(c.p->s.barrier, 1u);
+        // the arrival is a release at device scope: it orders every write the CTA made before the bar.sync above
+        // (the waiting side reads with acquire), so no separate fences are needed
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(c.p->s.barrier) : "memory");
         if (!aborted(c)) {
             uint32_t n = 0;
             unsigned long long t0 = 0;
@@ -157,7 +161,6 @@ __device__ __forceinline__ void grid_barrier(Cta &c) {
                 }
             }
         }
-        __threadfence();
     }
     bar_sync(1, kConsumerThreads);
 }
@@ -184,8 +187,50 @@ __device__ __forceinline__ void prog_next(const MegaParams &p, Prog &g) {
     }
 }
 
+// ---- rows of a step --------------------------------------------------------------------------
+// Target step: every sequence carries p.M rows at positions L .. L+M-1. Draft: step 0 carries up to p.M
+// "extend" rows per sequence -- the pairs (target hidden state, next token) of the positions committed
+// since the last call, causal among themselves at positions L .. L+n-1, n = n_ext[b] -- of which the
+// last one is draft step 1 (Sec. 2.3 "Drafting phase": step k = 1 runs over the shifted sequence with
+// the target's hidden states); the rows beyond n are padding: computed, never stored or published.
+// Every later step carries one row per sequence at position L + n - 1 + step.
+__device__ __forceinline__ void set_step_rows(Cta &c, int step) {
+    c.M = (c.p->mode == 0 && step > 0) ? 1 : c.p->M;
+    c.R = c.p->B * c.M;
+}
+__device__ __forceinline__ int seq_next(const MegaParams &p, int b) {
+    return p.n_ext ? min(max(p.n_ext[b], 1), p.M) : p.M;
+}
+__device__ __forceinline__ int step_rows(const MegaParams &p, int b, int step) {      // rows of sequence b that count
+    return p.mode == 1 ? p.M : (step == 0 ? seq_next(p, b) : 1);
+}
+// Row of the previous step whose output row r of this draft step continues (step >= 1).
+__device__ __forceinline__ int src_row(const MegaParams &p, int r, int step) {
+    return step == 1 ? r * p.M + seq_next(p, r) - 1 : r;
+}
+// Output index (sequence in a draft, row in a target step) of activation row r, -1 if it publishes nothing.
+__device__ __forceinline__ int out_row(const MegaParams &p, int r, int step) {
+    if (p.mode == 1 || step > 0) return r;
+    const int b = r / p.M;
+    return (r - b * p.M == seq_next(p, b) - 1) ? b : -1;
+}
+
 // ---- phase geometry ----------------------------------------------------------------------
-struct Geom { int rows, K, cap, nks, v0, v1; };
+// rows x K of the phase's matrix, tile height, this CTA's row range, and how K is cut into ring stages:
+// into segments of seglen (the projection has two, one per input vector; every other phase one) and each
+// segment into nks_seg stages of kc elements (the last one shorter). A stage slot holds 32 KB; a phase whose
+// CTAs own at most 25 rows (d x d-like matrices at the 7B width: 24-25 rows per CTA) takes 640 instead of 512
+// elements per stage, so that its stages are as full as those of the 32-row phases: the bytes a CTA has in
+// flight, not its issue rate, set its share of the HBM bandwidth.
+struct Geom { int rows, K, cap, nks, v0, v1, kc, rs, seglen, nks_seg; };
+struct StageK { int koff, klen; };
+__device__ __forceinline__ StageK stage_k(const Geom &g, int ks) {
+    const int seg = ks / g.nks_seg, j = ks - seg * g.nks_seg;
+    StageK s;
+    s.koff = seg * g.seglen + j * g.kc;
+    s.klen = min(g.kc, g.seglen - j * g.kc);
+    return s;
+}
 
 __device__ __forceinline__ Geom geom(const Cta &c, int kind) {
     const MegaParams &p = *c.p;
@@ -199,9 +244,19 @@ __device__ __forceinline__ Geom geom(const Cta &c, int kind) {
         default:     g.rows = p.N;                    g.K = p.d;     break;
     }
     g.cap = (kind == GATEUP) ? kTileRows / 2 : kTileRows;
-    g.nks = (g.K + p.KC - 1) / p.KC;
     g.v0 = (int)(((long long)c.cta * g.rows) / c.grid);
     g.v1 = (int)(((long long)(c.cta + 1) * g.rows) / c.grid);
+    const int per_cta = (g.rows + c.grid - 1) / c.grid;                              // most rows any CTA owns
+    const int stage_rows = (kind == GATEUP) ? 2 * min(g.cap, per_cta) : min(g.cap, per_cta);
+#ifdef FMTP_X_NO640
+    g.kc = p.KC;
+#else
+    g.kc = (p.KC == 512 && stage_rows * 1280 <= p.stage_bytes) ? 640 : p.KC;
+#endif
+    g.rs = g.kc * 2;
+    g.seglen = (kind == PROJ) ? p.d : g.K;
+    g.nks_seg = (g.seglen + g.kc - 1) / g.kc;
+    g.nks = ((kind == PROJ) ? 2 : 1) * g.nks_seg;
     return g;
 }
 
@@ -272,7 +327,11 @@ __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs 
     // producer warp have the parity of pw.
     const uint32_t lane16 = (uint32_t)c.lane * 16u;
     const uint32_t lane16d = (uint32_t)(c.lane ^ ((pw & 1) << 2)) * 16u;
-    const uint32_t rs = (uint32_t)p.row_stride;
+    const uint32_t rs = (uint32_t)g.rs;
+    // weights are read once per step: they enter L2 marked evict-first, so that the stream does not push out what
+    // the step keeps re-reading (activation vectors, partial sums, barrier words and the kernel's own code)
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
     // the loop starts one tile early: iteration t fetches the pointers of tile t + 1
 #pragma unroll 1
     for (int vr0 = g.v0 - g.cap; vr0 < g.v1; vr0 += g.cap) {
@@ -290,12 +349,13 @@ __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs 
             ok = __shfl_sync(0xffffffffu, ok, 0);
             PROF_ACC(c, 2, pw == 0 && c.lane == 0);
             if (!ok) return;   // abort: stop issuing copies
-            const int klen = min(p.KC, g.K - ks * p.KC);
+            const StageK sk = stage_k(g, ks);
+            const int klen = sk.klen;
             const uint32_t dst0 = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + (uint32_t)pw * rs + lane16d;
-            const size_t koff = (size_t)ks * p.KC * 2 + lane16;
-            if (klen == 512) {
-                // 1024 bytes per row: two instructions per row, sixteen per thread, all with their own
-                // address registers
+            const size_t koff = (size_t)sk.koff * 2 + lane16;
+            if (p.KC == 512 && (klen & 31) == 0) {
+                // up to 1536 bytes per row in 512-byte pieces, one instruction per piece and lane, all
+                // with their own address registers (the piece offsets are immediates)
                 uint32_t d[kRowsPerProducer];
                 const unsigned char *q[kRowsPerProducer];
 #pragma unroll
@@ -303,23 +363,28 @@ __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs 
                     q[i] = cur[i] + koff;
                     d[i] = dst0 + (uint32_t)(i * kProducerWarps) * rs;
                 }
+                const int k0 = c.lane * 8;
+                const bool p0 = k0 < klen, p1 = k0 + 256 < klen, p2 = k0 + 512 < klen;
 #pragma unroll
                 for (int i = 0; i < kRowsPerProducer; ++i) {
                     if (cur[i] != nullptr) {
-                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d[i]), "l"(q[i]) : "memory");
-                        asm volatile("cp.async.cg.shared.global [%0+512], [%1+512], 16;" ::"r"(d[i]), "l"(q[i]) : "memory");
+                        if (p0) asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(d[i]), "l"(q[i]), "l"(pol) : "memory");
+                        if (p1) asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0+512], [%1+512], 16, %2;" ::"r"(d[i]), "l"(q[i]), "l"(pol) : "memory");
+                        if (p2) asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0+1024], [%1+1024], 16, %2;" ::"r"(d[i]), "l"(q[i]), "l"(pol) : "memory");
                     }
                 }
             } else {
-                // other stage widths (small or odd geometries): generic loop
-                const int n16 = klen >> 3;
+                // other stage widths (small or odd geometries): generic loop; a row's tail up to the next
+                // multiple of 32 elements is filled with zeros (source size 0: nothing is read)
+                const int n16 = klen >> 3, n16z = ((klen + 31) & ~31) >> 3;
 #pragma unroll
                 for (int i = 0; i < kRowsPerProducer; ++i) {
                     const unsigned char *rp = cur[i];
                     if (rp != nullptr) {
-                        for (int u = c.lane; u < n16; u += 32) {
-                            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst0 + (uint32_t)(i * kProducerWarps) * rs + (uint32_t)(u - c.lane) * 16u),
-                                         "l"(rp + koff + (size_t)(u - c.lane) * 16) : "memory");
+                        for (int u = c.lane; u < n16z; u += 32) {
+                            const uint32_t nbytes = u < n16 ? 16u : 0u;
+                            asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;" ::"r"(dst0 + (uint32_t)(i * kProducerWarps) * rs + (uint32_t)(u - c.lane) * 16u),
+                                         "l"(u < n16 ? rp + koff + (size_t)(u - c.lane) * 16 : rp), "r"(nbytes), "l"(pol) : "memory");
                         }
                     }
                 }
@@ -441,7 +506,8 @@ __device__ __forceinline__ void epilogue(const Cta &c, int kind, EpiCtx &x, cons
                 if (p.out_logits_bf16) p.out_logits_bf16[(size_t)col * p.V + row] = lb;
                 lv = bf16bits_f32(lb);
             } else if (p.out_logits_f32) {
-                p.out_logits_f32[((size_t)col * p.K + x.step) * p.N + row] = v * c.misc->scale0[col];
+                const int orow = c.misc->outrow[col];
+                if (orow >= 0) p.out_logits_f32[((size_t)orow * p.K + x.step) * p.N + row] = v * c.misc->scale0[col];
             }
             unsigned long long key = argmax_key(lv, (uint32_t)id);
             x.best = key > x.best ? key : x.best;
@@ -458,12 +524,15 @@ __device__ __forceinline__ void mma_chunk(float (&acc)[2][2][4], const Frag &f, 
     mma_bf16(acc[0][1], f.u0.z, f.v0.z, f.u0.w, f.v0.w, b.z, b.w);
     mma_bf16(acc[1][1], f.u1.z, f.v1.z, f.u1.w, f.v1.w, b.z, b.w);
 }
-__device__ __forceinline__ Frag load_frag(uint32_t a, uint32_t rs) {
+// Rows g, g + 8, g + 16 and g + 24 of the stage. off24 is 24 * rs, or 0 where row g + 24 lies beyond the rows a
+// stage slot holds at this row stride (25 rows of 640 elements): that row is never a valid tile row, its
+// products are discarded, and the load must stay inside the slot.
+__device__ __forceinline__ Frag load_frag(uint32_t a, uint32_t rs, uint32_t off24) {
     Frag f;
     f.u0 = lds128_u32(a);
     f.v0 = lds128_u32(a + 8 * rs);
     f.u1 = lds128_u32(a + 16 * rs);
-    f.v1 = lds128_u32(a + 24 * rs);
+    f.v1 = lds128_u32(a + off24);
     return f;
 }
 
@@ -495,17 +564,18 @@ __device__ __forceinline__ void park(float (&acc)[2][2][4], float (&acd)[2][2][4
 // warps (warps 0-3 / 4-7) take alternate stages, so each warp does four chunks per barrier wait
 // and two stages are in work at once.
 template <bool two_sets>
-__device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActSrc &act, const int seg_stage, EpiCtx &ex) {
+__device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActSrc &act, EpiCtx &ex) {
     const MegaParams &p = *c.p;
     const Geom geo = geom(c, kind);
-    const int R = p.R;
+    const int R = c.R;
     const int g = c.lane >> 2, t = c.lane & 3;
     const int grp = c.warp >> 2, wi = c.warp & 3;
     const int arow = g >> 1;
     const bf16_t *abase = (g & 1) ? act.lo : act.hi;
     const bool has0 = arow < R, has1 = two_sets && (arow + 4 < R);
     const size_t aoff0 = (size_t)arow * act.stride + t * 8, aoff1 = (size_t)(arow + 4) * act.stride + t * 8;
-    const uint32_t rs = (uint32_t)p.row_stride;
+    const uint32_t rs = (uint32_t)geo.rs;
+    const uint32_t off24 = ((g + 25) * geo.rs <= p.stage_bytes) ? 24u * rs : 0u;
     const uint4 zero = make_uint4(0, 0, 0, 0);
     for (int vr0 = geo.v0; vr0 < geo.v1; vr0 += geo.cap) {
         const int nv = min(geo.cap, geo.v1 - vr0);
@@ -521,10 +591,10 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
                 acc0[i][j] = acd0[i][j] = 0.f;
             }
         // activations read from global memory (the ffn-wide vector of the down projection is not staged
-        // in shared memory): this warp's four B fragments of its next stage are fetched one stage ahead
-        uint4 bnext[4] = {zero, zero, zero, zero};
-        const bool gfast = !two_sets && !act.in_smem && (geo.K % p.KC) == 0 && p.KC == 512;
-        bool moved = false;
+        // in shared memory): this warp's B fragments of its next stage are fetched one stage ahead
+        constexpr int kCpw = 5;                                       // chunks a warp has in a stage: wi, wi + 4, ... (640 / 32 / 4)
+        uint4 bnext[kCpw] = {zero, zero, zero, zero, zero};
+        const bool gfast = !two_sets && !act.in_smem;
         // which half of the warps takes a stage depends only on the stage's index within the phase,
         // never on how many stages the CTA has seen before: the summation order of a row must not
         // depend on the batch or on earlier calls
@@ -532,56 +602,72 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
         if (gfast && has0) {
             const int ks0 = ((stage0 & 1) == grp) ? 0 : 1;          // first stage this warp owns
             if (ks0 < geo.nks) {
+                const StageK s0 = stage_k(geo, ks0);
+                const int n0 = (s0.klen + 31) >> 5;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) bnext[j] = ldcg128(abase + aoff0 + (size_t)ks0 * p.KC + (wi + 4 * j) * 32);
+                for (int j = 0; j < kCpw; ++j)
+                    if (wi + 4 * j < n0) bnext[j] = ldcg128(abase + aoff0 + (size_t)s0.koff + (wi + 4 * j) * 32);
             }
         }
 #pragma unroll 1
         for (int ks = 0; ks < geo.nks; ++ks) {
+            if (kind == PROJ && ks == geo.nks_seg) {
+                // the second input segment starts: every warp parks the sums of the first (whichever stages of it
+                // the warp owned)
+                park<two_sets>(acc, acd, acc0, acd0);
+            }
             if (((stage0 + ks) & 1) == grp) {
                 const int slot = c.slot;
                 const uint32_t parity = c.parity;
                 PROF_T0();
                 wait_bar(c, &c.misc->full[slot], parity);
                 PROF_ACC(c, 0, c.tid == 0);
-                if (kind == PROJ && !moved && ks >= seg_stage) {   // second input segment starts: park the first
-                    moved = true;
-                    park<two_sets>(acc, acd, acc0, acd0);
-                }
-                const int klen = min(p.KC, geo.K - ks * p.KC);
-                const int nchunk = (klen + 31) >> 5;
+
+                const StageK sk = stage_k(geo, ks);
+                const int nchunk = (sk.klen + 31) >> 5;
                 const uint32_t sb = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + t * 16 + g * rs;
                 const int par = g & 1;                    // odd rows: 64-byte halves swapped
-                const size_t kbase = (size_t)ks * p.KC;
-                // chunks wi, wi+4, wi+8, wi+12
-                if (!two_sets && nchunk == 16 && (act.in_smem || gfast)) {
-                    // common case (full 512-wide stage, at most four activation rows): two batches of
-                    // two chunks, all loads of a batch issued before its MMAs
-                    uint4 bq[4];
+                const size_t kbase = (size_t)sk.koff;
+                if (!two_sets && nchunk <= 4 * kCpw && (act.in_smem || gfast)) {
+                    // common case (at most four activation rows): this warp's chunks wi, wi + 4, ... in batches of
+                    // two, all loads of a batch issued before its MMAs
+                    uint4 bq[kCpw];
                     if (act.in_smem) {
                         const uint32_t ab = smem_u32(abase + aoff0 + kbase);
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) bq[j] = has0 ? lds128_u32(ab + (wi + 4 * j) * 64) : zero;
+                        for (int j = 0; j < kCpw; ++j) bq[j] = (has0 && wi + 4 * j < nchunk) ? lds128_u32(ab + (wi + 4 * j) * 64) : zero;
                     } else {
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) bq[j] = bnext[j];
+                        for (int j = 0; j < kCpw; ++j) bq[j] = bnext[j];
                         if (has0 && ks + 2 < geo.nks) {
+                            const StageK s2 = stage_k(geo, ks + 2);
+                            const int n2 = (s2.klen + 31) >> 5;
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) bnext[j] = ldcg128(abase + aoff0 + kbase + 2 * p.KC + (wi + 4 * j) * 32);
+                            for (int j = 0; j < kCpw; ++j)
+                                bnext[j] = (wi + 4 * j < n2) ? ldcg128(abase + aoff0 + (size_t)s2.koff + (wi + 4 * j) * 32) : zero;
                         }
                     }
 #pragma unroll
                     for (int b2 = 0; b2 < 2; ++b2) {
                         const int ch = wi + 8 * b2;
-                        Frag f0 = load_frag(sb + (ch ^ par) * 64, rs);
-                        Frag f1 = load_frag(sb + ((ch + 4) ^ par) * 64, rs);
-                        mma_chunk(acc, f0, bq[2 * b2]);
-                        mma_chunk(acc, f1, bq[2 * b2 + 1]);
+                        if (ch + 4 < nchunk) {
+                            Frag f0 = load_frag(sb + (ch ^ par) * 64, rs, off24);
+                            Frag f1 = load_frag(sb + ((ch + 4) ^ par) * 64, rs, off24);
+                            mma_chunk(acc, f0, bq[2 * b2]);
+                            mma_chunk(acc, f1, bq[2 * b2 + 1]);
+                        } else if (ch < nchunk) {
+                            Frag f0 = load_frag(sb + (ch ^ par) * 64, rs, off24);
+                            mma_chunk(acc, f0, bq[2 * b2]);
+                        }
+                    }
+                    if (wi + 16 < nchunk) {
+                        Frag f0 = load_frag(sb + ((wi + 16) ^ par) * 64, rs, off24);
+                        mma_chunk(acc, f0, bq[4]);
                     }
                 } else {
 #pragma unroll 1
                     for (int ch = wi; ch < nchunk; ch += 4) {
-                        Frag f0 = load_frag(sb + (ch ^ par) * 64, rs);
+                        Frag f0 = load_frag(sb + (ch ^ par) * 64, rs, off24);
                         uint4 b0 = zero, d0 = zero;
                         if (has0) b0 = act.in_smem ? lds128(abase + aoff0 + kbase + ch * 32) : ldcg128(abase + aoff0 + kbase + ch * 32);
                         if (has1) d0 = act.in_smem ? lds128(abase + aoff1 + kbase + ch * 32) : ldcg128(abase + aoff1 + kbase + ch * 32);
@@ -595,8 +681,6 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
             }
             next_stage(c);
         }
-        // a warp whose stages all lay in the first segment parks them now
-        if (kind == PROJ && !moved) park<two_sets>(acc, acd, acc0, acd0);
         // cross-warp reduction in a fixed order
         PROF_T0();
         float *red = c.red + (size_t)c.redbuf * kConsumerWarps * kTileRows * R + (size_t)c.warp * kTileRows * R;
@@ -661,10 +745,12 @@ __device__ __forceinline__ float reduce_partials(const float (&v)[kPartialRegs])
 // Copies R rows of a hi/lo activation pair from global scratch into the shared staging area.
 // `len` elements per row (multiple of 8), rows `stride_s` apart in shared memory, starting at
 // element offset `dst_off`.
+// With remap_step >= 1 row r is read from global row src_row(r, remap_step): the projection of draft step 1
+// continues each sequence's last extend row.
 __device__ __forceinline__ void stage_hilo(const Cta &c, const bf16_t *ghi, const bf16_t *glo, int gstride, int len, bf16_t *shi,
-                                           bf16_t *slo, int sstride, int dst_off) {
+                                           bf16_t *slo, int sstride, int dst_off, int remap_step = 0) {
     const int per_row = len / 8;
-    const int total = c.p->R * per_row;
+    const int total = c.R * per_row;
     // four units per thread and round: eight loads in flight before the first store waits
 #pragma unroll 1
     for (int i0 = c.tid; i0 < total; i0 += 4 * kConsumerThreads) {
@@ -673,8 +759,9 @@ __device__ __forceinline__ void stage_hilo(const Cta &c, const bf16_t *ghi, cons
         for (int q = 0; q < 4; ++q) {
             int i = min(i0 + q * kConsumerThreads, total - 1);
             int r = i / per_row, k = (i - r * per_row) * 8;
-            a[q] = ldcg128(ghi + (size_t)r * gstride + k);
-            b[q] = ldcg128(glo + (size_t)r * gstride + k);
+            const int rs = remap_step > 0 ? src_row(*c.p, r, remap_step) : r;
+            a[q] = ldcg128(ghi + (size_t)rs * gstride + k);
+            b[q] = ldcg128(glo + (size_t)rs * gstride + k);
         }
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -714,7 +801,7 @@ __device__ __forceinline__ void flush_sq(const Cta &c, const SqAcc &q, float *tb
 }
 
 // ---- attention phase -------------------------------------------------------------------------
-// Rows r = b*M + m sit at position seq_lens[b] + posoff + m. The context of a sequence is cut
+// Rows r = b*M + m sit at position step_base(b) + m (see "rows of a step"). The context of a sequence is cut
 // into fixed 64-token chunks from position 0; a work item is (sequence, KV head, chunk) and items
 // are dealt round-robin over the CTAs. A row's result therefore depends on its own position only.
 //
@@ -733,10 +820,10 @@ __device__ __forceinline__ void flush_sq(const Cta &c, const SqAcc &q, float *tb
 // The loop over query heads is a real loop (not unrolled) to keep this once-per-step code small.
 template <int DH>
 __device__ __forceinline__ void attn_rows(Cta &c, bf16_t *sk, const bf16_t *sv, const float *qs,
-                                          int b, int kvh, int chunk, int base, int max_tokens) {
+                                          int b, int kvh, int chunk, int base, int max_tokens, int rows) {
     const MegaParams &p = *c.p;
     constexpr int SEG = DH / 4, EPL = DH / 32, wstride = DH + 2;
-    const int Gq = p.Hq / p.Hkv, M = p.M;
+    const int Gq = p.Hq / p.Hkv, M = c.M;
     const int c0 = chunk * kAttnChunk;
     const int tl = c.warp * 8;                       // first token (within the chunk) of this warp
     // lanes of a quarter-warp share `part`, so a 128-bit query load is one broadcast per quarter
@@ -772,10 +859,10 @@ __device__ __forceinline__ void attn_rows(Cta &c, bf16_t *sk, const bf16_t *sv, 
     // wp[8 warps][Gq][DH + 2] (o, m, l) and the merge weights behind them
     bar_sync(1, kConsumerThreads);
     float *wp = reinterpret_cast<float *>(sk);
-    PROF(c);
+    PROF(c, ATTN * 8 + 6);
 #pragma unroll 1
     for (int m = 0; m < M; ++m) {
-        const int npos = min(base + m, max_tokens - 1);   // last visible position of this row
+        const int npos = min(base + min(m, rows - 1), max_tokens - 1);   // last visible position of this row
         const int nvis = min(8, npos - (c0 + tl) + 1);    // visible tokens of this warp (may be <= 0)
 #pragma unroll 1
         for (int h = 0; h < Gq; ++h) {
@@ -822,9 +909,7 @@ __device__ __forceinline__ void attn_rows(Cta &c, bf16_t *sk, const bf16_t *sv, 
             for (int e = 0; e < EPL; ++e) w[e0 + e] = o[e];
             if (c.lane == 0) { w[DH] = mx; w[DH + 1] = sm; }
         }
-        PROF(c);
         bar_sync(1, kConsumerThreads);
-        PROF(c);
         // ---- merge the 8 warps (fixed order) -> chunk partial in global memory.
         // weight of warp w for head h: thread (h, w) computes it once
         float *fw = wp + (size_t)kConsumerWarps * Gq * wstride;      // [Gq][8] weights, then [Gq][2] (m, l)
@@ -838,7 +923,6 @@ __device__ __forceinline__ void attn_rows(Cta &c, bf16_t *sk, const bf16_t *sv, 
             if (w == 0) fw[Gq * kConsumerWarps + 2 * h] = mx;
         }
         bar_sync(1, kConsumerThreads);
-        PROF(c);
         for (int i = c.tid; i < Gq * DH; i += kConsumerThreads) {
             const int h = i / DH, e = i - h * DH;
             float ov = 0.f, l = 0.f;
@@ -858,35 +942,53 @@ __device__ __forceinline__ void attn_rows(Cta &c, bf16_t *sk, const bf16_t *sv, 
     }
 }
 
-struct AttnItem { int b, kvh, chunk, Lb, nch; };
+struct AttnItem { int b, kvh, chunk, Lb, nch, base, rows; };
 
-__device__ __forceinline__ int attn_total(const MegaParams &p, const KvPtrs &kv, int posoff) {
+// Positions the cache of `kv` has slots for (positions beyond are flagged, never touched), the committed
+// length of a sequence brought into that range, the position of its row 0 in `step` and the chunks its
+// rows can see: every index the attention and merge phases form from seq_lens stays inside the block
+// table and the partial buffer, whatever the caller put there.
+__device__ __forceinline__ int kv_max_tokens(const MegaParams &p, const KvPtrs &kv) { return min(kv.max_pages * p.page, p.max_ctx); }
+__device__ __forceinline__ int committed_len(const MegaParams &p, const KvPtrs &kv, int b) {
+    return min(max(kv.seq_lens[b], 0), kv_max_tokens(p, kv));
+}
+__device__ __forceinline__ int step_base(const MegaParams &p, const KvPtrs &kv, int b, int step) {
+    return committed_len(p, kv, b) + ((p.mode == 0 && step > 0) ? seq_next(p, b) - 1 + step : 0);
+}
+__device__ __forceinline__ int visible_chunks(const MegaParams &p, const KvPtrs &kv, int b, int step) {
+    const int last = min(step_base(p, kv, b, step) + step_rows(p, b, step) - 1, kv_max_tokens(p, kv) - 1);
+    return min(last / kAttnChunk + 1, p.max_chunks);
+}
+
+__device__ __forceinline__ int attn_total(const MegaParams &p, const KvPtrs &kv, int step) {
     int total = 0;
-    for (int b = 0; b < p.B; ++b) total += p.Hkv * ((kv.seq_lens[b] + posoff + p.M - 1) / kAttnChunk + 1);
+    for (int b = 0; b < p.B; ++b) total += p.Hkv * visible_chunks(p, kv, b, step);
     return total;
 }
-__device__ __forceinline__ AttnItem attn_item(const MegaParams &p, const KvPtrs &kv, int posoff, int item) {
+__device__ __forceinline__ AttnItem attn_item(const MegaParams &p, const KvPtrs &kv, int step, int item) {
     AttnItem it;
-    int b = 0, rem = item, Lb = 0, nch = 1;
+    int b = 0, rem = item, nch = 1;
     for (; b < p.B; ++b) {
-        Lb = kv.seq_lens[b];
-        nch = (Lb + posoff + p.M - 1) / kAttnChunk + 1;
+        nch = visible_chunks(p, kv, b, step);
         if (rem < p.Hkv * nch) break;
         rem -= p.Hkv * nch;
     }
-    it.b = b; it.Lb = Lb; it.nch = nch;
+    if (b >= p.B) b = p.B - 1;
+    it.b = b; it.Lb = committed_len(p, kv, b); it.nch = nch;
+    it.base = step_base(p, kv, b, step);
+    it.rows = step_rows(p, b, step);
     it.kvh = rem / nch;
     it.chunk = rem - it.kvh * nch;
     return it;
 }
 
-__device__ __forceinline__ void produce_attention(Cta &c, const KvPtrs &kv, int posoff) {
+__device__ __forceinline__ void produce_attention(Cta &c, const KvPtrs &kv, int step) {
     const MegaParams &p = *c.p;
     const int ptid = c.tid - kConsumerThreads;               // 0 .. 127
     const int upt = p.dh >> 3;                                // 16-byte units per token row
-    const int total = attn_total(p, kv, posoff);
+    const int total = attn_total(p, kv, step);
     for (int item = c.cta; item < total; item += c.grid) {
-        const AttnItem it = attn_item(p, kv, posoff, item);
+        const AttnItem it = attn_item(p, kv, step, item);
         const int c0 = it.chunk * kAttnChunk;
         const int n_old = max(0, min(kAttnChunk, it.Lb - c0));   // committed tokens of this chunk
         const int32_t *bt = kv.block_table + (size_t)it.b * kv.max_pages;
@@ -928,20 +1030,21 @@ __device__ __forceinline__ void produce_attention(Cta &c, const KvPtrs &kv, int 
 }
 
 template <int DH>
-__device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int posoff) {
+__device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int step) {
     const MegaParams &p = *c.p;
     constexpr int dh = DH, half = DH >> 1;
-    const int Gq = p.Hq / p.Hkv, M = p.M;
+    const int Gq = p.Hq / p.Hkv, M = c.M;
     float *qs = reinterpret_cast<float *>(c.scr);
     const float qscale = rsqrtf((float)dh);
     const int max_tokens = min(kv.max_pages * p.page, p.max_ctx);   // positions beyond are flagged, not touched
     const int upt = dh >> 3;
 
-    const int total = attn_total(p, kv, posoff);
+    const int total = attn_total(p, kv, step);
     for (int item = c.cta; item < total; item += c.grid) {
-        const AttnItem it = attn_item(p, kv, posoff, item);
+        const AttnItem it = attn_item(p, kv, step, item);
         const int b = it.b, kvh = it.kvh, chunk = it.chunk, Lb = it.Lb;
-        const int base = Lb + posoff;              // position of row m = 0
+        const int base = it.base;                  // position of row m = 0
+        const int rows = it.rows;                  // rows of this sequence that count (the rest is padding)
         const int c0 = chunk * kAttnChunk;
         const int32_t *bt = kv.block_table + (size_t)b * kv.max_pages;
         const int slot = c.slot;
@@ -953,7 +1056,7 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
         for (int i = c.tid; i < M * Gq * half; i += kConsumerThreads) {
             int qi = i / half, e = i - qi * half;
             int m = qi / Gq, hq = kvh * Gq + (qi - m * Gq);
-            int r = b * M + m, pos = base + m;
+            int r = b * M + m, pos = base + min(m, rows - 1);
             if (pos >= max_tokens) pos = max_tokens - 1;
             const float *q = p.s.qkv + (size_t)r * (p.qdim + 2 * p.kvdim) + hq * dh;
             float x = ldcg_f32(q + e), y = ldcg_f32(q + e + half);
@@ -961,9 +1064,9 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
             qs[qi * dh + e] = (x * cs - y * sn) * qscale;
             qs[qi * dh + e + half] = (y * cs + x * sn) * qscale;
         }
-        PROF(c);
+        PROF(c, ATTN * 8 + 3);
         wait_bar(c, &c.misc->full[slot], parity);
-        PROF(c);
+        PROF(c, ATTN * 8 + 4);
         // -- positions written earlier in this launch (previous draft steps): from the pages
         {
             const int lo = max(Lb, c0), hi = min(min(base, c0 + kAttnChunk), max_tokens);
@@ -979,6 +1082,7 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
         // -- this call's rows: rotate, round to bf16, put into the stage and append to the cache
         for (int i = c.tid; i < M * half; i += kConsumerThreads) {
             int m = i / half, e = i - m * half;
+            if (m >= rows) continue;                              // padding row: nothing to store
             int r = b * M + m, pos = base + m;
             if (pos >= max_tokens) { if (chunk == 0) raise(c, kDevBadPos); continue; }
             if (pos < c0 || pos >= c0 + kAttnChunk) continue;     // another chunk's item owns it
@@ -999,10 +1103,9 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
             kv.v_pages[o + e + half] = v1;
         }
         bar_sync(1, kConsumerThreads);
-        PROF(c);
+        PROF(c, ATTN * 8 + 5);
 
-        attn_rows<DH>(c, sk, sv, qs, b, kvh, chunk, base, max_tokens);
-        PROF(c);
+        attn_rows<DH>(c, sk, sv, qs, b, kvh, chunk, base, max_tokens, rows);
         // the stage is free again (all consumer warps passed the barrier at the end of attn_rows)
         if (c.warp < kConsumerWarps / 2 && c.lane == 0) mbar_arrive(&c.misc->empty[slot]);
         next_stage(c);
@@ -1016,23 +1119,23 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int po
 // dealt round-robin over the CTAs. Thread = (output element, chunk group): it adds its chunks in
 // ascending order, the chunk groups are then added in ascending order, so the summation order
 // depends only on the number of visible chunks, i.e. on the row's position.
-__device__ __forceinline__ void merge_phase(Cta &c, const KvPtrs &kv, int posoff) {
+__device__ __forceinline__ void merge_phase(Cta &c, const KvPtrs &kv, int step) {
     const MegaParams &p = *c.p;
-    const int dh = p.dh, M = p.M, wstride = dh + 2;
+    const int dh = p.dh, M = c.M, wstride = dh + 2;
     const int qe = dh >> 2;                          // output elements per unit (32 or 16)
     const int ncg = kConsumerThreads / qe;           // chunk groups (8 or 16)
     const int max_tokens = min(kv.max_pages * p.page, p.max_ctx);
     float *ms = reinterpret_cast<float *>(c.scr);    // [max_chunks] chunk maxima
     float *ls = ms + p.max_chunks;                   // [max_chunks] chunk denominators
     float *red = ls + p.max_chunks;                  // [ncg][qe + 1] partial sums (+ denominators)
-    const int units = p.R * p.Hq * 4;
+    const int units = c.R * p.Hq * 4;
     const int el = c.tid % qe, cg = c.tid / qe;
     for (int u = c.cta; u < units; u += c.grid) {
         const int r = u / (p.Hq * 4), rem = u - r * (p.Hq * 4);
         const int hq = rem >> 2, e = (rem & 3) * qe + el;
         const int b = r / M, m = r - b * M;
-        const int pos = min(kv.seq_lens[b] + posoff + m, max_tokens - 1);
-        const int ncm = pos / kAttnChunk + 1;        // chunks visible to this row
+        const int pos = min(step_base(p, kv, b, step) + min(m, step_rows(p, b, step) - 1), max_tokens - 1);
+        const int ncm = min(pos / kAttnChunk + 1, p.max_chunks);        // chunks visible to this row
         const float *src = p.s.att_part + ((size_t)r * p.Hq + hq) * p.max_chunks * wstride;
         for (int i = c.tid; i < ncm; i += kConsumerThreads) {
             ms[i] = ldcg_f32(src + (size_t)i * wstride + dh);
@@ -1108,15 +1211,16 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
     const unsigned long long prof_n0 = global_timer_ns();
 #endif
     const bool is_producer = (c.warp >= kConsumerWarps);
-    const int R = p.R;
     const int n_steps = (p.mode == 0) ? p.K : 1;
+    set_step_rows(c, 0);
 
     if (is_producer) {
         setmaxnreg_dec<kProducerRegs>();
         // ---------------- producers: the weight / KV stream of every phase, in program order
         Prog g;
         for (prog_begin(p, g); g.kind != DONE; prog_next(p, g)) {
-            if (g.kind == ATTN) produce_attention(c, p.kvs[g.layer], (p.mode == 0) ? g.step : 0);
+            set_step_rows(c, g.step);
+            if (g.kind == ATTN) produce_attention(c, p.kvs[g.layer], g.step);
             else if (g.kind != EMBED && g.kind != MERGE) produce_phase(c, g.kind, p.layers[g.layer]);
         }
         cp_async_wait_all();   // every copy this thread issued has landed before the CTA may exit
@@ -1133,6 +1237,8 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
 #pragma unroll 1
     for (prog_begin(p, g); g.kind != DONE; prog_next(p, g)) {
         const int kind = g.kind, step = g.step;
+        set_step_rows(c, step);
+        const int R = c.R;
         const LayerPtrs &L = p.layers[g.layer];
         const bool last_layer = (p.mode == 0) || (g.layer + 1 == p.n_layers);
         ex.sq.a = 0.f; ex.sq.b = 0.f;
@@ -1140,16 +1246,16 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
         ex.step = step;
         ex.to_next_layer = (p.mode == 1) && !last_layer;
         ex.gnext = ex.to_next_layer ? p.layers[g.layer + 1].g_in : p.g_final;
-        PROF(c);
+        PROF(c, kind * 8);
         if (kind == ATTN) {
-            attention_phase<DH>(c, p.kvs[g.layer], (p.mode == 0) ? step : 0);
-            PROF(c);
+            attention_phase<DH>(c, p.kvs[g.layer], step);
+            PROF(c, kind * 8 + 2);
             grid_barrier(c);
             continue;
         }
         if (kind == MERGE) {
-            merge_phase(c, p.kvs[g.layer], (p.mode == 0) ? step : 0);
-            PROF(c);
+            merge_phase(c, p.kvs[g.layer], step);
+            PROF(c, kind * 8 + 2);
             grid_barrier(c);
             continue;
         }
@@ -1168,7 +1274,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                 }
             }
             flush_sq(c, ex.sq, p.s.ssA, nullptr);
-            PROF(c);
+            PROF(c, kind * 8 + 2);
             grid_barrier(c);
             continue;
         }
@@ -1178,18 +1284,20 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
         const int st = ((klen + 31) & ~31) + 32;      // +64 B: rows land in different banks
         bf16_t *a_hi = s_hi, *a_lo = s_hi + (size_t)R * st;
         ActSrc act{a_hi, a_lo, st, true};
-        int seg = 0;
         if (kind == PROJ) {
             // ---- x0 = W_p [ rms(h) ; rms(Emb(tok)) ]
-            seg = p.d / p.KC;
             // loads that do not depend on each other are issued first: the previous step's argmax key,
             // the partial sums that normalise the recursed state, and that state itself
             unsigned long long key = 0ull;
             if (step > 0 && c.tid < R) key = ldcg_u64(p.s.keys + (size_t)(step - 1) * kMaxRows + c.tid);
             float pvc[kPartialRegs], pvd[kPartialRegs];
             const bool renorm = step > 0 && c.warp < R;
-            if (renorm) { load_partials(c, p.s.ssC, c.warp, pvc); load_partials(c, p.s.ssD, c.warp, pvd); }
-            if (step > 0) stage_hilo(c, p.s.actR_hi, p.s.actR_lo, p.dp, p.d, a_hi, a_lo, st, 0);
+            if (renorm) {
+                const int col = src_row(p, c.warp, step);      // step 1 continues each sequence's last extend row
+                load_partials(c, p.s.ssC, col, pvc);
+                load_partials(c, p.s.ssD, col, pvd);
+            }
+            if (step > 0) stage_hilo(c, p.s.actR_hi, p.s.actR_lo, p.dp, p.d, a_hi, a_lo, st, 0, step);
             if (renorm) {
                 // recursed state: h = (x2*g_final) * s_x; rms(h) adds s_h = rsqrt(s_x^2 * mean((x2 g)^2) + eps)
                 float sx = rsqrtf(reduce_partials(pvc) / (float)p.d + p.eps);
@@ -1198,8 +1306,10 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
             }
             if (c.tid < R) {
                 int tok;
-                if (step == 0) tok = p.tokens[c.tid];
-                else {
+                if (step == 0) {
+                    const int b = c.tid / p.M;         // a padding row's token is never looked at
+                    tok = (c.tid - b * p.M < seq_next(p, b)) ? p.tokens[c.tid] : 0;
+                } else {
                     if ((key >> 32) == 0ull) raise(c, kDevAllNan);
                     tok = (int)argmax_key_id(key);
                     if (c.cta == 0) p.out_tokens[(size_t)c.tid * p.K + (step - 1)] = tok;
@@ -1266,27 +1376,30 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
             float pv[kPartialRegs];
             const bool norm = sstab != nullptr && c.warp < R;
             if (norm) load_partials(c, sstab, c.warp, pv);       // in flight while the vector is staged
-            if (kind == DOWN && !p.stage_F_in_smem) act = ActSrc{ghi, glo, gstride, false};
+            if (kind == DOWN) act = ActSrc{ghi, glo, gstride, false};     // read from global memory inside the loop
             else stage_hilo(c, ghi, glo, gstride, glen, a_hi, a_lo, st, 0);
             if (norm) {
                 float sc = rsqrtf(reduce_partials(pv) / (float)p.d + p.eps);
                 if (c.lane == 0) c.misc->scale0[c.warp] = sc;
             }
         }
+        if (kind == HEAD && c.tid < R) c.misc->outrow[c.tid] = out_row(p, c.tid, step);
         bar_sync(1, kConsumerThreads);
         if (kind == HEAD && p.out_h) {   // every CTA writes its slice of the post-final-norm hidden state
             int r0 = (int)(((long long)c.cta * p.d) / c.grid), r1 = (int)(((long long)(c.cta + 1) * p.d) / c.grid);
             for (int i = c.tid; i < R * (r1 - r0); i += kConsumerThreads) {
                 int r = i / (r1 - r0), k = r0 + (i - r * (r1 - r0));
+                const int orow = c.misc->outrow[r];
+                if (orow < 0) continue;                    // an extend row that is not its sequence's last
                 float y = bf16bits_f32(a_hi[(size_t)r * st + k]) + bf16bits_f32(a_lo[(size_t)r * st + k]);
-                size_t o = (p.mode == 0) ? ((size_t)r * p.K + step) * p.d + k : (size_t)r * p.d + k;
+                size_t o = (p.mode == 0) ? ((size_t)orow * p.K + step) * p.d + k : (size_t)orow * p.d + k;
                 p.out_h[o] = f32_bf16bits(y * c.misc->scale0[r]);
             }
         }
-        PROF(c);
+        PROF(c, kind * 8 + 1);
 
         // ============ ... stream the weights ...
-        consume_tiles<TWO>(c, kind, act, seg, ex);
+        consume_tiles<TWO>(c, kind, act, ex);
 
         // ============ ... and publish what the next phase needs besides the vector
         if (kind == PROJ) flush_sq(c, ex.sq, p.s.ssA, nullptr);
@@ -1304,14 +1417,15 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
             if (c.tid < R) {
                 unsigned long long m = 0ull;
                 for (int w = 0; w < kConsumerWarps; ++w) m = c.misc->keyred[w][c.tid] > m ? c.misc->keyred[w][c.tid] : m;
-                if (m != 0ull) atomicMax(p.s.keys + (size_t)step * kMaxRows + c.tid, m);
+                const int orow = c.misc->outrow[c.tid];
+                if (m != 0ull && orow >= 0) atomicMax(p.s.keys + (size_t)step * kMaxRows + orow, m);
             }
             ex.best = 0ull;
         }
-        PROF(c);
+        PROF(c, kind * 8 + 2);
         grid_barrier(c);
     }
-    PROF(c);
+    PROF(c, DONE * 8);
 
     PROF_FLUSH(c, 0, 2, c.tid == 0);
     PROF_FLUSH(c, 4, 5, c.tid == 0);
@@ -1322,7 +1436,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
     }
 #endif
     // ============ publish the last step's tokens and the status word
-    if (c.cta == 0 && c.tid < R) {
+    if (c.cta == 0 && c.tid < ((p.mode == 0) ? p.B : p.R)) {
         int last = n_steps - 1;
         unsigned long long key = ldcg_u64(p.s.keys + (size_t)last * kMaxRows + c.tid);
         if ((key >> 32) == 0ull) raise(c, kDevAllNan);
@@ -1373,6 +1487,8 @@ const void *kernel_for(int R, int dh) {
 }
 }  // namespace
 
+int mega_kernel_index(const MegaParams &p) { return (p.dh == 128 ? 2 : 0) + (p.R > 4 ? 1 : 0); }
+
 int mega_max_grid(const MegaParams &p, size_t smem_bytes, int *err) {
     int dev = 0, sms = 0, per_sm = 0;
     const void *fn = kernel_for(p.R, p.dh);
@@ -1388,11 +1504,8 @@ int mega_max_grid(const MegaParams &p, size_t smem_bytes, int *err) {
 int mega_launch(const MegaParams &p, int grid, cudaStream_t stream) {
     size_t smem = mega_smem_bytes(p);
     const void *fn = kernel_for(p.R, p.dh);
-    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return (int)e;
     void *args[] = {const_cast<MegaParams *>(&p)};
-    e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kThreads), args, smem, stream);
-    return (int)e;
+    return (int)cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kThreads), args, smem, stream);
 }
 
 }  // namespace fmtp

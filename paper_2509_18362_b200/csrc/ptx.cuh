@@ -1,7 +1,7 @@
-// Thin wrappers over the sm_100a PTX this library relies on: mbarriers, 1-D bulk async
-// copies (TMA engine, no tensor map), bf16 tensor-core MMA, cache-qualified loads and
-// bounded waits. Every wait in this file gives up after a fixed number of polls and reports
-// it, so a logic error can never hang the device.
+// Thin wrappers over the sm_100a PTX this library relies on: mbarriers, 16-byte asynchronous copies
+// whose completion is counted on an mbarrier, bf16 tensor-core MMA, cache-qualified loads, named
+// barriers and the packed argmax key. The waits themselves (bounded by the global timer, reporting
+// through a status word) live next to the kernels that use them.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -39,35 +39,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 
-// ---- bulk async copy global -> shared, completion counted on an mbarrier ----------------
-// dst, src 16-byte aligned; bytes a multiple of 16.
-__device__ __forceinline__ void bulk_g2s(void *dst_smem, const void *src_gmem, uint32_t bytes, uint64_t *bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_u32(dst_smem)),
-                 "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
-// Same with an L2 eviction-priority hint (created by make_policy_*).
-__device__ __forceinline__ void bulk_g2s_hint(void *dst_smem, const void *src_gmem, uint32_t bytes, uint64_t *bar,
-                                              uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::
-            "r"(smem_u32(dst_smem)),
-        "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
-        : "memory");
-}
-__device__ __forceinline__ uint64_t make_policy_evict_first() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-__device__ __forceinline__ void bulk_prefetch_l2(const void *src_gmem, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src_gmem), "r"(bytes) : "memory");
-}
 // ---- 16-byte asynchronous copies global -> shared through the load/store path ----------------
-// (measured on B200: this path sustains ~65 GB/s per SM against ~47 GB/s for bulk copies, and has
-// no per-request cost, so any row length and any shared-memory layout stream at full speed; its
-// throughput is limited per issuing warp, so at least eight warps must issue)
+// (measured on B200: this path sustains ~65 GB/s per SM against ~47 GB/s for 1-D bulk copies, and has
+// no per-request cost, so any row length and any shared-memory layout stream at full speed)
 __device__ __forceinline__ void cp_async16(void *dst_smem, const void *src_gmem) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src_gmem) : "memory");
 }
@@ -107,11 +81,6 @@ __device__ __forceinline__ uint4 ldcg128(const void *p) {
     asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
-__device__ __forceinline__ uint2 ldcg64(const void *p) {
-    uint2 v;
-    asm volatile("ld.global.cg.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
-    return v;
-}
 __device__ __forceinline__ float ldcg_f32(const float *p) {
     float v;
     asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
@@ -120,11 +89,6 @@ __device__ __forceinline__ float ldcg_f32(const float *p) {
 __device__ __forceinline__ uint32_t ldcg_u32(const void *p) {
     uint32_t v;
     asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
-}
-__device__ __forceinline__ uint16_t ldcg_u16(const void *p) {
-    uint16_t v;
-    asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(v) : "l"(p));
     return v;
 }
 __device__ __forceinline__ unsigned long long ldcg_u64(const void *p) {

@@ -21,7 +21,9 @@
 // Every wait is time-bounded; on expiry the CTA raises the timeout flag, drains and returns.
 #pragma once
 #include "umma.cuh"
+#include "batched.cuh"
 #include <cuda.h>
+#include <cstring>
 
 namespace fmtp {
 
@@ -450,7 +452,7 @@ inline int gemm_encode_xmap(CUtensorMap *map, const bf16_t *x, int ldx, int K, i
 
 // Launches the GEMM on `stream` with one CTA per SM (fewer when there are fewer work items).
 // Returns the cudaError_t of the launch.
-inline int skinny_gemm_launch(GemmArgs g, int n_sm, int smem_optin, cudaStream_t stream) {
+inline int skinny_gemm_launch(GemmArgs g, int n_sm, int smem_optin, cudaStream_t stream, TmapCache *cache) {
     const int avail = smem_optin - 1024 - (int)sizeof(GemmSmem);
     const int kbb = gemm_kblock_bytes(g.NB);
     // blocks per stage: as many as still leave a ring of three stages
@@ -465,11 +467,28 @@ inline int skinny_gemm_launch(GemmArgs g, int n_sm, int smem_optin, cudaStream_t
     const int grid = n_items < n_sm ? n_items : n_sm;
     void (*kern)(const GemmArgs, const CUtensorMap) = ka == 4 ? skinny_gemm_kernel<4> : ka == 2 ? skinny_gemm_kernel<2> : skinny_gemm_kernel<1>;
     if (ka != 1 && ka != 2 && ka != 4) return (int)cudaErrorInvalidConfiguration;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return (int)e;
+    cudaError_t e = cudaSuccess;
+    int &limit = cache->gemm_smem[ka == 4 ? 2 : ka == 2 ? 1 : 0];
+    if ((int)smem > limit) {                  // raise the kernel's shared-memory limit once per footprint
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+        limit = (int)smem;
+    }
+    // the operand's tensor map depends on (address, row pitch, K, rows) only: encoded once, then reused
     CUtensorMap xmap;
-    int rc = gemm_encode_xmap(&xmap, g.x, g.ldx, g.K, g.NB);
-    if (rc) return rc;
+    static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+    TmapEntry *hit = nullptr;
+    for (int i = 0; i < cache->n; ++i)
+        if (cache->e[i].x == g.x && cache->e[i].ldx == g.ldx && cache->e[i].K == g.K && cache->e[i].NB == g.NB) { hit = &cache->e[i]; break; }
+    if (hit) std::memcpy(&xmap, hit->map, sizeof(xmap));
+    else {
+        int rc = gemm_encode_xmap(&xmap, g.x, g.ldx, g.K, g.NB);
+        if (rc) return rc;
+        const int cap = (int)(sizeof(cache->e) / sizeof(cache->e[0]));
+        TmapEntry &dst = cache->e[cache->n < cap ? cache->n++ : (cache->next++ % cap)];
+        dst.x = g.x; dst.ldx = g.ldx; dst.K = g.K; dst.NB = g.NB;
+        std::memcpy(dst.map, &xmap, sizeof(xmap));
+    }
     e = launch_chained(kern, dim3(grid), dim3(kGemmThreads), smem, stream, g, xmap);
     return (int)e;
 }

@@ -114,7 +114,26 @@ __global__ void __launch_bounds__(kVThreads) verify_kernel(const bf16_t *__restr
     if (threadIdx.x == 0) *counter = 0u;
 }
 
+// The acceptance rule alone, for callers that already hold the target's greedy token of every row
+// (fastmtp_target_step's out_argmax): one thread per sequence walks its K drafts.
+__global__ void accept_ids_kernel(const int32_t *__restrict__ target_argmax, const int32_t *__restrict__ drafts, int B, int K,
+                                  int32_t *accept_len, int32_t *bonus) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int32_t *g = target_argmax + (size_t)b * (K + 1);
+    int a = 0;
+    while (a < K && drafts[(size_t)b * K + a] == g[a]) ++a;
+    accept_len[b] = a;
+    bonus[b] = g[a];
+}
+
 }  // namespace
+
+int accept_ids_launch(const int32_t *target_argmax, const int32_t *drafts, int B, int K, int32_t *accept_len, int32_t *bonus,
+                      cudaStream_t stream) {
+    accept_ids_kernel<<<(B + 127) / 128, 128, 0, stream>>>(target_argmax, drafts, B, K, accept_len, bonus);
+    return (int)cudaGetLastError();
+}
 
 int verify_launch(const bf16_t *logits, const int32_t *drafts, int B, int K, int V, int32_t *accept_len,
                   int32_t *bonus, int32_t *out_argmax, unsigned long long *keys, uint32_t *counter,

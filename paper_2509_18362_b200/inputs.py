@@ -24,7 +24,7 @@ import numpy as np
 
 __all__ = [
     "Shape", "TINY", "QWEN7B", "rng", "f32_to_bf16_bits", "bf16_bits_to_f32",
-    "normal_bf16", "mtp_weights", "layer_weights", "target_weights",
+    "normal_bf16", "mtp_weights", "layer_weights", "target_weights", "target_weights_cuda",
     "subset_uniform", "subset_zipf", "context_lengths", "paged_kv",
     "hidden_bf16", "token_ids", "verify_case", "verify_logits_natural",
 ]
@@ -143,6 +143,48 @@ def target_weights(s: Shape, seed: int, embed=None, lm_head=None) -> dict:
         "g_final": _gain(seed, "tgt.g_final", s.d),
         "layers": [layer_weights(s, seed, f"tgt.layer{i}") for i in range(s.n_layers)],
     }
+
+
+def target_weights_cuda(s: Shape, seed: int, device: str = "cuda"):
+    """A random-init target decoder drawn on the GPU, for depths at which the host generators take minutes
+    (28 layers of the 7B-class shape are 7.6e9 values): every tensor ~N(0, 0.02) in bf16 (gains 1 + N(0, 0.02)) from
+    a torch CUDA generator seeded by (seed, tensor name). Returns (device, host): the same bits as a nested dict of
+    torch bf16 tensors on the device and as numpy uint16 bit patterns on the host, laid out like target_weights().
+    The values differ from target_weights(s, seed): another generator, the same distribution."""
+    import torch
+
+    def draw(tag, shape, std, mean=0.0):
+        g = torch.Generator(device=device)
+        g.manual_seed((seed * 1000003 + zlib.crc32(tag.encode())) & 0x7FFFFFFFFFFFFFFF)
+        t = torch.empty(shape, dtype=torch.float32, device=device).normal_(mean, std, generator=g).to(torch.bfloat16)
+        return t
+
+    def layer(prefix):
+        return {
+            "g_in": draw(prefix + ".g_in", (s.d,), 0.02, 1.0),
+            "wq": draw(prefix + ".wq", (s.q_dim, s.d), 0.02),
+            "wk": draw(prefix + ".wk", (s.kv_dim, s.d), 0.02),
+            "wv": draw(prefix + ".wv", (s.kv_dim, s.d), 0.02),
+            "wo": draw(prefix + ".wo", (s.d, s.q_dim), 0.02),
+            "g_post": draw(prefix + ".g_post", (s.d,), 0.02, 1.0),
+            "w_gate": draw(prefix + ".w_gate", (s.ffn, s.d), 0.02),
+            "w_up": draw(prefix + ".w_up", (s.ffn, s.d), 0.02),
+            "w_down": draw(prefix + ".w_down", (s.d, s.ffn), 0.02),
+        }
+
+    dev = {
+        "embed": draw("embed", (s.vocab, s.d), 0.02),
+        "lm_head": draw("lm_head", (s.vocab, s.d), 0.02),
+        "g_final": draw("tgt.g_final", (s.d,), 0.02, 1.0),
+        "layers": [layer(f"tgt.layer{i}") for i in range(s.n_layers)],
+    }
+
+    def to_host(t):
+        return t.cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+    host = {k: to_host(v) for k, v in dev.items() if k != "layers"}
+    host["layers"] = [{k: to_host(v) for k, v in l.items()} for l in dev["layers"]]
+    return dev, host
 
 
 def subset_uniform(vocab: int, n: int, seed: int) -> np.ndarray:

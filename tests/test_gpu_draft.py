@@ -273,6 +273,197 @@ def test_bad_inputs_are_flagged_not_faulted():
     ctx.close()
 
 
+def _extend_case(shape, seed, L, n_ext, max_ext, K, N):
+    """Seeded inputs of a draft call with extend rows: h_last [B, max_ext, d], tok_last [B, max_ext]; the rows beyond
+    n_ext[b] are padding and are filled with NaN patterns and an invalid token so that any use of them shows."""
+    B = len(L)
+    W = I.mtp_weights(shape, seed)
+    kv = I.paged_kv(shape, list(L), max_ext + K, seed + 1)
+    h = I.hidden_bf16(seed + 2, (B, max_ext, shape.d))
+    tok = I.token_ids(seed + 3, (B, max_ext), shape.vocab)
+    for b in range(B):
+        h[b, n_ext[b]:] = 0x7FC0
+        tok[b, n_ext[b]:] = -7
+    ids = None if N is None else I.subset_uniform(shape.vocab, N, seed + 4)
+    return W, kv, h, tok, ids
+
+
+def _run_extend(Bd, shape, W, kv, h, tok, ids, n_ext, max_ext, K, max_ctx, pass_n_ext=True):
+    B = h.shape[0]
+    ctx = Bd.Context(shape, max_rows=max(8, B * max_ext), max_K=8, max_ctx=max_ctx)
+    dW, dkv = Bd.to_device(W), Bd.to_device(copy_kv(kv))
+    out_d = torch.full((B, K), -1, dtype=torch.int32, device="cuda")
+    out_h = torch.zeros((B, K, shape.d), dtype=torch.bfloat16, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dn = torch.tensor(list(n_ext), dtype=torch.int32, device="cuda") if pass_n_ext else None
+    ctx.fastmtp_draft(Bd.mtp_w(dW), Bd.bf16_tensor(h), torch.from_numpy(tok).cuda(), Bd.kv(dkv), B, K,
+                      None if ids is None else torch.from_numpy(ids).cuda(), out_d, out_h, None, st, n_ext=dn, max_ext=max_ext)
+    torch.cuda.synchronize()
+    res = {"drafts": out_d.cpu().numpy(), "h_out": out_h.float().cpu().numpy(), "h_bits": Bd.bf16_bits(out_h),
+           "status": int(st.item()), "k_pages": Bd.bf16_bits(dkv["k_pages"]), "v_pages": Bd.bf16_bits(dkv["v_pages"]),
+           "launches": ctx.launch_count}
+    ctx.close()
+    return res
+
+
+@pytest.mark.parametrize("L,n_ext,max_ext,K,N", [
+    ([64], [3], 4, 3, 1024),                         # one sequence, a padding row, persistent kernel
+    ([5, 130], [1, 4], 4, 2, 1000),                  # eight activation rows in one launch, contexts across a chunk edge
+    ([0], [8], 8, 3, None),                          # a whole short prompt as extend rows into an empty cache; full vocabulary
+    ([3, 17, 64, 127, 200, 9, 31, 250, 77, 140, 15, 1], [1, 4, 2, 3, 4, 1, 2, 3, 4, 1, 2, 3], 4, 3, 1024),   # batched path, one pass
+    (list(range(0, 400, 10)), [1 + (7 * b) % 3 for b in range(40)], 3, 2, 777),                             # 120 rows: two passes of 63
+])
+def test_extend_rows_in_one_call_match_the_oracle(L, n_ext, max_ext, K, N):
+    """Sec. 2.3 "Drafting phase", step k = 1: the pairs (target hidden state, next token) of the positions committed
+    since the last call run through the MTP module in one pass, causal among themselves; only the last one feeds the
+    head. Drafts, hidden states and both caches against the oracle, sequence by sequence (each with its own n_ext)."""
+    Bd = _binding()
+    shape, seed = I.TINY, 300 + len(L)
+    W, kv, h, tok, ids = _extend_case(shape, seed, L, n_ext, max_ext, K, N)
+    got = _run_extend(Bd, shape, W, kv, h, tok, ids, n_ext, max_ext, K, max(L) + max_ext + K + 1)
+    assert got["status"] == 0, f"device status {got['status']:#x}"
+    okv = copy_kv(kv)
+    exempt = 0
+    for b in range(len(L)):
+        one = dict(okv)                               # pools shared (written in place), tables of sequence b
+        one["block_table"], one["seq_lens"] = okv["block_table"][b:b + 1], okv["seq_lens"][b:b + 1]
+        ref = O.draft(shape, W, h[b:b + 1, :n_ext[b]], tok[b:b + 1, :n_ext[b]], one, K, ids, forced=got["drafts"][b:b + 1])
+        exempt += ids_match(got["drafts"][b], ref["drafts"], ref["gap"], f"extend drafts b={b}")
+        close(got["h_out"][b:b + 1], ref["h_out"], f"extend h_out b={b}")
+    close(O.bf16_to_f64(got["k_pages"]), O.bf16_to_f64(okv["k_pages"]), "extend K cache")
+    close(O.bf16_to_f64(got["v_pages"]), O.bf16_to_f64(okv["v_pages"]), "extend V cache")
+    if len(L) >= 12:
+        assert got["launches"] > 3                    # the batched path ran
+
+
+def test_extend_in_one_call_equals_one_pair_per_call_bit_for_bit():
+    """On the persistent path three extend rows in one call give the bits of three calls with one pair each (the
+    first two with K = 1, their drafts discarded): a row's arithmetic does not depend on the rows beside it."""
+    Bd = _binding()
+    shape, seed, K = I.TINY, 4100, 3
+    L, n = [70, 9], 3
+    W, kv, h, tok, ids = _extend_case(shape, seed, L, [n, n], n, K, 1024)
+    one = _run_extend(Bd, shape, W, kv, h, tok, ids, [n, n], n, K, 128, pass_n_ext=False)
+    ctx = Bd.Context(shape, max_rows=8, max_K=8, max_ctx=128)
+    dW, dkv = Bd.to_device(W), Bd.to_device(copy_kv(kv))
+    out_d = torch.full((2, K), -1, dtype=torch.int32, device="cuda")
+    out_h = torch.zeros((2, K, shape.d), dtype=torch.bfloat16, device="cuda")
+    dids = torch.from_numpy(ids).cuda()
+    for m in range(n):
+        steps = K if m == n - 1 else 1
+        ctx.fastmtp_draft(Bd.mtp_w(dW), Bd.bf16_tensor(np.ascontiguousarray(h[:, m])), torch.from_numpy(np.ascontiguousarray(tok[:, m])).cuda(),
+                          Bd.kv(dkv), 2, steps, dids, out_d[:, :steps].contiguous() if steps < K else out_d,
+                          None if steps < K else out_h)
+        dkv["seq_lens"] += 1
+    torch.cuda.synchronize()
+    assert np.array_equal(out_d.cpu().numpy(), one["drafts"])
+    assert np.array_equal(Bd.bf16_bits(out_h), one["h_bits"])
+    assert np.array_equal(Bd.bf16_bits(dkv["k_pages"]), one["k_pages"]) and np.array_equal(Bd.bf16_bits(dkv["v_pages"]), one["v_pages"])
+    ctx.close()
+
+
+@pytest.mark.parametrize("B", [2, 10])
+def test_positions_beyond_the_cache_are_flagged_and_leave_other_sequences_alone(B):
+    """Sequence 0 sits two tokens below the end of its block table (and of max_ctx) and is asked for three
+    draft steps: the step without a slot is flagged FMTP_DEV_BAD_POS, nothing is written outside the
+    workspace or the pages, and every other sequence of the launch gives the bits it gives in a call
+    of its own. B = 2 runs in the persistent kernel, B = 10 on the batched path."""
+    Bd = _binding()
+    shape, K, seed = I.TINY, 3, 900 + B
+    L = [62] + [20 + 3 * b for b in range(1, B)]
+    W = I.mtp_weights(shape, seed)
+    kv = I.paged_kv(shape, L, 2, seed + 1)                 # 64 slots for sequence 0: positions 62, 63 exist, 64 does not
+    assert kv["max_pages_per_seq"] * shape.page_size == 64
+    h = I.hidden_bf16(seed + 2, (B, shape.d))
+    tok = I.token_ids(seed + 3, (B,), shape.vocab)
+    ids = torch.from_numpy(I.subset_uniform(shape.vocab, 1024, seed + 4)).cuda()
+    dW = Bd.to_device(W)
+
+    def run(rows):
+        ctx = Bd.Context(shape, max_rows=16, max_K=8, max_ctx=64)
+        dkv = Bd.to_device(copy_kv(kv))
+        sub = dict(dkv)
+        sub["block_table"] = dkv["block_table"][rows].contiguous()
+        sub["seq_lens"] = dkv["seq_lens"][rows].contiguous()
+        n = len(rows)
+        out_d = torch.full((n, K), -1, dtype=torch.int32, device="cuda")
+        out_h = torch.zeros((n, K, shape.d), dtype=torch.bfloat16, device="cuda")
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        ctx.fastmtp_draft(Bd.mtp_w(dW), Bd.bf16_tensor(h[rows]), torch.from_numpy(tok[rows]).cuda(), Bd.kv(sub), n, K,
+                          ids, out_d, out_h, None, st)
+        torch.cuda.synchronize()
+        res = out_d.cpu().numpy(), out_h.float().cpu().numpy(), int(st.item()), Bd.bf16_bits(dkv["k_pages"])
+        ctx.close()
+        return res
+
+    d_all, h_all, st_all, k_all = run(list(range(B)))
+    assert st_all & Bd.DEV_BAD_POS and not st_all & Bd.DEV_TIMEOUT
+    d_rest, h_rest, st_rest, k_rest = run(list(range(1, B)))
+    assert st_rest == 0
+    assert np.array_equal(d_all[1:], d_rest) and np.array_equal(h_all[1:], h_rest)
+    # the pages of the other sequences hold the same bits; sequence 0's first two steps are in range and correct
+    own0 = set(int(x) for x in kv["block_table"][0] if x >= 0)
+    others = [pg for pg in range(kv["num_pages"]) if pg not in own0]
+    assert np.array_equal(k_all[others], k_rest[others])
+    okv = copy_kv(kv)
+    okv["block_table"], okv["seq_lens"] = okv["block_table"][:1], okv["seq_lens"][:1]
+    ref = O.draft(shape, W, h[:1], tok[:1], okv, 2, ids.cpu().numpy(), forced=d_all[:1, :2])
+    ids_match(d_all[:1, :2], ref["drafts"], ref["gap"], "in-range steps of the overflowing sequence")
+    close(h_all[:1, :2], ref["h_out"], "in-range steps of the overflowing sequence")
+
+
+@pytest.mark.parametrize("B,K", [(1, 3), (20, 3), (64, 2)])
+def test_draft_call_captured_in_a_cuda_graph_replays_on_the_current_state(B, K):
+    """One fastmtp_draft call (all K steps; the persistent kernel at B = 1, the batched path's chain of kernels
+    otherwise) is captured into a CUDA graph and replayed after the sequences have advanced and the inputs have
+    changed: sequence lengths, block tables, tokens and hidden states are read on the device, so the replay gives the
+    bits of an eager call on the same state."""
+    Bd = _binding()
+    shape, seed = I.TINY, 6100 + B
+    L = [int(x) for x in I.context_lengths(B, 0, 150, seed)]
+    W = I.mtp_weights(shape, seed)
+    kv = I.paged_kv(shape, L, K + 2, seed + 1)
+    dW, dkv = Bd.to_device(W), Bd.to_device(copy_kv(kv))
+    dh = Bd.bf16_tensor(I.hidden_bf16(seed + 2, (B, shape.d)))
+    dtok = torch.from_numpy(I.token_ids(seed + 3, (B,), shape.vocab)).cuda()
+    dids = torch.from_numpy(I.subset_uniform(shape.vocab, 1024, seed + 4)).cuda()
+    ctx = Bd.Context(shape, max_rows=max(8, B), max_K=8, max_ctx=max(L) + K + 3)
+    out_d = torch.full((B, K), -1, dtype=torch.int32, device="cuda")
+    out_h = torch.zeros((B, K, shape.d), dtype=torch.bfloat16, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    w, ckv = Bd.mtp_w(dW), Bd.kv(dkv)
+
+    def call():
+        ctx.fastmtp_draft(w, dh, dtok, ckv, B, K, dids, out_d, out_h, None, st)
+
+    call()                                       # eager warm-up: set-up that belongs outside a capture happens here
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(graph, stream=side):
+        call()
+    # the state moves on: one more committed token per sequence, new inputs
+    dkv["seq_lens"] += 1
+    dh.copy_(Bd.bf16_tensor(I.hidden_bf16(seed + 5, (B, shape.d))))
+    dtok.copy_(torch.from_numpy(I.token_ids(seed + 6, (B,), shape.vocab)).cuda())
+    torch.cuda.synchronize()
+    k0, v0 = dkv["k_pages"].clone(), dkv["v_pages"].clone()
+    out_d.fill_(-1); out_h.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    g_d, g_h, g_k, g_v = out_d.clone(), out_h.clone(), dkv["k_pages"].clone(), dkv["v_pages"].clone()
+    assert int(st.item()) == 0
+    dkv["k_pages"].copy_(k0); dkv["v_pages"].copy_(v0)
+    out_d.fill_(-1); out_h.zero_()
+    call()
+    torch.cuda.synchronize()
+    assert torch.equal(out_d, g_d) and torch.equal(out_h, g_h)
+    assert torch.equal(dkv["k_pages"], g_k) and torch.equal(dkv["v_pages"], g_v)
+    assert (g_d >= 0).all()
+    ctx.close()
+
+
 def test_host_entry_point_matches_device_entry_point():
     Bd = _binding()
     shape = I.TINY

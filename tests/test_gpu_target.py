@@ -196,105 +196,60 @@ def test_rows_do_not_depend_on_rows_per_call():
     assert torch.equal(one_l, torch.cat([l4a, l4b], dim=1))
 
 
-def _gpu_greedy(gpu, prompt, n_new):
-    P = len(prompt)
-    last = None
-    for lo in range(0, P, 8):
-        _, _, a = gpu.step(np.array([prompt[lo:lo + 8]]), want_logits=False)
-        gpu.advance(len(prompt[lo:lo + 8]))
-        last = int(a[0, -1])
-    out = [last]
-    while len(out) < n_new:
-        _, _, a = gpu.step(np.array([[out[-1]]]), want_logits=False)
-        gpu.advance(1)
-        out.append(int(a[0, 0]))
-    return out
+def oracle_checks_greedy_tokens(shape, Wt, prompt, tokens, mk_kvs):
+    """The oracle's target on [prompt ; tokens[:-1]] in one teacher-forced pass: at every generated position its greedy
+    choice (on bf16-rounded logits) equals the library's token, except at near ties. Returns the number of exemptions."""
+    n = len(tokens)
+    seq = np.array([list(prompt) + [int(t) for t in tokens[:-1]]])
+    okvs = mk_kvs()
+    hh, _ = O.target_forward(shape, Wt, seq, okvs, want_logits=False)
+    exempt = 0
+    for i in range(n):
+        row = O.head_logits(hh[0, len(prompt) - 1 + i], Wt["lm_head"])
+        t, _ = O.argmax_token(O.round_bf16(row))
+        if t != int(tokens[i]):
+            assert _bf16_gap(row) < GAP_TOL, f"token {i}: oracle {t}, gpu {int(tokens[i])}"
+            exempt += 1
+    return exempt
 
 
 def speculative_vs_greedy(shape, seed, K, n_new, prompt_len, N, max_ctx, n_oracle):
-    """Greedy decoding and speculative decoding (MTP drafts, every other round drafts that are right for a
-    planted number of positions) by the library on the same random model; returns both token lists and
-    the accepted lengths, after checking the first n_oracle greedy tokens against the oracle."""
+    """Greedy decoding and speculative decoding (MTP drafts; every other round drafts that are right for a planted
+    number of positions) by the library on the same random model, through the loops of paper_2509_18362_b200.loop
+    (extend rows in one draft call, target argmax only, acceptance on token ids). Returns both token lists and the
+    accepted lengths, after checking the first n_oracle greedy tokens against the oracle."""
     Bd = _binding()
+    from paper_2509_18362_b200 import loop
     L = shape.n_layers
     Wt = I.target_weights(shape, seed)
     Wm = I.mtp_weights(shape, seed + 1, embed=Wt["embed"], lm_head=Wt["lm_head"])
     prompt = [int(t) for t in I.token_ids(seed + 2, (prompt_len,), shape.vocab)]
     ids = I.subset_uniform(shape.vocab, N, seed + 3)
     mk = lambda: [I.empty_paged_kv(shape, 1, max_ctx, seed + 10 + l) for l in range(L)]
+    ctx = Bd.Context(shape, max_rows=64, max_K=8, max_ctx=max_ctx)
+    dW = Bd.to_device(Wt)
 
-    g = GpuTarget(shape, Wt, mk(), max_ctx)
-    ref = _gpu_greedy(g, prompt, n_new + K + 1)
-    g.close()
+    ref = loop.greedy_decode(loop.Target(ctx, shape, dW, [Bd.to_device(kv) for kv in mk()]), prompt, n_new + K + 1)
 
-    gpu = GpuTarget(shape, Wt, mk(), max_ctx)
+    tgt = loop.Target(ctx, shape, dW, [Bd.to_device(kv) for kv in mk()])
     dWm = dict(Bd.to_device({k: v for k, v in Wm.items() if k not in ("embed", "lm_head")}),
-               embed=gpu.dW["embed"], lm_head=gpu.dW["lm_head"])          # shared with the target, one copy
-    wm = Bd.mtp_w(dWm)
+               embed=dW["embed"], lm_head=dW["lm_head"])                   # shared with the target, one copy
     mkv = Bd.to_device(I.empty_paged_kv(shape, 1, max_ctx, seed + 20))
-    dids = torch.from_numpy(ids).cuda()
-    # prefill the target; feed the MTP cache with pairs (h_j, t_{j+1}) one position per call
-    hs = []
-    last = None
-    for lo in range(0, len(prompt), 8):
-        h, _, a = gpu.step(np.array([prompt[lo:lo + 8]]), want_logits=False)
-        gpu.advance(len(prompt[lo:lo + 8]))
-        hs.append(h)
-        last = int(a[0, -1])
-    hP = torch.cat(hs, dim=1)[0]
-    out = [last]
-    pend_h = hP
-    pend_t = prompt[1:] + [last]
-    drafts_d = torch.zeros((1, K), dtype=torch.int32, device="cuda")
-    accepted = []
-    rnd = 0
-    while len(out) < n_new:
-        for m in range(len(pend_t)):
-            steps = K if m == len(pend_t) - 1 else 1
-            gpu.ctx.fastmtp_draft(wm, pend_h[m:m + 1].contiguous(),
-                                  torch.tensor([pend_t[m]], dtype=torch.int32, device="cuda"),
-                                  Bd.kv(mkv), 1, steps, dids, drafts_d)
-            mkv["seq_lens"] += 1
-        torch.cuda.synchronize()
-        drafts = [int(t) for t in drafts_d.cpu().numpy()[0]]
-        if rnd % 2 == 1:
-            # every other round: inject drafts that are right for a planted number of positions
-            e = len(out)
-            n_ok = (rnd // 2) % (K + 1)
-            good = ref[e:e + K]
-            drafts = list(good[:n_ok]) + [(t + 1) % shape.vocab for t in good[n_ok:]]
-        row = np.array([[out[-1]] + drafts], dtype=np.int32)
-        h, logits, _ = gpu.step(row)
-        acc = torch.zeros(1, dtype=torch.int32, device="cuda")
-        bon = torch.zeros(1, dtype=torch.int32, device="cuda")
-        gpu.ctx.fastmtp_verify_accept(logits, torch.tensor([drafts], dtype=torch.int32, device="cuda"), 1, K,
-                                      shape.vocab, acc, bon)
-        torch.cuda.synchronize()
-        a, bonus = int(acc.item()), int(bon.item())
-        gpu.advance(a + 1)
-        new = drafts[:a] + [bonus]
-        out.extend(new)
-        accepted.append(a)
-        pend_h = h[0, :a + 1]
-        pend_t = new
-        rnd += 1
-    gpu.close()
 
-    # oracle greedy on the first tokens, teacher-forced on near ties (logits of the newest row only)
-    okvs = mk()
-    hh, _ = O.target_forward(shape, Wt, np.array([prompt]), okvs, want_logits=False)
-    for kv in okvs:
-        kv["seq_lens"][0] = len(prompt)
-    row = O.head_logits(hh[0, -1], Wt["lm_head"])
-    for i in range(n_oracle):
-        t, _ = O.argmax_token(O.round_bf16(row))
-        assert t == ref[i] or _bf16_gap(row) < GAP_TOL, f"token {i}: oracle {t}, gpu {ref[i]}"
-        hh, _ = O.target_forward(shape, Wt, np.array([[ref[i]]]), okvs, want_logits=False)
-        for kv in okvs:
-            kv["seq_lens"][0] += 1
-        row = O.head_logits(hh[0, 0], Wt["lm_head"])
+    def inject(rnd, K, emitted):
+        if rnd % 2 == 0:
+            return None
+        n_ok = (rnd // 2) % (K + 1)                                          # drafts right for a planted number of positions
+        good = ref[emitted:emitted + K]
+        return list(good[:n_ok]) + [(t + 1) % shape.vocab for t in good[n_ok:]]
+
+    out, stats = loop.speculative_decode(tgt, Bd.mtp_w(dWm), mkv, torch.from_numpy(ids).cuda(), prompt, n_new, K, inject)
+    assert int(mkv["seq_lens"].item()) == int(tgt.dkvs[0]["seq_lens"].item())   # MTP and target caches committed alike
+    ctx.close()
+    exempt = oracle_checks_greedy_tokens(shape, Wt, prompt, ref[:n_oracle], mk)
     O.clear_weight_memo()
-    return ref, out, accepted
+    print(f"loop: tau {stats['tau']:.2f}, accepted {stats['accepted']}, oracle exemptions {exempt}/{n_oracle}")
+    return ref, out, stats["accepted"]
 
 
 def test_speculative_loop_is_token_identical_to_greedy_on_gpu():

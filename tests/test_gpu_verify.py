@@ -82,6 +82,29 @@ def test_special_values_and_unaligned_rows():
     ctx.close()
 
 
+@pytest.mark.parametrize("B,K,V", [(1, 3, 4096), (5, 0, 1000), (64, 3, 152064), (300, 7, 33)])
+def test_accept_on_token_ids_equals_the_oracle(B, K, V):
+    """fastmtp_accept_ids consumes the target's per-row greedy tokens instead of logits: same accepted lengths and
+    bonus tokens as the oracle's verification of the logits those tokens came from (planted prefixes and natural ties)."""
+    Bd, ctx = _ctx()
+    case = I.verify_case(B, K, V, 2000 + B)
+    for logits, drafts in ((case["logits"], case["drafts"]),
+                           (I.verify_logits_natural(min(B, 8), K + 1, V, 5), case["drafts"][:min(B, 8)])):
+        ra, rb, rg = O.verify_accept(logits, drafts)
+        n = logits.shape[0]
+        if K > 0 and n > 1:
+            drafts = drafts.copy()
+            drafts[1, :K] = rg[1, :K]                      # one fully accepted sequence
+            ra, rb, rg = O.verify_accept(logits, drafts)
+        acc = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        bon = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        ctx.fastmtp_accept_ids(torch.from_numpy(rg).cuda(), torch.from_numpy(np.ascontiguousarray(drafts)).cuda() if K > 0 else None,
+                               n, K, acc, bon)
+        torch.cuda.synchronize()
+        assert np.array_equal(acc.cpu().numpy(), ra) and np.array_equal(bon.cpu().numpy(), rb)
+    ctx.close()
+
+
 def test_host_entry_point():
     Bd, ctx = _ctx()
     case = I.verify_case(9, 3, 5000, 21)

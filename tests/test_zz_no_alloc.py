@@ -4,13 +4,15 @@ A host that has given all device memory to its own pool, or that sits inside a d
 allocation would stall the GPU, cannot provide the workspace the regular call needs; this entry point
 keeps its scratch in a fixed array inside the library. The test calls it through the C ABI twice in a
 row (the second call finds the first one's leftovers in the shared array) and compares with the
-regular entry point, which is itself checked against the oracle elsewhere. Integer results: bit-exact.
+regular entry point and with the oracle's verification of the same logits. Integer results: bit-exact.
+It also checks what the call exists for: device memory in use is the same before and after the calls.
 Collected last on purpose, so a run that stops at the first failure has already run everything else.
 """
 import numpy as np
 import pytest
 import torch
 
+from oracle import fastmtp_oracle as O
 from paper_2509_18362_b200 import inputs as I
 
 pytestmark = pytest.mark.gpu
@@ -50,9 +52,20 @@ def test_static_entry_point_matches_regular_one_on_two_calls_in_a_row():
         for w, g in zip(want, got):
             assert np.array_equal(w, g)
         assert np.array_equal(got[0], case["length"])            # and the planted answer
-    # the same inputs once more: the array still holds the previous call's contents
-    got2 = _static(Bd, dl, dd, B, K, V)
-    assert all(np.array_equal(a, b) for a, b in zip(got, got2))
+        ra, rb, rg = O.verify_accept(case["logits"], case["drafts"])
+        assert np.array_equal(got[0], ra) and np.array_equal(got[1], rb) and np.array_equal(got[2], rg)
+    # the same inputs once more: the array still holds the previous call's contents. Around these calls (the
+    # entry point's per-device set-up happened above) the device's free memory and torch's own
+    # allocations must not move: the call creates no device memory, directly or through a library.
+    acc = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    bon = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    free0, alloc0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+    for _ in range(2):
+        Bd.fastmtp_verify_accept_static(dl, dd, B, K, V, acc, bon)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0
+    assert np.array_equal(acc.cpu().numpy(), got[0]) and np.array_equal(bon.cpu().numpy(), got[1])
     ctx.close()
 
 
