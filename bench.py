@@ -49,6 +49,14 @@ def parse_args():
     ap.add_argument("--target-layers", type=int, default=0,
                     help="instead of the draft path, time fastmtp_target_step on a random target of this many layers "
                          "(1 row and draft-steps+1 rows per sequence); one JSON line per row count")
+    ap.add_argument("--e2e-loop", action="store_true",
+                    help="the end-to-end configuration: random 28-layer target of the 7B-class shape + the MTP layer, 512-token "
+                         "prompt, 256 generated tokens, draft-steps=3, subset 32768; greedy and speculative decoding by the library "
+                         "(token-identical), the oracle on the first 16 tokens; one JSON line")
+    ap.add_argument("--loop-layers", type=int, default=28)
+    ap.add_argument("--loop-prompt", type=int, default=512)
+    ap.add_argument("--loop-tokens", type=int, default=256)
+    ap.add_argument("--loop-oracle-tokens", type=int, default=16)
     ap.add_argument("--sweep", action="store_true",
                     help="vocabulary-compression sweep on one GPU: subset size x batch x draft steps, one JSON line each")
     return ap.parse_args()
@@ -493,8 +501,92 @@ def run_target(a):
         ctx.close()
 
 
+def run_e2e_loop(a):
+    """Greedy and speculative decoding of one sequence through the C ABI on a random target + MTP head; checks that the
+    two emit the same tokens and that the first tokens agree with the oracle (teacher-forced, near ties exempt)."""
+    import torch
+    import __graft_entry__ as G
+    G.build()
+    from paper_2509_18362_b200 import binding as Bd, inputs as I, loop
+    torch.cuda.set_device(0)
+    s = (I.QWEN7B if a.shape == "7b" else I.TINY).with_layers(a.loop_layers)
+    P, n_new, K, n_or = a.loop_prompt, a.loop_tokens, a.draft_steps, a.loop_oracle_tokens
+    N = a.subset if 0 < a.subset < s.vocab else s.vocab
+    max_ctx = P + n_new + K + 3
+    t0 = time.time()
+    dWt, Wt = I.target_weights_cuda(s, a.seed)
+    Wm = I.mtp_weights(s, a.seed + 1, embed=Wt["embed"], lm_head=Wt["lm_head"])
+    prompt = [int(t) for t in I.token_ids(a.seed + 2, (P,), s.vocab)]
+    ids = None if N >= s.vocab else I.subset_uniform(s.vocab, N, a.seed + 3)
+    mk = lambda: [I.empty_paged_kv(s, 1, max_ctx, a.seed + 10 + l) for l in range(s.n_layers)]
+    ctx = Bd.Context(s, max_rows=64, max_K=max(8, K), max_ctx=max_ctx)
+    t_gen = time.time() - t0
+
+    def timed(fn):
+        torch.cuda.synchronize()
+        t = time.time()
+        r = fn()
+        torch.cuda.synchronize()
+        return r, time.time() - t
+
+    ref, t_greedy = timed(lambda: loop.greedy_decode(loop.Target(ctx, s, dWt, [Bd.to_device(kv) for kv in mk()]), prompt, n_new + K + 1))
+    dWm = dict(Bd.to_device({k: v for k, v in Wm.items() if k not in ("embed", "lm_head")}), embed=dWt["embed"], lm_head=dWt["lm_head"])
+    dids = None if ids is None else torch.from_numpy(ids).cuda()
+
+    def spec(inject):
+        tgt = loop.Target(ctx, s, dWt, [Bd.to_device(kv) for kv in mk()])
+        mkv = Bd.to_device(I.empty_paged_kv(s, 1, max_ctx, a.seed + 20))
+        return loop.speculative_decode(tgt, Bd.mtp_w(dWm), mkv, dids, prompt, n_new, K, inject)
+
+    def inject(rnd, K_, emitted):          # every other round: drafts right for a planted number of positions
+        if rnd % 2 == 0:
+            return None
+        n_ok = (rnd // 2) % (K_ + 1)
+        good = ref[emitted:emitted + K_]
+        return list(good[:n_ok]) + [(t + 1) % s.vocab for t in good[n_ok:]]
+
+    (out_mtp, st_mtp), t_mtp = timed(lambda: spec(None))
+    (out_inj, st_inj), t_inj = timed(lambda: spec(inject))
+    lossless = out_mtp == ref[:n_new] and out_inj == ref[:n_new]
+
+    from oracle import fastmtp_oracle as O
+    t0 = time.time()
+    rows = list(range(P - 1, P - 1 + n_or))
+    _, logits = O.target_forward_block(s, Wt, prompt + [int(t) for t in ref[:n_or - 1]], mk(), logit_rows=rows)
+    t_oracle = time.time() - t0
+    exempt, wrong = 0, 0
+    for i, r in enumerate(rows):
+        t, _ = O.argmax_token(O.round_bf16(logits[r]))
+        if t != ref[i]:
+            top2 = np.partition(logits[r], logits[r].shape[0] - 2)[-2:]
+            ulp = 2.0 ** (np.floor(np.log2(max(abs(top2[1]), 1e-30))) - 7)
+            if top2[1] - top2[0] - ulp < 1e-2:
+                exempt += 1
+            else:
+                wrong += 1
+    print(json.dumps({
+        "e2e_loop": True, "layers": s.n_layers, "prompt": P, "generated": n_new, "draft_steps": K, "subset": N,
+        "token_identical_to_greedy": bool(lossless),
+        "greedy": {"seconds": t_greedy, "tokens_per_s": (n_new + K + 1) / t_greedy, "note": "prefill of the prompt included"},
+        "speculative_mtp_drafts": {"seconds": t_mtp, "tokens_per_s": n_new / t_mtp, "tau": st_mtp["tau"],
+                                   "accept_rate_by_position": st_mtp["accept_rate_by_position"], "target_calls": st_mtp["target_calls"],
+                                   "note": "random weights: the head's drafts are almost never accepted"},
+        "speculative_injected_drafts": {"seconds": t_inj, "tokens_per_s": n_new / t_inj, "tau": st_inj["tau"],
+                                        "accept_rate_by_position": st_inj["accept_rate_by_position"],
+                                        "target_calls": st_inj["target_calls"],
+                                        "note": "every other round drafts right for 0..K positions in turn"},
+        "oracle": {"tokens_checked": n_or, "mismatches_outside_near_ties": wrong, "near_tie_exemptions": exempt,
+                   "seconds": t_oracle, "cores": os.cpu_count(), "how": "prompt + tokens teacher-forced in one layer-grouped pass"},
+        "weights_seconds": t_gen, "data": "synthetic (weights drawn on the device, seeded)"}))
+    ctx.close()
+    if not lossless or wrong:
+        raise SystemExit(1)
+
+
 def main():
     a = parse_args()
+    if a.e2e_loop:
+        return run_e2e_loop(a)
     if a.target_layers > 0:
         return run_target(a)
     if a.sweep:

@@ -145,6 +145,18 @@ long long fmtp_launch_count(const fmtp_ctx *ctx);
  * (ring stages, grid barriers) use the same loop with a 2 s limit. */
 int fmtp_selftest_wait_timeout(uint32_t *dev_status, int limit_ms, unsigned long long *dev_waited_ns, void *stream);
 
+/* Diagnostic (no counterpart in the paper): arms the NEXT fastmtp_draft call on this context so that one of its own
+ * device-side waits cannot end, with every wait of that call limited to `limit_ms` milliseconds (1..1000):
+ *   which = 1  the persistent kernel's grid barrier expects one arrival more than there are CTAs
+ *              (takes effect if that call runs on the persistent path);
+ *   which = 2  the first ring stage of the call's first tensor-core GEMM expects one copy more than is made
+ *              (takes effect if that call runs on the batched path).
+ * The wait runs out, the kernel ORs FMTP_DEV_TIMEOUT into the status word, every other CTA / role sees the abort
+ * flag and stops waiting, copies in flight are drained, tensor memory is freed, and the launch -- and the rest of
+ * the call's launches, on garbage that stays inside the caller's buffers -- ends normally: nothing hangs, traps or
+ * faults. The call's outputs are invalid; the context and the device stay usable and the next call is unaffected. */
+int fmtp_selftest_inject_wait_timeout(fmtp_ctx *ctx, int limit_ms, int which);
+
 /* ---- draft: Sec. 2.3 "Drafting phase", Sec. 2.1 steps k=1 / k>1, Sec. 2.2 Eq. 3 -------- */
 
 /* Recursive K-step draft for B sequences.

@@ -24,7 +24,8 @@ FMTP_OK = 0
 DEV_BAD_TOKEN, DEV_BAD_PAGE, DEV_BAD_POS, DEV_TIMEOUT, DEV_ALL_NAN = 1, 2, 4, 8, 16
 
 EXPORTS = ["fmtp_create", "fmtp_destroy", "fmtp_workspace_bytes", "fmtp_set_workspace", "fmtp_strerror",
-           "fmtp_last_cuda_error", "fmtp_launch_count", "fmtp_selftest_wait_timeout", "fastmtp_draft", "fastmtp_draft_host",
+           "fmtp_last_cuda_error", "fmtp_launch_count", "fmtp_selftest_wait_timeout", "fmtp_selftest_inject_wait_timeout",
+           "fastmtp_draft", "fastmtp_draft_host",
            "fastmtp_verify_accept", "fastmtp_verify_accept_host", "fastmtp_verify_accept_static", "fastmtp_accept_ids",
            "fastmtp_target_step"]
 
@@ -72,6 +73,8 @@ lib.fmtp_launch_count.argtypes = [_p]
 lib.fmtp_launch_count.restype = C.c_longlong
 lib.fmtp_selftest_wait_timeout.argtypes = [_p, C.c_int, _p, _p]
 lib.fmtp_selftest_wait_timeout.restype = C.c_int
+lib.fmtp_selftest_inject_wait_timeout.argtypes = [_p, C.c_int, C.c_int]
+lib.fmtp_selftest_inject_wait_timeout.restype = C.c_int
 lib.fastmtp_draft.argtypes = [_p, C.POINTER(fmtp_mtp_w), _p, _p, _p, C.c_int, C.POINTER(fmtp_kv), C.c_int, C.c_int, _p,
                               C.c_int, _p, _p, _p, _p, _p]
 lib.fastmtp_draft.restype = C.c_int
@@ -185,6 +188,10 @@ class Context:
             self.close()
         except Exception:
             pass
+
+    def fmtp_selftest_inject_wait_timeout(self, limit_ms, which):
+        self._check(lib.fmtp_selftest_inject_wait_timeout(self.handle, int(limit_ms), int(which)),
+                    "fmtp_selftest_inject_wait_timeout")
 
     @property
     def launch_count(self) -> int:

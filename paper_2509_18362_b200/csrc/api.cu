@@ -46,11 +46,15 @@ struct fmtp_ctx {
     struct { int mode, B, M, G; } group_memo[16];                  // sequences per launch for (mode, B, M)
     int n_group_memo;
     TmapCache tmaps;                                               // tensor maps of the batched path's GEMM operands
+    // fmtp_selftest_inject_wait_timeout: the next draft call runs with this wait limit and one wait that cannot end
+    unsigned long long inject_limit_ns;
+    int inject_which;                                              // 0 none, 1 grid barrier of the persistent kernel, 2 ring stage of a GEMM
 };
 
 namespace {
 
 constexpr int kVerifyMaxRows = 4096;
+constexpr unsigned long long kDefaultWaitNs = 2000000000ull;     // a device-side wait gives up after 2 s
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -146,6 +150,7 @@ int configure(fmtp_ctx *c, MegaParams &p, int mode, int B, int M) {
     }
     p.max_chunks = c->max_chunks;
     p.max_ctx = sh.max_ctx;
+    p.wait_limit_ns = kDefaultWaitNs;
     p.mode = mode; p.B = B; p.M = M; p.R = B * M;
     const int R = p.R, Gq = p.Hq / p.Hkv;
     size_t attn = (size_t)M * Gq * p.dh * 4;
@@ -304,6 +309,14 @@ int fmtp_create(const fmtp_shape *sh, fmtp_ctx **out) {
     return FMTP_OK;
 }
 
+int fmtp_selftest_inject_wait_timeout(fmtp_ctx *c, int limit_ms, int which) {
+    if (!c || (which != 1 && which != 2)) return FMTP_EINVAL;
+    if (limit_ms < 1 || limit_ms > 1000) return FMTP_EINVAL;      // bounded on purpose
+    c->inject_limit_ns = (unsigned long long)limit_ms * 1000000ull;
+    c->inject_which = which;
+    return FMTP_OK;
+}
+
 int fmtp_destroy(fmtp_ctx *c) {
     if (!c) return FMTP_EINVAL;
     if (c->pinned) cudaFreeHost(c->pinned);
@@ -385,6 +398,8 @@ int fastmtp_draft(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_last, con
             bc.sh = c->bsh; bc.ws = c->bws;
             bc.rope_cos = c->s.rope_cos; bc.rope_sin = c->s.rope_sin;
             bc.n_sm = c->n_sm; bc.smem_optin = c->smem_optin; bc.cache = &c->tmaps;
+            bc.wait_limit_ns = kDefaultWaitNs;
+            if (c->inject_which == 2) { bc.wait_limit_ns = c->inject_limit_ns; bc.inject_gemm_timeout = 1; c->inject_which = 0; }
             bc.B = (B - b0 < kBatchRows) ? B - b0 : kBatchRows;
             bc.K = K; bc.N = Neff; bc.ids = subset;
             bc.M0 = max_ext; bc.n_ext = n_ext ? n_ext + b0 : nullptr;
@@ -413,6 +428,7 @@ int fastmtp_draft(fmtp_ctx *c, const fmtp_mtp_w *w, const fmtp_bf16 *h_last, con
         p.K = K;
         p.N = Neff;
         p.ids = subset;
+        if (c->inject_which == 1) { p.wait_limit_ns = c->inject_limit_ns; p.extra_arrivals = 1; c->inject_which = 0; }
         p.h_last = h_last + (size_t)b0 * max_ext * d;
         p.tokens = tok_last + (size_t)b0 * max_ext;
         p.n_ext = n_ext ? n_ext + b0 : nullptr;
@@ -556,7 +572,7 @@ int fastmtp_target_step(fmtp_ctx *c, const fmtp_target_w *w, const int32_t *toke
             std::memset(&tc, 0, sizeof(tc));
             tc.sh = c->bsh; tc.ws = c->bws;
             tc.rope_cos = c->s.rope_cos; tc.rope_sin = c->s.rope_sin;
-            tc.n_sm = c->n_sm; tc.smem_optin = c->smem_optin; tc.cache = &c->tmaps;
+            tc.n_sm = c->n_sm; tc.smem_optin = c->smem_optin; tc.cache = &c->tmaps; tc.wait_limit_ns = kDefaultWaitNs;
             tc.B = Bg; tc.M = M; tc.n_layers = nl;
             tc.tokens = tokens + (size_t)b0 * M;
             tc.out_h = out_h ? out_h + (size_t)b0 * M * d : nullptr;

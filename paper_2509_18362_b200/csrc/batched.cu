@@ -303,6 +303,7 @@ __global__ void qkv_finish_kernel(const QkvArgs a) {
 struct AttnArgs {
     int Hq, Hkv, dh, page, page_shift, max_ctx, max_chunks, B;    // B: rows
     RowGeo geo;                  // which sequence and position a row has
+    unsigned long long wait_limit_ns;   // a ring wait gives up after this long
     const float *q;              // [rows][Hq*dh] words: the scaled query values as {hi, lo} bf16 pairs
     KvPtrs kv;
     float *att_part;             // [rows][Hq][max_chunks][dh+2]
@@ -312,7 +313,6 @@ struct AttnArgs {
 constexpr int kAttnBlk = 64;                 // tokens per ring stage
 constexpr int kAttnStages = 5;
 constexpr int kAttnThreads = 128;            // compute threads (warps 0-3); warps 4-7 only issue the copies
-constexpr unsigned long long kAttnWaitNs = 2000000000ull;
 
 struct AttnItem {                            // one (sequence, KV head, chunk), CTA-uniform
     int r, kvh, chunk, t0, n_ctx, n_blk;
@@ -357,7 +357,7 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
         while (!mbar_try_wait(bar, parity)) {
             if ((++polls & 63u) == 0) {
                 if (*abort_flag) return false;
-                if (global_timer_ns() - t_begin > kAttnWaitNs) { *abort_flag = 1u; return false; }
+                if (global_timer_ns() - t_begin > a.wait_limit_ns) { *abort_flag = 1u; return false; }
             }
         }
         return true;
@@ -371,7 +371,7 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
     __syncthreads();
     if (threadIdx.x == 0) {
         int acc = 0;
-        for (int r = 0; r < a.B; ++r) { prefix[r] = acc; acc += (nctx[r] + kBatchAttnChunk - 1) / kBatchAttnChunk; }
+        for (int r = 0; r < a.B; ++r) { prefix[r] = acc; const int ct = attn_chunk_tokens(nctx[r]); acc += (nctx[r] + ct - 1) / ct; }
         prefix[a.B] = acc;
     }
     __syncthreads();
@@ -384,9 +384,10 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
         while (prefix[r + 1] <= cidx) ++r;
         it.r = r;
         it.chunk = cidx - prefix[r];
-        it.t0 = it.chunk * kBatchAttnChunk;
         it.n_ctx = nctx[r];
-        it.n_blk = (min(kBatchAttnChunk, it.n_ctx - it.t0) + kAttnBlk - 1) / kAttnBlk;
+        const int ct = attn_chunk_tokens(it.n_ctx);
+        it.t0 = it.chunk * ct;
+        it.n_blk = (min(ct, it.n_ctx - it.t0) + kAttnBlk - 1) / kAttnBlk;
         it.bt = a.kv.block_table + (size_t)(r / a.geo.M) * a.kv.max_pages;
     };
 
@@ -397,6 +398,7 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
     constexpr int NIT = kAttnBlk * PIECES / kAttnThreads;
     constexpr int TSTEP = kAttnThreads / PIECES;        // tokens between a thread's consecutive pieces
     const int pc = tid % PIECES, tl = tid / PIECES;
+    const uint64_t kv_policy = l2_evict_first();
     auto load_pages = [&](const AttnItem &it_, int blk, int (&pg)[NIT]) {
 #pragma unroll
         for (int it = 0; it < NIT; ++it) {
@@ -439,8 +441,8 @@ __global__ void __launch_bounds__(2 * kAttnThreads, 1) attn_kernel(const AttnArg
         const uint32_t d0 = smem_u32(st + tl * ROWB + pc * 16);
 #pragma unroll
         for (int it = 0; it < NIT; ++it) {
-            cp_async16_off<0>(d0 + it * TSTEP * ROWB, a.kv.k_pages + off[it], ok[it]);
-            cp_async16_off<0>(d0 + kAttnBlk * ROWB + it * TSTEP * ROWB, a.kv.v_pages + off[it], ok[it]);
+            cp_async16_off_hint<0>(d0 + it * TSTEP * ROWB, a.kv.k_pages + off[it], ok[it], kv_policy);
+            cp_async16_off_hint<0>(d0 + kAttnBlk * ROWB + it * TSTEP * ROWB, a.kv.v_pages + off[it], ok[it], kv_policy);
         }
         if (fb == 0) {     // the item's query vectors ride with its first block
             const float *qsrc = a.q + ((size_t)fc.r * a.Hq + (size_t)fc.kvh * gq) * DH;    // packed {hi, lo} words
@@ -620,7 +622,7 @@ __global__ void attn_merge_kernel(const MergeArgs a) {
     const int max_tokens = min(a.kv.max_pages * a.page, a.max_ctx);
     bool valid;
     const int n_ctx = min(geo_pos(a.geo, a.kv, r, &valid), max_tokens - 1) + 1;
-    const int n_chunks = (n_ctx + kBatchAttnChunk - 1) / kBatchAttnChunk;
+    const int n_chunks = (n_ctx + attn_chunk_tokens(n_ctx) - 1) / attn_chunk_tokens(n_ctx);
     const int stride = a.dh + 2;
     const float *base = a.att_part + ((size_t)r * a.Hq + head) * a.max_chunks * stride;
     // the chunks' maxima: each thread reads some, then a block-wide maximum (exact, order-free)
@@ -693,6 +695,8 @@ __global__ void __launch_bounds__(kRowThreads) embed_kernel(const int32_t *token
 // its rows, and gathering head rows in address order keeps the 128 rows of a GEMM tile within a few
 // memory pages (an unsorted subset spreads them over the whole matrix and the address translation
 // misses cost ~25 % of the head's stream rate). Membership bitmap, then a one-block compaction.
+// (The two kernels run under the first kernels of step 0; the head GEMM, the only reader of the sorted ids, waits
+// for the whole chain before it looks at them.)
 __global__ void ids_mark_kernel(const int32_t *ids, int N, int V, uint32_t *bitmap, uint32_t *status) {
     chain_release();
     chain_wait();
@@ -797,6 +801,7 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
     const int B = c.B, K = c.K, d = sh.d;
     const int M0 = c.M0 > 1 ? c.M0 : 1;
     const bool ext = M0 > 1;                       // step 0 carries up to M0 extend rows per sequence
+    int inject_left = c.inject_gemm_timeout ? 1 : 0;
     const int qdim = sh.Hq * sh.dh, kvdim = sh.Hkv * sh.dh;
     cudaError_t e = cudaMemsetAsync(ws.keys, 0, ws.keys_bytes, st);     // argmax keys and the status word
     if (e != cudaSuccess) return (int)e;
@@ -818,6 +823,9 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
     auto gemm = [&](GemmArgs &g, int rows, int n_rows, int Kdim, int lda, const bf16_t *x, int ldx) -> int {
         g.n_rows = n_rows; g.K = Kdim; g.lda = lda; g.x = x; g.ldx = ldx; g.NB = (2 * rows + 15) / 16 * 16; g.R = rows;
         g.status = ws.status;
+        g.wait_limit_ns = c.wait_limit_ns;
+        g.extra_arrivals = inject_left > 0 ? 1 : 0;      // self-test: the call's first GEMM waits for a copy that never comes
+        if (inject_left > 0) --inject_left;
         const int n_tiles = (n_rows + kGemmTileM - 1) / kGemmTileM, n_kb = (Kdim + kGemmBK - 1) / kGemmBK;
         g.splits = g.epi == EPI_PARTIAL ? pick_splits(n_tiles, n_kb, c.n_sm) : 1;
         g.kb_per_split = (n_kb + g.splits - 1) / g.splits;
@@ -884,7 +892,7 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
             AttnArgs a{};
             a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.dh = sh.dh; a.page = sh.page; a.max_ctx = sh.max_ctx; a.geo = geo;
             a.max_chunks = ws.max_chunks; a.q = ws.q; a.kv = kv; a.att_part = ws.att_part; a.status = ws.status;
-            a.page_shift = page_shift; a.B = rows;
+            a.page_shift = page_shift; a.B = rows; a.wait_limit_ns = c.wait_limit_ns;
             ++*launches;
             if (sh.dh == 128) rc = (int)launch_chained(attn_kernel<128>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
             else rc = (int)launch_chained(attn_kernel<64>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
@@ -958,6 +966,7 @@ int batched_target(const BatchedTargetCall &c, cudaStream_t st, long long *launc
     auto gemm = [&](GemmArgs &g, int n_rows, int Kdim, int lda, const bf16_t *x, int ldx) -> int {
         g.n_rows = n_rows; g.K = Kdim; g.lda = lda; g.x = x; g.ldx = ldx; g.NB = NB; g.R = R;
         g.status = ws.status;
+        g.wait_limit_ns = c.wait_limit_ns;
         const int n_tiles = (n_rows + kGemmTileM - 1) / kGemmTileM, n_kb = (Kdim + kGemmBK - 1) / kGemmBK;
         g.splits = g.epi == EPI_PARTIAL ? pick_splits(n_tiles, n_kb, c.n_sm) : 1;
         g.kb_per_split = (n_kb + g.splits - 1) / g.splits;
@@ -1008,7 +1017,7 @@ int batched_target(const BatchedTargetCall &c, cudaStream_t st, long long *launc
             AttnArgs a{};
             a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.dh = sh.dh; a.page = sh.page; a.max_ctx = sh.max_ctx; a.geo = geo;
             a.max_chunks = ws.max_chunks; a.q = ws.q; a.kv = kv; a.att_part = ws.att_part; a.status = ws.status;
-            a.page_shift = page_shift; a.B = R;
+            a.page_shift = page_shift; a.B = R; a.wait_limit_ns = c.wait_limit_ns;
             ++*launches;
             if (sh.dh == 128) rc = (int)launch_chained(attn_kernel<128>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);
             else rc = (int)launch_chained(attn_kernel<64>, dim3(c.n_sm), dim3(2 * kAttnThreads), attn_smem, st, a);

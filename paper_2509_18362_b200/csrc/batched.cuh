@@ -1,13 +1,20 @@
-// Batched draft path: the K recursive MTP steps for 5..64 sequences per group as a sequence of
-// kernels on one stream, with every weight matrix streamed once per step by the tcgen05 GEMM of
-// skinny_gemm.cuh. (Up to four or eight sequences run in the persistent kernel of megakernel.cu.)
+// Batched path of the draft and target calls: groups of up to 64 activation rows run as a sequence of kernels
+// on one stream, with every weight matrix streamed once per step and group by the tcgen05 GEMM of
+// skinny_gemm.cuh. (Calls whose rows fit one launch of the persistent kernel of megakernel.cu -- up to 8 rows,
+// and fewer than 3 sequences at 7B-class widths -- run there instead.)
 #pragma once
 #include "mega.cuh"
 
 namespace fmtp {
 
 constexpr int kBatchRows = 64;        // sequences per group (activation columns = 2 x rows <= 128)
-constexpr int kBatchAttnChunk = 256;  // context tokens per attention work item
+constexpr int kBatchAttnChunk = 256;  // fewest context tokens per attention work item (sizes the partial buffer)
+// Context tokens per attention work item for a row that sees n_ctx positions. An item ends with serial work (the
+// compute warps merge their partials and write the chunk's) while the K/V stream of the next items waits, so long
+// contexts take four times longer items (measured at 64 sequences with contexts in [512, 8192]: -13 us of 393 per
+// step); up to 4096 positions a row keeps 256-token items so that a small batch still spreads over all SMs. The size
+// is a function of the row's own context only: a row's summation order does not depend on the batch it is in.
+__host__ __device__ inline int attn_chunk_tokens(int n_ctx) { return n_ctx > 4096 ? 1024 : kBatchAttnChunk; }
 constexpr int kBatchMaxSplits = 8;
 
 // What the launches of the batched path would otherwise ask the driver for on every call; lives in the context
@@ -56,6 +63,8 @@ struct BatchedCall {
     const float *rope_cos, *rope_sin;     // [max_ctx][dh/2]
     int n_sm, smem_optin;
     TmapCache *cache;
+    unsigned long long wait_limit_ns;     // every device-side wait gives up after this long
+    int inject_gemm_timeout;              // self-test: the call's first GEMM expects a copy that is never made
     int B, K, N;
     const int32_t *ids;                   // subset or NULL
     int M0;                               // extend rows per sequence in step 0 (layout of h_last / tok_last), >= 1
@@ -77,6 +86,7 @@ struct BatchedTargetCall {
     const float *rope_cos, *rope_sin;
     int n_sm, smem_optin;
     TmapCache *cache;
+    unsigned long long wait_limit_ns;
     int B, M, n_layers;                   // B * M <= kBatchRows rows
     const int32_t *tokens;                // [B][M]
     bf16_t *out_h;                        // [B][M][d] or NULL

@@ -60,6 +60,8 @@ struct MegaParams {
     int scratch_smem;                 // bytes of the per-phase shared scratch region
     int max_chunks;                   // capacity of att_part's chunk dimension
     int max_ctx;                      // rows of the rotary table
+    unsigned long long wait_limit_ns; // every device-side wait gives up after this long (2 s outside the self-test)
+    int extra_arrivals;               // self-test only: arrivals the grid barrier expects beyond the CTAs that exist
     // call
     int mode;                         // 0: MTP draft, 1: target step
     int B, M, R;                      // sequences, rows per sequence (draft: extend rows of step 0), R = B*M

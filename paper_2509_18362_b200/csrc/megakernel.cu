@@ -38,7 +38,6 @@ namespace {
 
 constexpr uint32_t kDevBadToken = 0x1u, kDevBadPage = 0x2u, kDevBadPos = 0x4u, kDevTimeout = 0x8u,
                    kDevAllNan = 0x10u;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait gives up after 2 s
 
 
 enum Kind { PROJ = 0, QKV = 1, OPROJ = 2, GATEUP = 3, DOWN = 4, HEAD = 5, ATTN = 6, EMBED = 7, MERGE = 8, DONE = 9 };
@@ -111,7 +110,8 @@ __device__ __forceinline__ bool aborted(const Cta &c) { return *((volatile uint3
 
 // Bounded wait on an mbarrier phase (kept inline: a real call makes ptxas ignore setmaxnreg), called
 // from every ring wait. Returns false on timeout or abort, after setting the status bits.
-__device__ __forceinline__ bool wait_bar_impl(Misc *misc, uint64_t *bar, uint32_t parity, uint32_t *abort_flag, uint32_t *status) {
+__device__ __forceinline__ bool wait_bar_impl(Misc *misc, uint64_t *bar, uint32_t parity, uint32_t *abort_flag, uint32_t *status,
+                                              unsigned long long limit_ns) {
     if (*((volatile uint32_t *)&misc->aborted) != 0) return false;
     unsigned long long t0 = 0;
     for (uint32_t n = 0;; ++n) {
@@ -123,7 +123,7 @@ __device__ __forceinline__ bool wait_bar_impl(Misc *misc, uint64_t *bar, uint32_
             }
             unsigned long long now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) break;
+            else if (now - t0 > limit_ns) break;
         }
     }
     misc->aborted = 1;
@@ -133,7 +133,7 @@ __device__ __forceinline__ bool wait_bar_impl(Misc *misc, uint64_t *bar, uint32_
 }
 __device__ __forceinline__ bool wait_bar(const Cta &c, uint64_t *bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;          // fast path: already complete
-    return wait_bar_impl(c.misc, bar, parity, c.p->s.abort_flag, c.p->s.status);
+    return wait_bar_impl(c.misc, bar, parity, c.p->s.abort_flag, c.p->s.status, c.p->wait_limit_ns);
 }
 __device__ __forceinline__ void do_abort(const Cta &c) {
     c.misc->aborted = 1;
@@ -144,7 +144,7 @@ __device__ __forceinline__ void do_abort(const Cta &c) {
 // Grid-wide barrier among the consumer threads of all CTAs (the producer warp never joins).
 __device__ __forceinline__ void grid_barrier(Cta &c) {
     bar_sync(1, kConsumerThreads);
-    c.bar_target += (uint32_t)c.grid;
+    c.bar_target += (uint32_t)(c.grid + c.p->extra_arrivals);     // extra_arrivals: 0, or 1 in the wait-timeout self-test
     if (c.tid == 0) {
         // the arrival is a release at device scope: it orders every write the CTA made before the bar.sync above
         // (the waiting side reads with acquire), so no separate fences are needed
@@ -157,7 +157,7 @@ __device__ __forceinline__ void grid_barrier(Cta &c) {
                     if (ldcg_u32(c.p->s.abort_flag) != 0) { c.misc->aborted = 1; break; }
                     unsigned long long now = global_timer_ns();
                     if (t0 == 0) t0 = now;
-                    else if (now - t0 > kWaitLimitNs) { do_abort(c); break; }
+                    else if (now - t0 > c.p->wait_limit_ns) { do_abort(c); break; }
                 }
             }
         }
@@ -218,10 +218,7 @@ __device__ __forceinline__ int out_row(const MegaParams &p, int r, int step) {
 // ---- phase geometry ----------------------------------------------------------------------
 // rows x K of the phase's matrix, tile height, this CTA's row range, and how K is cut into ring stages:
 // into segments of seglen (the projection has two, one per input vector; every other phase one) and each
-// segment into nks_seg stages of kc elements (the last one shorter). A stage slot holds 32 KB; a phase whose
-// CTAs own at most 25 rows (d x d-like matrices at the 7B width: 24-25 rows per CTA) takes 640 instead of 512
-// elements per stage, so that its stages are as full as those of the 32-row phases: the bytes a CTA has in
-// flight, not its issue rate, set its share of the HBM bandwidth.
+// segment into nks_seg stages of kc = KC elements (the last one shorter).
 struct Geom { int rows, K, cap, nks, v0, v1, kc, rs, seglen, nks_seg; };
 struct StageK { int koff, klen; };
 __device__ __forceinline__ StageK stage_k(const Geom &g, int ks) {
@@ -246,13 +243,7 @@ __device__ __forceinline__ Geom geom(const Cta &c, int kind) {
     g.cap = (kind == GATEUP) ? kTileRows / 2 : kTileRows;
     g.v0 = (int)(((long long)c.cta * g.rows) / c.grid);
     g.v1 = (int)(((long long)(c.cta + 1) * g.rows) / c.grid);
-    const int per_cta = (g.rows + c.grid - 1) / c.grid;                              // most rows any CTA owns
-    const int stage_rows = (kind == GATEUP) ? 2 * min(g.cap, per_cta) : min(g.cap, per_cta);
-#ifdef FMTP_X_NO640
     g.kc = p.KC;
-#else
-    g.kc = (p.KC == 512 && stage_rows * 1280 <= p.stage_bytes) ? 640 : p.KC;
-#endif
     g.rs = g.kc * 2;
     g.seglen = (kind == PROJ) ? p.d : g.K;
     g.nks_seg = (g.seglen + g.kc - 1) / g.kc;
@@ -353,9 +344,11 @@ __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs 
             const int klen = sk.klen;
             const uint32_t dst0 = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + (uint32_t)pw * rs + lane16d;
             const size_t koff = (size_t)sk.koff * 2 + lane16;
-            if (p.KC == 512 && (klen & 31) == 0) {
-                // up to 1536 bytes per row in 512-byte pieces, one instruction per piece and lane, all
-                // with their own address registers (the piece offsets are immediates)
+            if (klen == 512) {
+                // the stage width of the large shapes, from fully unrolled code: two 512-byte pieces per row, one
+                // instruction per piece and lane, all with their own address registers (the piece offsets are
+                // immediates). The loop is this tight on purpose: a predicate or branch per instruction costs
+                // several per cent of the stream rate (measured: -5 % with three predicated pieces per row).
                 uint32_t d[kRowsPerProducer];
                 const unsigned char *q[kRowsPerProducer];
 #pragma unroll
@@ -363,14 +356,11 @@ __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs 
                     q[i] = cur[i] + koff;
                     d[i] = dst0 + (uint32_t)(i * kProducerWarps) * rs;
                 }
-                const int k0 = c.lane * 8;
-                const bool p0 = k0 < klen, p1 = k0 + 256 < klen, p2 = k0 + 512 < klen;
 #pragma unroll
                 for (int i = 0; i < kRowsPerProducer; ++i) {
                     if (cur[i] != nullptr) {
-                        if (p0) asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(d[i]), "l"(q[i]), "l"(pol) : "memory");
-                        if (p1) asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0+512], [%1+512], 16, %2;" ::"r"(d[i]), "l"(q[i]), "l"(pol) : "memory");
-                        if (p2) asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0+1024], [%1+1024], 16, %2;" ::"r"(d[i]), "l"(q[i]), "l"(pol) : "memory");
+                        asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(d[i]), "l"(q[i]), "l"(pol) : "memory");
+                        asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0+512], [%1+512], 16, %2;" ::"r"(d[i]), "l"(q[i]), "l"(pol) : "memory");
                     }
                 }
             } else {
@@ -524,15 +514,12 @@ __device__ __forceinline__ void mma_chunk(float (&acc)[2][2][4], const Frag &f, 
     mma_bf16(acc[0][1], f.u0.z, f.v0.z, f.u0.w, f.v0.w, b.z, b.w);
     mma_bf16(acc[1][1], f.u1.z, f.v1.z, f.u1.w, f.v1.w, b.z, b.w);
 }
-// Rows g, g + 8, g + 16 and g + 24 of the stage. off24 is 24 * rs, or 0 where row g + 24 lies beyond the rows a
-// stage slot holds at this row stride (25 rows of 640 elements): that row is never a valid tile row, its
-// products are discarded, and the load must stay inside the slot.
-__device__ __forceinline__ Frag load_frag(uint32_t a, uint32_t rs, uint32_t off24) {
+__device__ __forceinline__ Frag load_frag(uint32_t a, uint32_t rs) {
     Frag f;
     f.u0 = lds128_u32(a);
     f.v0 = lds128_u32(a + 8 * rs);
     f.u1 = lds128_u32(a + 16 * rs);
-    f.v1 = lds128_u32(a + off24);
+    f.v1 = lds128_u32(a + 24 * rs);
     return f;
 }
 
@@ -575,7 +562,6 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
     const bool has0 = arow < R, has1 = two_sets && (arow + 4 < R);
     const size_t aoff0 = (size_t)arow * act.stride + t * 8, aoff1 = (size_t)(arow + 4) * act.stride + t * 8;
     const uint32_t rs = (uint32_t)geo.rs;
-    const uint32_t off24 = ((g + 25) * geo.rs <= p.stage_bytes) ? 24u * rs : 0u;
     const uint4 zero = make_uint4(0, 0, 0, 0);
     for (int vr0 = geo.v0; vr0 < geo.v1; vr0 += geo.cap) {
         const int nv = min(geo.cap, geo.v1 - vr0);
@@ -590,23 +576,35 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
                 acc[i][0][j] = acc[i][1][j] = acd[i][0][j] = acd[i][1][j] = 0.f;
                 acc0[i][j] = acd0[i][j] = 0.f;
             }
-        // activations read from global memory (the ffn-wide vector of the down projection is not staged
-        // in shared memory): this warp's B fragments of its next stage are fetched one stage ahead
-        constexpr int kCpw = 5;                                       // chunks a warp has in a stage: wi, wi + 4, ... (640 / 32 / 4)
-        uint4 bnext[kCpw] = {zero, zero, zero, zero, zero};
-        const bool gfast = !two_sets && !act.in_smem;
+        // Activations read from global memory (the ffn-wide vector of the down projection is not staged whole in
+        // shared memory). A warp needs 512 bytes of it per stage and activation row -- its four 32-element chunks,
+        // hi and lo part -- and fetches them one owned stage ahead with ONE 16-byte cp.async per lane into a small
+        // ring in the (otherwise unused) staging area, then reads its fragments from there: per-lane global loads
+        // straight into the fragment registers were four load instructions per stage and warp, a third on top of the
+        // producers' copies in the same load/store path, and held this phase a quarter below the others' stream rate.
+        constexpr int kCpw = 4;                                       // chunks a warp has in a full stage: wi, wi + 4, wi + 8, wi + 12
+        const bool gfast = !two_sets && !act.in_smem && 16 * R * 512 <= p.scratch_smem;      // the slice ring must fit the staging area
         // which half of the warps takes a stage depends only on the stage's index within the phase,
         // never on how many stages the CTA has seen before: the summation order of a row must not
         // depend on the batch or on earlier calls
         const int stage0 = ((vr0 - geo.v0) / geo.cap) * geo.nks;
-        if (gfast && has0) {
+        // slice ring: slot (stage index mod 4) x warp of the owning group x activation row x 512 bytes
+        const uint32_t slice_base = smem_u32(c.scr) + (uint32_t)(wi * R) * 512u;
+        auto slice_slot = [&](int sa) -> uint32_t { return slice_base + (uint32_t)((sa & 3) * 4 * R) * 512u; };
+        auto slice_fetch = [&](int sa, const StageK &sk) {           // lane = (chunk j, hi/lo, 16-byte piece)
+            const int j = c.lane >> 3, hl = (c.lane >> 2) & 1, tp = c.lane & 3;
+            const bf16_t *src = (hl ? act.lo : act.hi) + (size_t)sk.koff + (wi + 4 * j) * 32 + tp * 8;
+            const uint32_t dst = slice_slot(sa) + (uint32_t)c.lane * 16u;
+#pragma unroll 1
+            for (int r = 0; r < R; ++r)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)r * 512u), "l"(src + (size_t)r * act.stride) : "memory");
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+        if (gfast) {
             const int ks0 = ((stage0 & 1) == grp) ? 0 : 1;          // first stage this warp owns
             if (ks0 < geo.nks) {
                 const StageK s0 = stage_k(geo, ks0);
-                const int n0 = (s0.klen + 31) >> 5;
-#pragma unroll
-                for (int j = 0; j < kCpw; ++j)
-                    if (wi + 4 * j < n0) bnext[j] = ldcg128(abase + aoff0 + (size_t)s0.koff + (wi + 4 * j) * 32);
+                if (s0.klen == 512) slice_fetch(stage0 + ks0, s0);
             }
         }
 #pragma unroll 1
@@ -628,46 +626,42 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
                 const uint32_t sb = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + t * 16 + g * rs;
                 const int par = g & 1;                    // odd rows: 64-byte halves swapped
                 const size_t kbase = (size_t)sk.koff;
-                if (!two_sets && nchunk <= 4 * kCpw && (act.in_smem || gfast)) {
-                    // common case (at most four activation rows): this warp's chunks wi, wi + 4, ... in batches of
-                    // two, all loads of a batch issued before its MMAs
+                if (!two_sets && nchunk == 16 && (act.in_smem || gfast)) {
+                    // the stage width of the large shapes with at most four activation rows: this warp's chunks
+                    // wi, wi + 4, wi + 8, wi + 12 in two batches of two, all loads of a batch issued before its MMAs,
+                    // nothing predicated (see the producer: this loop sets the stream rate)
                     uint4 bq[kCpw];
                     if (act.in_smem) {
                         const uint32_t ab = smem_u32(abase + aoff0 + kbase);
 #pragma unroll
-                        for (int j = 0; j < kCpw; ++j) bq[j] = (has0 && wi + 4 * j < nchunk) ? lds128_u32(ab + (wi + 4 * j) * 64) : zero;
+                        for (int j = 0; j < kCpw; ++j) bq[j] = has0 ? lds128_u32(ab + (wi + 4 * j) * 64) : zero;
                     } else {
-#pragma unroll
-                        for (int j = 0; j < kCpw; ++j) bq[j] = bnext[j];
-                        if (has0 && ks + 2 < geo.nks) {
+                        // request the slices of the next owned stage, then wait for this stage's (requested one owned
+                        // stage ago) and read the fragments from the slice ring
+                        bool more = false;
+                        if (ks + 2 < geo.nks) {
                             const StageK s2 = stage_k(geo, ks + 2);
-                            const int n2 = (s2.klen + 31) >> 5;
-#pragma unroll
-                            for (int j = 0; j < kCpw; ++j)
-                                bnext[j] = (wi + 4 * j < n2) ? ldcg128(abase + aoff0 + (size_t)s2.koff + (wi + 4 * j) * 32) : zero;
+                            if (s2.klen == 512) { slice_fetch(stage0 + ks + 2, s2); more = true; }   // (a shorter last stage is read directly by the loop below)
                         }
+                        if (more) asm volatile("cp.async.wait_group 1;" ::: "memory");
+                        else asm volatile("cp.async.wait_group 0;" ::: "memory");
+                        __syncwarp();
+                        const uint32_t sl = slice_slot(stage0 + ks) + (uint32_t)(arow * 512 + ((g & 1) * 4 + t) * 16);
+#pragma unroll
+                        for (int j = 0; j < kCpw; ++j) bq[j] = has0 ? lds128_u32(sl + j * 128) : zero;
                     }
 #pragma unroll
                     for (int b2 = 0; b2 < 2; ++b2) {
                         const int ch = wi + 8 * b2;
-                        if (ch + 4 < nchunk) {
-                            Frag f0 = load_frag(sb + (ch ^ par) * 64, rs, off24);
-                            Frag f1 = load_frag(sb + ((ch + 4) ^ par) * 64, rs, off24);
-                            mma_chunk(acc, f0, bq[2 * b2]);
-                            mma_chunk(acc, f1, bq[2 * b2 + 1]);
-                        } else if (ch < nchunk) {
-                            Frag f0 = load_frag(sb + (ch ^ par) * 64, rs, off24);
-                            mma_chunk(acc, f0, bq[2 * b2]);
-                        }
-                    }
-                    if (wi + 16 < nchunk) {
-                        Frag f0 = load_frag(sb + ((wi + 16) ^ par) * 64, rs, off24);
-                        mma_chunk(acc, f0, bq[4]);
+                        Frag f0 = load_frag(sb + (ch ^ par) * 64, rs);
+                        Frag f1 = load_frag(sb + ((ch + 4) ^ par) * 64, rs);
+                        mma_chunk(acc, f0, bq[2 * b2]);
+                        mma_chunk(acc, f1, bq[2 * b2 + 1]);
                     }
                 } else {
 #pragma unroll 1
                     for (int ch = wi; ch < nchunk; ch += 4) {
-                        Frag f0 = load_frag(sb + (ch ^ par) * 64, rs, off24);
+                        Frag f0 = load_frag(sb + (ch ^ par) * 64, rs);
                         uint4 b0 = zero, d0 = zero;
                         if (has0) b0 = act.in_smem ? lds128(abase + aoff0 + kbase + ch * 32) : ldcg128(abase + aoff0 + kbase + ch * 32);
                         if (has1) d0 = act.in_smem ? lds128(abase + aoff1 + kbase + ch * 32) : ldcg128(abase + aoff1 + kbase + ch * 32);
@@ -1052,17 +1046,30 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int st
         bf16_t *sk = reinterpret_cast<bf16_t *>(c.ring + (size_t)slot * p.stage_bytes);
         bf16_t *sv = sk + (size_t)kAttnChunk * dh;
 
-        // -- rotated, pre-scaled queries of this KV head (independent of the stage)
-        for (int i = c.tid; i < M * Gq * half; i += kConsumerThreads) {
-            int qi = i / half, e = i - qi * half;
-            int m = qi / Gq, hq = kvh * Gq + (qi - m * Gq);
-            int r = b * M + m, pos = base + min(m, rows - 1);
-            if (pos >= max_tokens) pos = max_tokens - 1;
-            const float *q = p.s.qkv + (size_t)r * (p.qdim + 2 * p.kvdim) + hq * dh;
-            float x = ldcg_f32(q + e), y = ldcg_f32(q + e + half);
-            float cs = p.s.rope_cos[(size_t)pos * half + e], sn = p.s.rope_sin[(size_t)pos * half + e];
-            qs[qi * dh + e] = (x * cs - y * sn) * qscale;
-            qs[qi * dh + e + half] = (y * cs + x * sn) * qscale;
+        // -- rotated, pre-scaled queries of this KV head (independent of the stage); two elements per thread and
+        // round, all eight loads of a round issued before the first use (they are L2 round trips)
+        for (int i0 = c.tid; i0 < M * Gq * half; i0 += 2 * kConsumerThreads) {
+            float x[2], y[2], cs[2], sn[2];
+            int qi[2], e[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int i = min(i0 + u * kConsumerThreads, M * Gq * half - 1);
+                qi[u] = i / half; e[u] = i - qi[u] * half;
+                const int m = qi[u] / Gq, hq = kvh * Gq + (qi[u] - m * Gq);
+                const int r = b * M + m;
+                int pos = base + min(m, rows - 1);
+                if (pos >= max_tokens) pos = max_tokens - 1;
+                const float *q = p.s.qkv + (size_t)r * (p.qdim + 2 * p.kvdim) + hq * dh;
+                x[u] = ldcg_f32(q + e[u]); y[u] = ldcg_f32(q + e[u] + half);
+                cs[u] = p.s.rope_cos[(size_t)pos * half + e[u]]; sn[u] = p.s.rope_sin[(size_t)pos * half + e[u]];
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                if (i0 + u * kConsumerThreads < M * Gq * half) {
+                    qs[qi[u] * dh + e[u]] = (x[u] * cs[u] - y[u] * sn[u]) * qscale;
+                    qs[qi[u] * dh + e[u] + half] = (y[u] * cs[u] + x[u] * sn[u]) * qscale;
+                }
+            }
         }
         PROF(c, ATTN * 8 + 3);
         wait_bar(c, &c.misc->full[slot], parity);

@@ -32,7 +32,6 @@ constexpr int kGemmThreads = 160 + kGemmProducers;
 constexpr int kGemmBK = 64;                 // K elements per swizzled block: one 128-byte row
 constexpr int kGemmTileM = 128;
 constexpr int kGemmMaxStages = 10;
-constexpr unsigned long long kGemmWaitNs = 2000000000ull;
 
 enum GemmEpilogue {
     EPI_PARTIAL = 0,   // fp32 partial sums  partial[split][r][m] = D[m,2r] + D[m,2r+1]
@@ -65,6 +64,8 @@ struct GemmArgs {
     uint32_t *status;
     int n_stages;
     int force_ka;                // 0: pick the blocks per stage from the shared memory available
+    unsigned long long wait_limit_ns;   // every wait of the kernel gives up after this long
+    int extra_arrivals;          // self-test only: arrivals a ring stage expects beyond the copies that are made
 };
 
 struct GemmSmem {
@@ -78,20 +79,38 @@ struct GemmSmem {
 __host__ __device__ inline int gemm_kblock_bytes(int NB) { return kGemmTileM * 128 + NB * 128; }
 __host__ __device__ inline int gemm_tile_rows(int epi) { return epi == EPI_SWIGLU ? 64 : kGemmTileM; }
 
-__device__ __forceinline__ bool gemm_wait(GemmSmem *sm, uint64_t *bar, uint32_t parity) {
+__device__ __forceinline__ bool gemm_wait(GemmSmem *sm, uint64_t *bar, uint32_t parity, unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     uint32_t polls = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++polls & 63u) == 0) {
             if (*reinterpret_cast<volatile uint32_t *>(&sm->abort_flag)) return false;
-            if (global_timer_ns() - t0 > kGemmWaitNs) {
+            if (global_timer_ns() - t0 > limit_ns) {
                 *reinterpret_cast<volatile uint32_t *>(&sm->abort_flag) = 1u;
                 return false;
             }
         }
     }
     return true;
+}
+
+// Work items of a CTA: items (tile of 128 rows, K range) are dealt round-robin over the CTAs. (Giving every CTA
+// an equal contiguous share of the output head's rows instead -- 221 rows as a full and a partial tile at the 7B
+// shape, where 256 tiles are 1.7 rounds of 148 CTAs -- was measured 3 % slower: the second round's 108 CTAs still
+// saturate HBM, and partial tiles cost issue slots.)
+struct GemmItem { int row0, row_end, split; };
+__device__ __forceinline__ int gemm_my_items(const GemmArgs &g, int n_items) {
+    return (int)blockIdx.x < n_items ? (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+}
+__device__ __forceinline__ GemmItem gemm_my_item(const GemmArgs &g, int i) {
+    GemmItem it;
+    const int item = (int)blockIdx.x + i * (int)gridDim.x;
+    const int tile = item / g.splits, tile_rows = gemm_tile_rows(g.epi);
+    it.split = item - tile * g.splits;
+    it.row0 = tile * tile_rows;
+    it.row_end = min(it.row0 + tile_rows, g.n_rows);
+    return it;
 }
 
 // True on all 128 epilogue threads (warps 0-3) if `flag` is set on any of them.
@@ -127,6 +146,7 @@ struct GemmProducer {
     uint32_t dst_x;           // shared address of the X tile in block 0 of stage 0
     const CUtensorMap *xmap;
     uint64_t *full;
+    uint64_t policy;          // L2 eviction policy of the weight stream
 };
 
 // Copies this thread's share of K block kb + J (if it is inside the item) into block J of the
@@ -145,10 +165,10 @@ __device__ __forceinline__ void produce_kblock(const GemmArgs &g, const GemmProd
     const uint32_t dst = pr.dst0 + (uint32_t)pr.stage * pr.stage_bytes + (uint32_t)J * pr.kblock_bytes;
     if (kvalid && (aok[0] & aok[1] & aok[2] & aok[3]) != 0u) {      // the common case: plain 16-byte copies
 #pragma unroll
-        for (int i = 0; i < 4; ++i) cp_async16_full<J * 128>(dst + i * 4096, ap[i]);
+        for (int i = 0; i < 4; ++i) cp_async16_full_hint<J * 128>(dst + i * 4096, ap[i], pr.policy);
     } else if (kvalid) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) cp_async16_off<J * 128>(dst + i * 4096, ap[i], aok[i]);
+        for (int i = 0; i < 4; ++i) cp_async16_off_hint<J * 128>(dst + i * 4096, ap[i], aok[i], pr.policy);
     } else {   // this chunk column lies beyond K: zeros, nothing is read
 #pragma unroll
         for (int i = 0; i < 4; ++i) cp_async16_off<0>(dst + i * 4096, g.a[0], 0u);
@@ -183,7 +203,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
     while ((int)alloc_cols < 2 * buf_cols) alloc_cols <<= 1;
 
     if (tid == 0) {
-        for (int s = 0; s < S; ++s) { mbar_init(&sm->full[s], kGemmProducers + 1); mbar_init(&sm->empty[s], 1); }
+        for (int s = 0; s < S; ++s) { mbar_init(&sm->full[s], kGemmProducers + 1 + g.extra_arrivals); mbar_init(&sm->empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&sm->tfull[b], 1); mbar_init(&sm->tempty[b], 128); }
         mbar_init(&sm->drain, 1);
         sm->abort_flag = 0;
@@ -212,14 +232,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
         pr.dst0 = smem_u32(ring) + (uint32_t)(r0 * 128 + ((c ^ (r0 & 7)) << 4));
         pr.stage_bytes = stage_bytes; pr.kblock_bytes = kblock_bytes; pr.S = S; pr.c = c;
         pr.stage = 0; pr.phase = 0;
+        pr.policy = l2_evict_first();
         pr.tma_thread = pt == 0; pr.dst_x = smem_u32(ring) + 16384; pr.xmap = &xmap; pr.full = sm->full;
         bool ok_run = true;
         const bf16_t *ap[4];
         uint32_t aok[4];
         int kb0 = 0, kb1 = 0;
-        auto setup_item = [&](int item) {
-            const int tile = item / g.splits, split = item - tile * g.splits;
-            kb0 = split * g.kb_per_split;
+        auto setup_item = [&](int i) {
+            const GemmItem gi = gemm_my_item(g, i);
+            kb0 = gi.split * g.kb_per_split;
             kb1 = kb0 + g.kb_per_split;
             if (kb1 > n_kb) kb1 = n_kb;
 #pragma unroll
@@ -228,13 +249,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
                 const bf16_t *base = g.a[0];
                 int m;
                 if (g.epi == EPI_SWIGLU) {             // tile rows 0-63: gate rows, 64-127: the up rows of the same indices
-                    m = tile * 64 + (tr & 63);
+                    m = gi.row0 + (tr & 63);
                     if (tr >= 64) base = g.a_up;
                 } else {
-                    m = tile * kGemmTileM + tr;
+                    m = gi.row0 + tr;
                 }
-                aok[i] = m < g.n_rows ? 16u : 0u;
-                if (m >= g.n_rows) m = g.n_rows - 1;
+                aok[i] = m < gi.row_end ? 16u : 0u;
+                if (m >= gi.row_end) m = gi.row_end - 1;
                 int row = m;
                 if (g.row_ids) {
                     int id = g.row_ids[m];
@@ -250,9 +271,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
                 ap[i] = base + (size_t)row * g.lda + (size_t)kb0 * kGemmBK + c * 8;
             }
         };
-        // The weights (and the row ids, written several kernels ago) do not depend on the predecessor in the
-        // stream: the weight part of the first item's first stages goes out before waiting for it.
-        setup_item(blockIdx.x);
+        // The weights do not depend on the predecessor in the stream: the weight part of the first item's first
+        // stages goes out before waiting for it.
+        const int n_my = gemm_my_items(g, n_items);
+        // The gathered head reads its row ids, which a kernel earlier in the same call wrote: that is a real
+        // dependency, so those GEMMs wait for the chain first (and give up the early weight requests below).
+        if (g.row_ids) chain_wait();
+        if (n_my > 0) setup_item(0);
         int pre = 0;
         for (int kb = kb0; kb < kb1 && pre < S; kb += KA, ++pre) {
             pr.stage = pre;
@@ -262,10 +287,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
         }
         pr.stage = 0;
         chain_wait();
-        for (int item = blockIdx.x; item < n_items && ok_run; item += gridDim.x) {
-            if (item != (int)blockIdx.x) setup_item(item);
+        for (int i = 0; i < n_my && ok_run; ++i) {
+            if (i > 0) setup_item(i);
             for (int kb = kb0; kb < kb1; kb += KA) {
-                if (!gemm_wait(sm, &sm->empty[pr.stage], pr.phase ^ 1u)) { ok_run = false; break; }
+                if (!gemm_wait(sm, &sm->empty[pr.stage], pr.phase ^ 1u, g.wait_limit_ns)) { ok_run = false; break; }
                 if (pr.tma_thread) {   // the X tiles of this stage: their bytes are expected on the stage's barrier
                     const int nv = kb1 - kb < KA ? kb1 - kb : KA;
                     mbar_arrive_expect_tx(&sm->full[pr.stage], (uint32_t)(nv * g.NB * 128));
@@ -293,16 +318,16 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
             uint32_t phase = 0, tphase[2] = {0, 0};
             int buf = 0;
             bool ok_run = true;
-            for (int item = blockIdx.x; item < n_items && ok_run; item += gridDim.x) {
-                const int tile = item / g.splits, split = item - tile * g.splits;
-                const int kb0 = split * g.kb_per_split;
+            const int n_my = gemm_my_items(g, n_items);
+            for (int i = 0; i < n_my && ok_run; ++i) {
+                const int kb0 = gemm_my_item(g, i).split * g.kb_per_split;
                 int kb1 = kb0 + g.kb_per_split;
                 if (kb1 > n_kb) kb1 = n_kb;
-                if (!gemm_wait(sm, &sm->tempty[buf], tphase[buf] ^ 1u)) break;
+                if (!gemm_wait(sm, &sm->tempty[buf], tphase[buf] ^ 1u, g.wait_limit_ns)) break;
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + (uint32_t)(buf * buf_cols);
                 for (int kb = kb0; kb < kb1; kb += KA) {
-                    if (!gemm_wait(sm, &sm->full[stage], phase)) { ok_run = false; break; }
+                    if (!gemm_wait(sm, &sm->full[stage], phase, g.wait_limit_ns)) { ok_run = false; break; }
                     fence_proxy_async();          // the copies' shared-memory writes, before the tensor core reads them
                     tc_fence_after_sync();
 #pragma unroll
@@ -326,7 +351,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
             }
             // every MMA issued above has completed once this arrival lands
             umma_commit(&sm->drain);
-            gemm_wait(sm, &sm->drain, 0);
+            gemm_wait(sm, &sm->drain, 0, g.wait_limit_ns);
         }
         __syncwarp();
     } else {
@@ -334,14 +359,16 @@ __global__ void __launch_bounds__(kGemmThreads, 1) skinny_gemm_kernel(const Gemm
         chain_wait();
         uint32_t tphase[2] = {0, 0};
         int buf = 0;
-        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-            const int tile = item / g.splits, split = item - tile * g.splits;
+        const int n_my = gemm_my_items(g, n_items);
+        for (int i = 0; i < n_my; ++i) {
+            const GemmItem gi = gemm_my_item(g, i);
+            const int split = gi.split;
             // the 128 epilogue threads agree on the outcome of the wait before any of them moves on
-            if (epi_any(!gemm_wait(sm, &sm->tfull[buf], tphase[buf]))) break;
+            if (epi_any(!gemm_wait(sm, &sm->tfull[buf], tphase[buf], g.wait_limit_ns))) break;
             tc_fence_after_sync();
             const int tr = warp * 32 + lane;
-            const int m = g.epi == EPI_SWIGLU ? tile * 64 + (tr & 63) : tile * kGemmTileM + tr;
-            const bool m_ok = m < g.n_rows;
+            const int m = g.epi == EPI_SWIGLU ? gi.row0 + (tr & 63) : gi.row0 + tr;
+            const bool m_ok = m < gi.row_end;
             const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * buf_cols);
             uint32_t row_id = (uint32_t)m;
             if (g.epi == EPI_ARGMAX && g.row_ids && m_ok) {

@@ -84,10 +84,23 @@ __device__ __forceinline__ void cp_async16_off(uint32_t dst_smem, const void *sr
     asm volatile("cp.async.cg.shared.global [%0], [%1+%2], 16, %3;" ::"r"(dst_smem), "l"(src), "n"(OFF), "r"(src_bytes)
                  : "memory");
 }
-// The same copy without the source-size operand (always 16 bytes).
+// The same copies with an L2 eviction policy (see l2_evict_first): for data that is read once per step.
 template <int OFF>
-__device__ __forceinline__ void cp_async16_full(uint32_t dst_smem, const void *src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1+%2], 16;" ::"r"(dst_smem), "l"(src), "n"(OFF) : "memory");
+__device__ __forceinline__ void cp_async16_off_hint(uint32_t dst_smem, const void *src, uint32_t src_bytes, uint64_t policy) {
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1+%2], 16, %3, %4;" ::"r"(dst_smem), "l"(src), "n"(OFF),
+                 "r"(src_bytes), "l"(policy) : "memory");
+}
+template <int OFF>
+__device__ __forceinline__ void cp_async16_full_hint(uint32_t dst_smem, const void *src, uint64_t policy) {
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1+%2], 16, %3;" ::"r"(dst_smem), "l"(src), "n"(OFF), "l"(policy)
+                 : "memory");
+}
+// Weights and cached K/V are streamed once per step: marked evict-first they do not push out of L2 what the step
+// keeps re-reading (the activation operand every tile re-reads, partial sums, the kernels' own code).
+__device__ __forceinline__ uint64_t l2_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait_group() {

@@ -126,5 +126,6 @@ def speculative_decode(tgt: Target, mtp_w, mtp_kv, subset, prompt, n_new, K, inj
     assert int(status.item()) == 0 and int(tgt.status.item()) == 0, "a kernel flagged an out-of-range id, page or position"
     emitted = sum(a + 1 for a in accepted)
     stats = {"accepted": accepted, "tau": emitted / max(1, len(accepted)), "target_calls": tgt.calls - calls0,
+             "pending_pairs": len(pend_t),      # committed by the target, not yet in the MTP cache (the next round's extend rows)
              "accept_rate_by_position": [float(np.mean([a > k for a in accepted])) for k in range(K)] if accepted else []}
     return out[:n_new], stats

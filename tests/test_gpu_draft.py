@@ -464,6 +464,48 @@ def test_draft_call_captured_in_a_cuda_graph_replays_on_the_current_state(B, K):
     ctx.close()
 
 
+@pytest.mark.parametrize("which,B", [(1, 2), (2, 12)])
+def test_a_wait_inside_the_draft_kernels_runs_out_and_the_context_stays_usable(which, B):
+    """Failure detection without a fault, in the kernels' own code: the next draft call is armed so that the
+    persistent kernel's grid barrier (which = 1) or a ring stage of the batched path's first GEMM (which = 2) waits
+    for an arrival that never comes, with a 20 ms limit. The wait gives up, FMTP_DEV_TIMEOUT reaches the status word,
+    the other CTAs and warp roles stop waiting, the call returns in bounded time, and the same context then gives the
+    bits it gave before."""
+    import time
+    Bd = _binding()
+    shape, K, seed = I.TINY, 2, 7300 + which
+    L = [int(x) for x in I.context_lengths(B, 0, 100, seed)]
+    W = I.mtp_weights(shape, seed)
+    kv = I.paged_kv(shape, L, K + 1, seed + 1)
+    dW = Bd.to_device(W)
+    dh = Bd.bf16_tensor(I.hidden_bf16(seed + 2, (B, shape.d)))
+    dtok = torch.from_numpy(I.token_ids(seed + 3, (B,), shape.vocab)).cuda()
+    dids = torch.from_numpy(I.subset_uniform(shape.vocab, 1024, seed + 4)).cuda()
+    ctx = Bd.Context(shape, max_rows=16, max_K=8, max_ctx=128)
+
+    def run():
+        dkv = Bd.to_device(copy_kv(kv))
+        out_d = torch.full((B, K), -1, dtype=torch.int32, device="cuda")
+        out_h = torch.zeros((B, K, shape.d), dtype=torch.bfloat16, device="cuda")
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        t0 = time.time()
+        ctx.fastmtp_draft(Bd.mtp_w(dW), dh, dtok, Bd.kv(dkv), B, K, dids, out_d, out_h, None, st)
+        torch.cuda.synchronize()
+        return out_d.cpu().numpy(), Bd.bf16_bits(out_h), int(st.item()), time.time() - t0
+
+    d0, h0, st0, _ = run()
+    assert st0 == 0
+    ctx.fmtp_selftest_inject_wait_timeout(20, which)
+    _, _, st1, dt = run()
+    assert st1 & Bd.DEV_TIMEOUT
+    assert 0.015 < dt < 2.0                                  # gave up soon after the limit, nothing hung
+    d2, h2, st2, _ = run()                                   # the arming was for one call; tensor memory and barriers are clean
+    assert st2 == 0 and np.array_equal(d2, d0) and np.array_equal(h2, h0)
+    with pytest.raises(Bd.FastMTPError):
+        ctx.fmtp_selftest_inject_wait_timeout(5000, which)   # limits above one second are refused on the host
+    ctx.close()
+
+
 def test_host_entry_point_matches_device_entry_point():
     Bd = _binding()
     shape = I.TINY

@@ -244,7 +244,8 @@ def speculative_vs_greedy(shape, seed, K, n_new, prompt_len, N, max_ctx, n_oracl
         return list(good[:n_ok]) + [(t + 1) % shape.vocab for t in good[n_ok:]]
 
     out, stats = loop.speculative_decode(tgt, Bd.mtp_w(dWm), mkv, torch.from_numpy(ids).cuda(), prompt, n_new, K, inject)
-    assert int(mkv["seq_lens"].item()) == int(tgt.dkvs[0]["seq_lens"].item())   # MTP and target caches committed alike
+    # the MTP cache trails the target's by exactly the pairs the next round would extend it with
+    assert int(mkv["seq_lens"].item()) + stats["pending_pairs"] == int(tgt.dkvs[0]["seq_lens"].item())
     ctx.close()
     exempt = oracle_checks_greedy_tokens(shape, Wt, prompt, ref[:n_oracle], mk)
     O.clear_weight_memo()
