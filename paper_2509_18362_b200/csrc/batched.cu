@@ -707,43 +707,67 @@ __global__ void ids_mark_kernel(const int32_t *ids, int N, int V, uint32_t *bitm
     }
 }
 
-__global__ void __launch_bounds__(1024) ids_compact_kernel(const uint32_t *bitmap, int n_words, int32_t *sorted, int N) {
+// Compaction of the membership bitmap into ascending ids. Block b owns a contiguous range of bitmap words; the
+// number of ids before its range is the population count of all earlier words, which every block sums for itself
+// (the whole bitmap is 19 KB at V = 152064), so no block waits for another. Duplicates in the caller's array leave
+// fewer distinct ids than N: the tail repeats `fill` (a member of the subset; a repeated row cannot change an argmax).
+constexpr int kCompactThreads = 256;
+__global__ void __launch_bounds__(kCompactThreads) ids_compact_kernel(const uint32_t *bitmap, int n_words, int32_t *sorted, int N,
+                                                                      const int32_t *ids, int V) {
     chain_release();
     chain_wait();
-    __shared__ int warp_tot[32];
-    __shared__ int s_total, s_last;
+    __shared__ int wsum[kCompactThreads / 32];
+    __shared__ int s_base, s_total;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int per = (n_words + 1023) / 1024;
-    const int w0 = tid * per, w1 = min(w0 + per, n_words);
-    int cnt = 0;
-    for (int w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
-    int incl = cnt;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
+    const int w0 = (int)(((long long)blockIdx.x * n_words) / gridDim.x), w1 = (int)(((long long)(blockIdx.x + 1) * n_words) / gridDim.x);
+    // ids before this block's words, and in the whole bitmap
+    int before = 0, all = 0;
+    for (int w = tid; w < n_words; w += kCompactThreads) {
+        const int c = __popc(bitmap[w]);
+        all += c;
+        if (w < w0) before += c;
     }
-    if (lane == 31) warp_tot[warp] = incl;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { before += __shfl_xor_sync(0xffffffffu, before, o); all += __shfl_xor_sync(0xffffffffu, all, o); }
+    if (lane == 0) wsum[warp] = before;
     __syncthreads();
-    int base = 0;
-    for (int w = 0; w < warp; ++w) base += warp_tot[w];
-    if (tid == 1023) s_total = base + incl;
-    int pos = base + incl - cnt;
-    for (int w = w0; w < w1; ++w) {
-        uint32_t bits = bitmap[w];
+    if (tid == 0) { int t = 0; for (int w = 0; w < kCompactThreads / 32; ++w) t += wsum[w]; s_base = t; }
+    __syncthreads();
+    if (lane == 0) wsum[warp] = all;
+    __syncthreads();
+    if (tid == 0) { int t = 0; for (int w = 0; w < kCompactThreads / 32; ++w) t += wsum[w]; s_total = t; }
+    __syncthreads();
+    // this block's words: one word per thread and round, exclusive scan of the counts within the block
+    int run = s_base;
+    for (int r0 = w0; r0 < w1; r0 += kCompactThreads) {
+        const int w = r0 + tid;
+        uint32_t bits = w < w1 ? bitmap[w] : 0u;
+        const int cnt = __popc(bits);
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        __syncthreads();
+        if (lane == 31) wsum[warp] = incl;
+        __syncthreads();
+        int base = run;
+        for (int q = 0; q < warp; ++q) base += wsum[q];
+        int pos = base + incl - cnt;
         while (bits) {
             const int b = __ffs(bits) - 1;
             bits &= bits - 1;
             if (pos < N) sorted[pos] = w * 32 + b;
             ++pos;
         }
+        for (int q = 0; q < kCompactThreads / 32; ++q) run += wsum[q];
     }
-    __syncthreads();
-    // duplicates in the caller's array leave fewer distinct ids than N: repeat the last one
-    const int total = min(s_total, N);
-    if (tid == 0) s_last = sorted[total - 1];
-    __syncthreads();
-    for (int j = total + tid; j < N; j += 1024) sorted[j] = s_last;
+    if (blockIdx.x == 0) {
+        int fill = ids[0];
+        if ((unsigned)fill >= (unsigned)V) fill = 0;
+        for (int j = min(s_total, N) + tid; j < N; j += kCompactThreads) sorted[j] = fill;
+    }
 }
 
 int pick_splits(int n_tiles, int n_kb, int n_sm) {
@@ -814,7 +838,7 @@ int batched_draft(const BatchedCall &c, cudaStream_t st, long long *launches) {
         if (e != cudaSuccess) return (int)e;
         e = launch_chained(ids_mark_kernel, dim3((c.N + 255) / 256 < 1024 ? (c.N + 255) / 256 : 1024), dim3(256), 0, st, c.ids, c.N, sh.V,
                            ws.id_bitmap, ws.status);
-        if (e == cudaSuccess) e = launch_chained(ids_compact_kernel, dim3(1), dim3(1024), 0, st, ws.id_bitmap, n_words, ws.sorted_ids, c.N);
+        if (e == cudaSuccess) e = launch_chained(ids_compact_kernel, dim3(32), dim3(kCompactThreads), 0, st, ws.id_bitmap, n_words, ws.sorted_ids, c.N, c.ids, sh.V);
         *launches += 2;
         if (e != cudaSuccess) return (int)e;
         head_ids = ws.sorted_ids;
