@@ -1,7 +1,11 @@
 """Benchmark of the FastMTP draft / verify hot path.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--batch B] [--subset N] [--ctx L] [--draft-steps K] [--subset-kind uniform|zipf]
+                    [--batch B] [--subset N] [--ctx L | --ctx-min A --ctx-max B] [--draft-steps K]
+                    [--subset-kind uniform|zipf] [--no-cpu-baseline]
+    python bench.py --sweep                      subset x batch x K table (one JSON line per point)
+    python bench.py --target-layers L [--batch B]  fastmtp_target_step on a random L-layer target
+    python bench.py --e2e-loop                   greedy vs speculative decoding loops at full depth, oracle-checked
 
 One step = one pass of the hot path over one batch of synthetic input: fastmtp_draft (the K
 recursive MTP steps with the compressed-vocabulary head, one kernel launch) followed by

@@ -41,8 +41,9 @@ struct fmtp_ctx {
     BatchedShape bsh;
     BatchedWs bws;
     int batched_min;           // calls with at least this many sequences take the batched path (env FMTP_BATCHED_MIN)
+    int tmem_staging;          // the persistent kernel stages weights through tensor memory where the shape allows (env FMTP_TMEM=1)
     // answers that depend on the geometry only, kept so that the hot calls make no CUDA attribute / occupancy query:
-    struct { size_t smem; int grid; } mega_cfg[4];                 // per kernel instantiation: footprint its limit was raised to
+    struct { size_t smem; int grid; } mega_cfg[6];                 // per kernel instantiation: footprint its limit was raised to
     struct { int mode, B, M, G; } group_memo[16];                  // sequences per launch for (mode, B, M)
     int n_group_memo;
     TmapCache tmaps;                                               // tensor maps of the batched path's GEMM operands
@@ -166,7 +167,13 @@ int configure(fmtp_ctx *c, MegaParams &p, int mode, int B, int M) {
     // the ffn-wide input of the down projection is used once per CTA: it is read from global memory (L2), one
     // stage ahead, and the shared memory goes to a deeper ring
     p.scratch_smem = (int)base;
-    int ns = fixed + base < avail ? (int)((avail - fixed - base) / p.stage_bytes) : 0;
+    // tensor memory as a second staging level: full-width stages only (every K a multiple of the stage width), at most
+    // four activation rows, the down projection's slice ring inside the staging area
+    p.use_tmem = c->tmem_staging && R <= 4 && p.KC == 512 && p.stage_bytes == kTileRows * 512 * 2 && p.d % 512 == 0 &&
+                 p.qdim % 512 == 0 && p.F % 512 == 0 && (size_t)16 * R * 512 <= base;
+    size_t ring_off = fixed + base;
+    if (p.use_tmem) ring_off = align_up(ring_off, 1024) + 1024;        // as mega_smem_bytes lays it out
+    int ns = ring_off < avail ? (int)((avail - ring_off) / p.stage_bytes) : 0;
     if (ns > kMaxStages) ns = kMaxStages;
     if (ns < 2) return FMTP_ESHAPE;
     p.n_stages = ns;
@@ -301,6 +308,8 @@ int fmtp_create(const fmtp_shape *sh, fmtp_ctx **out) {
         if (layer_bytes >= 256e6 && c->batched_min > 3) c->batched_min = 3;
     }
     if (const char *v = std::getenv("FMTP_BATCHED_MIN")) { int n = std::atoi(v); if (n >= 1) c->batched_min = n; }
+    c->tmem_staging = 0;       // measured slower than the plain ring so far: opt-in
+    if (const char *v = std::getenv("FMTP_TMEM")) c->tmem_staging = std::atoi(v) != 0;
     c->pinned_bytes = (size_t)sh->max_rows * sh->d * 2 + (size_t)sh->max_rows * 4 * (3 + (sh->max_K > 1 ? sh->max_K : 1)) +
                       2 * kVerifyMaxRows * 4 + 256;
     e = cudaMallocHost(&c->pinned, c->pinned_bytes);

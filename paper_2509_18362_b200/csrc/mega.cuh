@@ -18,6 +18,15 @@ constexpr int kConsumerRegs = 200;
 constexpr int kTileRows = 32;        // weight rows per pipeline stage (two 16-row MMA tiles)
 constexpr int kAttnChunk = 64;       // context tokens per attention work item
 constexpr int kMaxStages = 8;
+// Second staging level in tensor memory (see the kernel): a fourth warpgroup (one warp of it works) moves every landed
+// 32 KB weight stage from the shared-memory ring into one of eight 64-column slots of the SM's 256 KB tensor memory,
+// the consumers read their fragments from there. 512 threads launch with 128 registers each; the mover's warpgroup
+// and the producers hand back what takes the consumers to 192.
+constexpr int kTmThreads = 512;
+constexpr int kTmMoverRegs = 32;
+constexpr int kTmConsumerRegs = 192;
+constexpr int kTmSlots = 8;
+constexpr int kTmSlotCols = 64;
 
 typedef uint16_t bf16_t;
 
@@ -62,6 +71,7 @@ struct MegaParams {
     int max_ctx;                      // rows of the rotary table
     unsigned long long wait_limit_ns; // every device-side wait gives up after this long (2 s outside the self-test)
     int extra_arrivals;               // self-test only: arrivals the grid barrier expects beyond the CTAs that exist
+    int use_tmem;                     // weight stages pass through tensor memory (stage = 32 rows x 512, every K a multiple of 512, R <= 4)
     // call
     int mode;                         // 0: MTP draft, 1: target step
     int B, M, R;                      // sequences, rows per sequence (draft: extend rows of step 0), R = B*M
@@ -94,7 +104,8 @@ int mega_launch(const MegaParams &p, int grid, cudaStream_t stream);
 // Raises the shared-memory limit of the kernel these parameters select and returns the largest co-resident
 // grid for this footprint on the current device. The answer depends on (kernel, footprint) only: callers cache it.
 int mega_max_grid(const MegaParams &p, size_t smem_bytes, int *err);
-// Which of the kernel's instantiations (head dimension, more than four activation rows) the parameters select: 0..3.
+// Which of the kernel's instantiations (head dimension, more than four activation rows, tensor-memory staging) the
+// parameters select: 0..5.
 int mega_kernel_index(const MegaParams &p);
 
 // Verification kernel (verify.cu).

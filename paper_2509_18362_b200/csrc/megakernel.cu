@@ -24,11 +24,20 @@
 //   * Producers and consumers each walk the phase program from ONE loop with a runtime phase
 //     kind: the code is much larger than the instruction cache, and straight-line code that runs
 //     once per step is fetched from L2 (measured: 3-10x slower than the same code in a loop).
+//   * Tensor memory as a second staging level (large shapes with at most four activation rows): the ring of
+//     shared-memory stages holds 4 us of the stream, a phase end (epilogue, grid barrier, the wait for the slowest
+//     CTA, staging of the next input vector) lasts 5-7 us, so HBM idled at every phase end. A mover thread copies
+//     the first eight stages of every phase, as they land, into the eight slots of the SM's 256 KB tensor memory
+//     (tcgen05.cp, 32 KB per stage; measured 0.47 us per stage, faster than the 0.67 us at which stages arrive but
+//     slower than the consumers, hence only the head of a phase) and frees their shared-memory stages at once; the
+//     consumers read those stages' MMA fragments from tensor memory (tcgen05.ld), the rest from shared memory.
+//     The producers then run up to 14 stages (9 us) ahead of the consumers.
 //   * The output head gathers rows W[ids[j]] (Eq. 3 of the paper), keeps a running (value, id)
 //     maximum per activation row and publishes it with one 64-bit atomicMax per CTA; logits are
 //     never written unless a debug buffer is passed.
 #include "mega.cuh"
 #include "ptx.cuh"
+#include "umma.cuh"
 
 #include <cooperative_groups.h>
 
@@ -50,6 +59,11 @@ struct Prog { int step, layer, kind; };
 struct Misc {   // small shared-memory block
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
+    uint64_t tfull[kTmSlots];     // tensor-memory slots: filled by the mover's copies / read out by the four owning warps
+    uint64_t tempty[kTmSlots];
+    uint64_t tdrain;              // the mover's last copies, before the tensor memory is freed
+    uint32_t tmem_base;
+    uint32_t use_done[kMaxStages];   // per ring slot: uses whose data has been taken out (read by consumers or moved)
     float scale0[kMaxRows];
     float scale1[kMaxRows];
     float ssred[kConsumerWarps][kMaxRows][2];
@@ -57,6 +71,8 @@ struct Misc {   // small shared-memory block
     unsigned long long keyred[kConsumerWarps][kMaxRows];
     int tok[kMaxRows];
     int outrow[kMaxRows];   // where the head publishes activation row r (out_row), set when the head's input is staged
+    int seqlen[kMaxRows];   // committed length of every sequence and its number of extend rows, read once at kernel start:
+    int next[kMaxRows];     // neither changes during a launch, and every phase that needs them saves an L2 round trip
     unsigned long long rowptr[kProducerWarps][32];   // tile row pointers, one line per producer warp
     int flag;
     uint32_t aborted;
@@ -97,12 +113,18 @@ struct Cta {
     int R, M;              // activation rows and rows per sequence of the current step (see set_step_rows)
     int slot;              // ring slot of the next stage (same sequence in producer and consumers)
     uint32_t parity;       // mbarrier phase parity of that slot
+    int tslot;             // tensor-memory slot of the next matrix stage (same sequence in mover and consumers)
+    uint32_t tparity;
+    uint32_t tmem;         // base address of the CTA's tensor memory
     uint32_t bar_target;   // grid barrier generation
     int redbuf;
 };
 
 __device__ __forceinline__ void next_stage(Cta &c) {
     if (++c.slot == c.p->n_stages) { c.slot = 0; c.parity ^= 1u; }
+}
+__device__ __forceinline__ void next_tslot(Cta &c) {
+    if (++c.tslot == kTmSlots) { c.tslot = 0; c.tparity ^= 1u; }
 }
 __device__ __forceinline__ void raise(const Cta &c, uint32_t bits) { atomicOr(c.p->s.status, bits); }
 
@@ -134,6 +156,27 @@ __device__ __forceinline__ bool wait_bar_impl(Misc *misc, uint64_t *bar, uint32_
 __device__ __forceinline__ bool wait_bar(const Cta &c, uint64_t *bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;          // fast path: already complete
     return wait_bar_impl(c.misc, bar, parity, c.p->s.abort_flag, c.p->s.status, c.p->wait_limit_ns);
+}
+// The same wait for a thread that is in no hurry (the mover of the tensor-memory path): it sleeps between polls, so
+// that its spinning does not take issue slots and load/store bandwidth from the producer and consumer warps that
+// share its scheduler.
+__device__ __forceinline__ bool wait_bar_idle(const Cta &c, uint64_t *bar, uint32_t parity) {
+    if (aborted(c)) return false;
+    unsigned long long t0 = 0;
+    for (uint32_t n = 0;; ++n) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(64);
+        if ((n & 63u) == 63u) {
+            if (ldcg_u32(c.p->s.abort_flag) != 0) { c.misc->aborted = 1; return false; }
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > c.p->wait_limit_ns) break;
+        }
+    }
+    c.misc->aborted = 1;
+    atomicOr(c.p->s.status, kDevTimeout);
+    atomicExch(c.p->s.abort_flag, 1u);
+    return false;
 }
 __device__ __forceinline__ void do_abort(const Cta &c) {
     c.misc->aborted = 1;
@@ -198,21 +241,19 @@ __device__ __forceinline__ void set_step_rows(Cta &c, int step) {
     c.M = (c.p->mode == 0 && step > 0) ? 1 : c.p->M;
     c.R = c.p->B * c.M;
 }
-__device__ __forceinline__ int seq_next(const MegaParams &p, int b) {
-    return p.n_ext ? min(max(p.n_ext[b], 1), p.M) : p.M;
-}
-__device__ __forceinline__ int step_rows(const MegaParams &p, int b, int step) {      // rows of sequence b that count
-    return p.mode == 1 ? p.M : (step == 0 ? seq_next(p, b) : 1);
+__device__ __forceinline__ int seq_next(const Cta &c, int b) { return c.misc->next[b]; }
+__device__ __forceinline__ int step_rows(const Cta &c, int b, int step) {      // rows of sequence b that count
+    return c.p->mode == 1 ? c.p->M : (step == 0 ? seq_next(c, b) : 1);
 }
 // Row of the previous step whose output row r of this draft step continues (step >= 1).
-__device__ __forceinline__ int src_row(const MegaParams &p, int r, int step) {
-    return step == 1 ? r * p.M + seq_next(p, r) - 1 : r;
+__device__ __forceinline__ int src_row(const Cta &c, int r, int step) {
+    return step == 1 ? r * c.p->M + seq_next(c, r) - 1 : r;
 }
 // Output index (sequence in a draft, row in a target step) of activation row r, -1 if it publishes nothing.
-__device__ __forceinline__ int out_row(const MegaParams &p, int r, int step) {
-    if (p.mode == 1 || step > 0) return r;
-    const int b = r / p.M;
-    return (r - b * p.M == seq_next(p, b) - 1) ? b : -1;
+__device__ __forceinline__ int out_row(const Cta &c, int r, int step) {
+    if (c.p->mode == 1 || step > 0) return r;
+    const int b = r / c.p->M;
+    return (r - b * c.p->M == seq_next(c, b) - 1) ? b : -1;
 }
 
 // ---- phase geometry ----------------------------------------------------------------------
@@ -306,6 +347,14 @@ __device__ __forceinline__ void tile_ptrs(Cta &c, int kind, const LayerPtrs &L, 
     for (int i = 0; i < kRowsPerProducer; ++i) out[i] = reinterpret_cast<const unsigned char *>(tbl[pw + i * kProducerWarps]);
 }
 
+// Stage layout with tensor-memory staging (TM): the stage is the image of its tensor-memory slot, 128 lane rows x
+// 256 bytes, stored as two 16 KB tiles of 128-byte rows with the 128-byte swizzle the tcgen05 descriptors describe
+// (16-byte piece c of lane row L at c ^ (L & 7)). Lane row 32*wi + 4*g + t belongs to thread (g, t) of the consumer
+// warps wi and wi + 4 and holds, in fragment order, the sixteen 16-byte pieces that thread multiplies: piece
+// 4*j + rb = weight row g + 8*rb, k elements [32*ch + 8*t, +8) with ch = 8*(j >> 1) + 2*wi + (j & 1). A producer
+// instruction still copies 512 contiguous bytes of one weight row; the eight lanes of a quarter-warp land in eight
+// different 16-byte bank groups.
+template <bool TM>
 __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs &L) {
     const MegaParams &p = *c.p;
     const Geom g = geom(c, kind);
@@ -313,6 +362,16 @@ __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs 
     const unsigned char *cur[kRowsPerProducer], *nxt[kRowsPerProducer];
 #pragma unroll
     for (int i = 0; i < kRowsPerProducer; ++i) nxt[i] = nullptr;
+    uint32_t toff[kRowsPerProducer];
+    if (TM) {
+        const int t = c.lane & 3, jlow = (c.lane >> 2) & 1, wq = c.lane >> 3;
+#pragma unroll
+        for (int i = 0; i < kRowsPerProducer; ++i) {
+            const int gr = pw + 4 * (i & 1), rb = i >> 1;            // tile row pw + 4*i = gr + 8*rb
+            const int lrow = 32 * wq + 4 * gr + t;
+            toff[i] = (uint32_t)(lrow * 128 + ((4 * (jlow ^ (pw & 1)) + (rb ^ t)) << 4));
+        }
+    }
     // rows are stored without padding; in odd rows the two 64-byte halves of every 128 bytes are
     // swapped, which keeps the consumers' 128-bit fragment loads free of bank conflicts. All rows of a
     // producer warp have the parity of pw.
@@ -344,7 +403,25 @@ __device__ __forceinline__ void produce_phase(Cta &c, int kind, const LayerPtrs 
             const int klen = sk.klen;
             const uint32_t dst0 = smem_u32(c.ring + (size_t)slot * p.stage_bytes) + (uint32_t)pw * rs + lane16d;
             const size_t koff = (size_t)sk.koff * 2 + lane16;
-            if (klen == 512) {
+            if (TM) {
+                // every stage is 512 wide here: the second piece of a row (k elements 256..511) belongs to the second
+                // 16 KB tile of the stage
+                const uint32_t sbase = smem_u32(c.ring + (size_t)slot * p.stage_bytes);
+                uint32_t d[kRowsPerProducer];
+                const unsigned char *q[kRowsPerProducer];
+#pragma unroll
+                for (int i = 0; i < kRowsPerProducer; ++i) {
+                    q[i] = cur[i] + koff;
+                    d[i] = sbase + toff[i];
+                }
+#pragma unroll
+                for (int i = 0; i < kRowsPerProducer; ++i) {
+                    if (cur[i] != nullptr) {
+                        asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(d[i]), "l"(q[i]), "l"(pol) : "memory");
+                        asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0+16384], [%1+512], 16, %2;" ::"r"(d[i]), "l"(q[i]), "l"(pol) : "memory");
+                    }
+                }
+            } else if (klen == 512) {
                 // the stage width of the large shapes, from fully unrolled code: two 512-byte pieces per row, one
                 // instruction per piece and lane, all with their own address registers (the piece offsets are
                 // immediates). The loop is this tight on purpose: a predicate or branch per instruction costs
@@ -550,7 +627,12 @@ __device__ __forceinline__ void park(float (&acc)[2][2][4], float (&acd)[2][2][4
 // added at the end); rows 4..7 use a second set of accumulators. The two halves of the consumer
 // warps (warps 0-3 / 4-7) take alternate stages, so each warp does four chunks per barrier wait
 // and two stages are in work at once.
-template <bool two_sets>
+//
+// With tensor-memory staging (TM) the stage has the layout of a tensor-memory slot (see the producer): the thread's
+// sixteen 16-byte pieces, already in fragment order, come by two tcgen05.ld of 32 registers each (the first eight
+// stages of a phase) or by sixteen conflict-free 128-bit loads from the shared-memory stage (the rest), and the
+// warp's four k chunks of a stage are 8*(j >> 1) + 2*wi + (j & 1), j = 0..3.
+template <bool two_sets, bool TM>
 __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActSrc &act, EpiCtx &ex) {
     const MegaParams &p = *c.p;
     const Geom geo = geom(c, kind);
@@ -583,6 +665,9 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
         // straight into the fragment registers were four load instructions per stage and warp, a third on top of the
         // producers' copies in the same load/store path, and held this phase a quarter below the others' stream rate.
         constexpr int kCpw = 4;                                       // chunks a warp has in a full stage: wi, wi + 4, wi + 8, wi + 12
+        uint32_t xo[8];                                               // TM: where this lane's piece s of a 16 KB tile sits in its row
+#pragma unroll
+        for (int s8 = 0; s8 < 8; ++s8) xo[s8] = (uint32_t)(32 * wi + c.lane) * 128u + (((uint32_t)s8 ^ ((uint32_t)c.lane & 7u)) << 4);
         const bool gfast = !two_sets && !act.in_smem && 16 * R * 512 <= p.scratch_smem;      // the slice ring must fit the staging area
         // which half of the warps takes a stage depends only on the stage's index within the phase,
         // never on how many stages the CTA has seen before: the summation order of a row must not
@@ -593,7 +678,8 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
         auto slice_slot = [&](int sa) -> uint32_t { return slice_base + (uint32_t)((sa & 3) * 4 * R) * 512u; };
         auto slice_fetch = [&](int sa, const StageK &sk) {           // lane = (chunk j, hi/lo, 16-byte piece)
             const int j = c.lane >> 3, hl = (c.lane >> 2) & 1, tp = c.lane & 3;
-            const bf16_t *src = (hl ? act.lo : act.hi) + (size_t)sk.koff + (wi + 4 * j) * 32 + tp * 8;
+            const int ch = TM ? 8 * (j >> 1) + 2 * wi + (j & 1) : wi + 4 * j;
+            const bf16_t *src = (hl ? act.lo : act.hi) + (size_t)sk.koff + ch * 32 + tp * 8;
             const uint32_t dst = slice_slot(sa) + (uint32_t)c.lane * 16u;
 #pragma unroll 1
             for (int r = 0; r < R; ++r)
@@ -614,7 +700,86 @@ __device__ __forceinline__ void consume_tiles(Cta &c, const int kind, const ActS
                 // the warp owned)
                 park<two_sets>(acc, acd, acc0, acd0);
             }
-            if (((stage0 + ks) & 1) == grp) {
+            if (TM) {
+                // the first kTmSlots stages of a phase come through tensor memory (they land while the consumers are still
+                // busy with the previous phase's end), the rest is read from the shared-memory stage directly
+                const bool via_tmem = stage0 + ks < kTmSlots;
+                if (((stage0 + ks) & 1) == grp) {
+                    const StageK sk = stage_k(geo, ks);
+                    uint32_t w0[32], w1[32];
+                    const int ts = c.tslot, slot = c.slot;
+                    PROF_T0();
+                    if (via_tmem) {
+                        wait_bar(c, &c.misc->tfull[ts], c.tparity);
+                        PROF_ACC(c, 0, c.tid == 0);
+                        tc_fence_after_sync();
+                        const uint32_t ta = c.tmem + ((uint32_t)(32 * wi) << 16) + (uint32_t)(ts * kTmSlotCols);
+                        tmem_ld32_issue(ta, w0);
+                        tmem_ld32_issue(ta + 32, w1);
+                    } else {
+                        wait_bar(c, &c.misc->full[slot], c.parity);
+                        PROF_ACC(c, 0, c.tid == 0);
+                    }
+                    uint4 bq[kCpw];
+                    if (act.in_smem) {
+                        const uint32_t ab = smem_u32(abase + aoff0 + (size_t)sk.koff);
+#pragma unroll
+                        for (int j = 0; j < kCpw; ++j) bq[j] = has0 ? lds128_u32(ab + (8 * (j >> 1) + 2 * wi + (j & 1)) * 64) : zero;
+                    } else {
+                        if (ks + 2 < geo.nks) slice_fetch(stage0 + ks + 2, stage_k(geo, ks + 2));
+                        if (ks + 2 < geo.nks) asm volatile("cp.async.wait_group 1;" ::: "memory");
+                        else asm volatile("cp.async.wait_group 0;" ::: "memory");
+                        __syncwarp();
+                        const uint32_t sl = slice_slot(stage0 + ks) + (uint32_t)(arow * 512 + ((g & 1) * 4 + t) * 16);
+#pragma unroll
+                        for (int j = 0; j < kCpw; ++j) bq[j] = has0 ? lds128_u32(sl + j * 128) : zero;
+                    }
+                    if (via_tmem) {
+                        tmem_ld_wait();
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (c.lane == 0) mbar_arrive(&c.misc->tempty[ts]);       // the slot's data is in registers
+                    } else {
+                        // the stage has the slot's layout: lane row 32*wi + lane, piece s of it at (s & 7) ^ (lane & 7) in tile s >> 3
+                        const uint32_t lb = smem_u32(c.ring + (size_t)slot * p.stage_bytes);
+#pragma unroll
+                        for (int s8 = 0; s8 < 8; ++s8) {
+                            const uint4 a = lds128_u32(lb + xo[s8]);
+                            const uint4 b = lds128_u32(lb + xo[s8] + 16384u);
+                            w0[4 * s8] = a.x; w0[4 * s8 + 1] = a.y; w0[4 * s8 + 2] = a.z; w0[4 * s8 + 3] = a.w;
+                            w1[4 * s8] = b.x; w1[4 * s8 + 1] = b.y; w1[4 * s8 + 2] = b.z; w1[4 * s8 + 3] = b.w;
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        Frag f;
+                        f.u0 = make_uint4(w0[16 * j + 0], w0[16 * j + 1], w0[16 * j + 2], w0[16 * j + 3]);
+                        f.v0 = make_uint4(w0[16 * j + 4], w0[16 * j + 5], w0[16 * j + 6], w0[16 * j + 7]);
+                        f.u1 = make_uint4(w0[16 * j + 8], w0[16 * j + 9], w0[16 * j + 10], w0[16 * j + 11]);
+                        f.v1 = make_uint4(w0[16 * j + 12], w0[16 * j + 13], w0[16 * j + 14], w0[16 * j + 15]);
+                        mma_chunk(acc, f, bq[j]);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        Frag f;
+                        f.u0 = make_uint4(w1[16 * j + 0], w1[16 * j + 1], w1[16 * j + 2], w1[16 * j + 3]);
+                        f.v0 = make_uint4(w1[16 * j + 4], w1[16 * j + 5], w1[16 * j + 6], w1[16 * j + 7]);
+                        f.u1 = make_uint4(w1[16 * j + 8], w1[16 * j + 9], w1[16 * j + 10], w1[16 * j + 11]);
+                        f.v1 = make_uint4(w1[16 * j + 12], w1[16 * j + 13], w1[16 * j + 14], w1[16 * j + 15]);
+                        mma_chunk(acc, f, bq[2 + j]);
+                    }
+                    if (!via_tmem) {
+                        __syncwarp();
+                        if (c.lane == 0) {
+                            // counted before the arrival, so that the count of a use is never written after the slot's next use
+                            if (wi == 0) { volatile uint32_t *ud = &c.misc->use_done[slot]; *ud = *ud + 1; }   // see the mover
+                            mbar_arrive(&c.misc->empty[slot]);
+                        }
+                    }
+                    PROF_ACC(c, 1, c.tid == 0);
+                }
+                if (via_tmem) next_tslot(c);
+            } else if (((stage0 + ks) & 1) == grp) {
                 const int slot = c.slot;
                 const uint32_t parity = c.parity;
                 PROF_T0();
@@ -753,7 +918,7 @@ __device__ __forceinline__ void stage_hilo(const Cta &c, const bf16_t *ghi, cons
         for (int q = 0; q < 4; ++q) {
             int i = min(i0 + q * kConsumerThreads, total - 1);
             int r = i / per_row, k = (i - r * per_row) * 8;
-            const int rs = remap_step > 0 ? src_row(*c.p, r, remap_step) : r;
+            const int rs = remap_step > 0 ? src_row(c, r, remap_step) : r;
             a[q] = ldcg128(ghi + (size_t)rs * gstride + k);
             b[q] = ldcg128(glo + (size_t)rs * gstride + k);
         }
@@ -943,34 +1108,35 @@ struct AttnItem { int b, kvh, chunk, Lb, nch, base, rows; };
 // rows can see: every index the attention and merge phases form from seq_lens stays inside the block
 // table and the partial buffer, whatever the caller put there.
 __device__ __forceinline__ int kv_max_tokens(const MegaParams &p, const KvPtrs &kv) { return min(kv.max_pages * p.page, p.max_ctx); }
-__device__ __forceinline__ int committed_len(const MegaParams &p, const KvPtrs &kv, int b) {
-    return min(max(kv.seq_lens[b], 0), kv_max_tokens(p, kv));
+__device__ __forceinline__ int committed_len(const Cta &c, const KvPtrs &kv, int b) {
+    return min(max(c.misc->seqlen[b], 0), kv_max_tokens(*c.p, kv));
 }
-__device__ __forceinline__ int step_base(const MegaParams &p, const KvPtrs &kv, int b, int step) {
-    return committed_len(p, kv, b) + ((p.mode == 0 && step > 0) ? seq_next(p, b) - 1 + step : 0);
+__device__ __forceinline__ int step_base(const Cta &c, const KvPtrs &kv, int b, int step) {
+    return committed_len(c, kv, b) + ((c.p->mode == 0 && step > 0) ? seq_next(c, b) - 1 + step : 0);
 }
-__device__ __forceinline__ int visible_chunks(const MegaParams &p, const KvPtrs &kv, int b, int step) {
-    const int last = min(step_base(p, kv, b, step) + step_rows(p, b, step) - 1, kv_max_tokens(p, kv) - 1);
-    return min(last / kAttnChunk + 1, p.max_chunks);
+__device__ __forceinline__ int visible_chunks(const Cta &c, const KvPtrs &kv, int b, int step) {
+    const int last = min(step_base(c, kv, b, step) + step_rows(c, b, step) - 1, kv_max_tokens(*c.p, kv) - 1);
+    return min(last / kAttnChunk + 1, c.p->max_chunks);
 }
 
-__device__ __forceinline__ int attn_total(const MegaParams &p, const KvPtrs &kv, int step) {
+__device__ __forceinline__ int attn_total(const Cta &c, const KvPtrs &kv, int step) {
     int total = 0;
-    for (int b = 0; b < p.B; ++b) total += p.Hkv * visible_chunks(p, kv, b, step);
+    for (int b = 0; b < c.p->B; ++b) total += c.p->Hkv * visible_chunks(c, kv, b, step);
     return total;
 }
-__device__ __forceinline__ AttnItem attn_item(const MegaParams &p, const KvPtrs &kv, int step, int item) {
+__device__ __forceinline__ AttnItem attn_item(const Cta &c, const KvPtrs &kv, int step, int item) {
+    const MegaParams &p = *c.p;
     AttnItem it;
     int b = 0, rem = item, nch = 1;
     for (; b < p.B; ++b) {
-        nch = visible_chunks(p, kv, b, step);
+        nch = visible_chunks(c, kv, b, step);
         if (rem < p.Hkv * nch) break;
         rem -= p.Hkv * nch;
     }
     if (b >= p.B) b = p.B - 1;
-    it.b = b; it.Lb = committed_len(p, kv, b); it.nch = nch;
-    it.base = step_base(p, kv, b, step);
-    it.rows = step_rows(p, b, step);
+    it.b = b; it.Lb = committed_len(c, kv, b); it.nch = nch;
+    it.base = step_base(c, kv, b, step);
+    it.rows = step_rows(c, b, step);
     it.kvh = rem / nch;
     it.chunk = rem - it.kvh * nch;
     return it;
@@ -980,9 +1146,9 @@ __device__ __forceinline__ void produce_attention(Cta &c, const KvPtrs &kv, int 
     const MegaParams &p = *c.p;
     const int ptid = c.tid - kConsumerThreads;               // 0 .. 127
     const int upt = p.dh >> 3;                                // 16-byte units per token row
-    const int total = attn_total(p, kv, step);
+    const int total = attn_total(c, kv, step);
     for (int item = c.cta; item < total; item += c.grid) {
-        const AttnItem it = attn_item(p, kv, step, item);
+        const AttnItem it = attn_item(c, kv, step, item);
         const int c0 = it.chunk * kAttnChunk;
         const int n_old = max(0, min(kAttnChunk, it.Lb - c0));   // committed tokens of this chunk
         const int32_t *bt = kv.block_table + (size_t)it.b * kv.max_pages;
@@ -1033,9 +1199,9 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int st
     const int max_tokens = min(kv.max_pages * p.page, p.max_ctx);   // positions beyond are flagged, not touched
     const int upt = dh >> 3;
 
-    const int total = attn_total(p, kv, step);
+    const int total = attn_total(c, kv, step);
     for (int item = c.cta; item < total; item += c.grid) {
-        const AttnItem it = attn_item(p, kv, step, item);
+        const AttnItem it = attn_item(c, kv, step, item);
         const int b = it.b, kvh = it.kvh, chunk = it.chunk, Lb = it.Lb;
         const int base = it.base;                  // position of row m = 0
         const int rows = it.rows;                  // rows of this sequence that count (the rest is padding)
@@ -1114,6 +1280,7 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int st
 
         attn_rows<DH>(c, sk, sv, qs, b, kvh, chunk, base, max_tokens, rows);
         // the stage is free again (all consumer warps passed the barrier at the end of attn_rows)
+        if (c.tid == 0) { volatile uint32_t *ud = &c.misc->use_done[slot]; *ud = *ud + 1; }   // see the mover of the tensor-memory path
         if (c.warp < kConsumerWarps / 2 && c.lane == 0) mbar_arrive(&c.misc->empty[slot]);
         next_stage(c);
         bar_sync(1, kConsumerThreads);   // the query / partial scratch is reused by the next item
@@ -1141,7 +1308,7 @@ __device__ __forceinline__ void merge_phase(Cta &c, const KvPtrs &kv, int step) 
         const int r = u / (p.Hq * 4), rem = u - r * (p.Hq * 4);
         const int hq = rem >> 2, e = (rem & 3) * qe + el;
         const int b = r / M, m = r - b * M;
-        const int pos = min(step_base(p, kv, b, step) + min(m, step_rows(p, b, step) - 1), max_tokens - 1);
+        const int pos = min(step_base(c, kv, b, step) + min(m, step_rows(c, b, step) - 1), max_tokens - 1);
         const int ncm = min(pos / kAttnChunk + 1, p.max_chunks);        // chunks visible to this row
         const float *src = p.s.att_part + ((size_t)r * p.Hq + hq) * p.max_chunks * wstride;
         for (int i = c.tid; i < ncm; i += kConsumerThreads) {
@@ -1174,8 +1341,9 @@ __device__ __forceinline__ void merge_phase(Cta &c, const KvPtrs &kv, int step) 
 // ---- the kernel --------------------------------------------------------------------------------
 // One instantiation per (more than four activation rows?, head dimension): each contains only the
 // code it runs, which keeps it near the size of the instruction cache.
-template <bool TWO, int DH>
-__global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant__ MegaParams p) {
+template <bool TWO, int DH, bool TM>
+__global__ void __launch_bounds__(TM ? kTmThreads : kThreads, 1) mega_kernel(const __grid_constant__ MegaParams p) {
+    static_assert(!(TM && TWO), "tensor-memory staging serves at most four activation rows");
     extern __shared__ __align__(128) unsigned char smem[];
     Cta c;
     c.p = &p;
@@ -1185,6 +1353,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
     off += ((size_t)2 * kConsumerWarps * kTileRows * p.R * sizeof(float) + 127) & ~size_t(127);
     c.scr = smem + off;
     off += (size_t)p.scratch_smem;
+    if (TM) off = (size_t)(((smem_u32(smem) + (uint32_t)off + 1023u) & ~1023u) - smem_u32(smem));   // swizzled tiles: 1024-byte aligned
     c.ring = smem + off;
     c.cta = blockIdx.x;
     c.grid = gridDim.x;
@@ -1193,6 +1362,9 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
     c.lane = threadIdx.x & 31;
     c.slot = 0;
     c.parity = 0;
+    c.tslot = 0;
+    c.tparity = 0;
+    c.tmem = 0;
     c.bar_target = 0;
     c.redbuf = 0;
 #ifdef FMTP_PROF
@@ -1203,15 +1375,39 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
     if (c.tid == 0) {
         for (int i = 0; i < p.n_stages; ++i) {
             mbar_init(&c.misc->full[i], kProducerWarps * 32);
-            mbar_init(&c.misc->empty[i], kConsumerWarps / 2);   // the four warps that own the stage
+            mbar_init(&c.misc->empty[i], kConsumerWarps / 2);   // the four warps that own the stage (or the mover in their place)
         }
+        if (TM) {
+            for (int i = 0; i < kTmSlots; ++i) {
+                mbar_init(&c.misc->tfull[i], 1);
+                mbar_init(&c.misc->tempty[i], kConsumerWarps / 2);
+            }
+            mbar_init(&c.misc->tdrain, 1);
+        }
+        for (int i = 0; i < kMaxStages; ++i) c.misc->use_done[i] = 0;
         c.misc->aborted = 0;
         mbar_fence_init();
     }
+    if (c.tid < p.B) {
+        c.misc->seqlen[c.tid] = p.kvs[0].seq_lens[c.tid];
+        c.misc->next[c.tid] = (p.mode == 0 && p.n_ext) ? min(max(p.n_ext[c.tid], 1), p.M) : p.M;
+    }
     // the ring starts zeroed so that never-written tails multiply as finite numbers
-    for (size_t i = (size_t)c.tid * 16; i < (size_t)p.n_stages * p.stage_bytes; i += (size_t)kThreads * 16)
+    for (size_t i = (size_t)c.tid * 16; i < (size_t)p.n_stages * p.stage_bytes; i += (size_t)blockDim.x * 16)
         *reinterpret_cast<uint4 *>(c.ring + i) = make_uint4(0, 0, 0, 0);
+    constexpr int kMoverWarp = kConsumerWarps + kProducerWarps;
+    if (TM) {
+        if (c.warp == kMoverWarp) {          // the whole tensor memory of the SM (this kernel has the SM to itself)
+            tmem_alloc(&c.misc->tmem_base, 512);
+            tmem_relinquish();
+        }
+        tc_fence_before_sync();
+    }
     __syncthreads();
+    if (TM) {
+        tc_fence_after_sync();
+        c.tmem = c.misc->tmem_base;
+    }
 
 #ifdef FMTP_PROF
     const long long prof_c0 = clock64();
@@ -1221,6 +1417,83 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
     const int n_steps = (p.mode == 0) ? p.K : 1;
     set_step_rows(c, 0);
 
+    if (TM && c.warp >= kMoverWarp) {
+        // ---------------- fourth warpgroup: one thread moves landed weight stages into tensor memory, in program
+        // order; the other warps only give their registers back
+        setmaxnreg_dec<kTmMoverRegs>();
+        if (c.warp == kMoverWarp) {
+            if (c.lane == 0) {
+                bool ok = true;
+                uint32_t wraps = 0;            // times the ring position has wrapped = earlier uses of the current slot
+                Prog g;
+#pragma unroll 1
+                for (prog_begin(p, g); g.kind != DONE && ok; prog_next(p, g)) {
+                    set_step_rows(c, g.step);
+                    if (g.kind == EMBED || g.kind == MERGE) continue;
+                    if (g.kind == ATTN) {      // K/V stages stay in shared memory: skip this CTA's items
+                        const int total = attn_total(c, p.kvs[g.layer], g.step);
+                        for (int item = c.cta; item < total; item += c.grid) { if (c.slot + 1 == p.n_stages) ++wraps; next_stage(c); }
+                        continue;
+                    }
+                    const Geom geo = geom(c, g.kind);
+                    const int tiles = (geo.v1 - geo.v0 + geo.cap - 1) / geo.cap;
+                    const int total = tiles * geo.nks;
+#pragma unroll 1
+                    for (int n = 0; n < total && ok; ++n) {
+                        if (n < kTmSlots) {           // the head of the phase goes through tensor memory
+                            const int slot = c.slot, ts = c.tslot;
+                            // A wait names a barrier phase by its parity only, so it must not be asked more than one phase
+                            // ahead of the barrier; this thread skips the stages the consumers read themselves, possibly
+                            // many uses of a slot. It therefore first waits until every earlier use of the slot has been
+                            // taken out (counted by whoever took it), which puts the slot's barrier in this use's phase.
+                            {
+                                volatile uint32_t *ud = &c.misc->use_done[slot];
+                                unsigned long long t0 = 0;
+                                for (uint32_t it = 0; *ud < wraps; ++it) {
+                                    __nanosleep(128);
+                                    if ((it & 63u) == 63u) {
+                                        if (ldcg_u32(p.s.abort_flag) != 0) { c.misc->aborted = 1; ok = false; break; }
+                                        const unsigned long long now = global_timer_ns();
+                                        if (t0 == 0) t0 = now;
+                                        else if (now - t0 > p.wait_limit_ns) { do_abort(c); ok = false; break; }
+                                    }
+                                }
+                                __threadfence_block();
+                            }
+                            ok = ok && wait_bar_idle(c, &c.misc->full[slot], c.parity) && wait_bar_idle(c, &c.misc->tempty[ts], c.tparity ^ 1u);
+                            if (!ok) break;
+                            fence_proxy_async();          // the copies' shared-memory writes, before the tensor core reads them
+                            tc_fence_after_sync();
+                            const uint32_t sa = smem_u32(c.ring + (size_t)slot * p.stage_bytes);
+                            const uint32_t ta = c.tmem + (uint32_t)(ts * kTmSlotCols);
+#pragma unroll
+                            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                                for (int q = 0; q < 4; ++q)
+                                    tmem_cp_128x256b(ta + (uint32_t)(h * 32 + q * 8), umma_smem_desc(sa + (uint32_t)(h * 16384 + q * 32)));
+                            // the stage may be overwritten once the copies have read it: the arrivals of the four warps that
+                            // would have read it
+#pragma unroll
+                            for (int q = 0; q < kConsumerWarps / 2; ++q) umma_commit(&c.misc->empty[slot]);
+                            umma_commit(&c.misc->tfull[ts]);
+                            c.misc->use_done[slot] = wraps + 1;
+                            next_tslot(c);
+                        }
+                        if (c.slot + 1 == p.n_stages) ++wraps;
+                        next_stage(c);
+                    }
+                }
+                // every copy issued has completed before the tensor memory is freed
+                umma_commit(&c.misc->tdrain);
+                for (uint32_t n = 0; n < (1u << 22) && !mbar_try_wait(&c.misc->tdrain, 0u); ++n) { }
+            }
+            __syncwarp();
+            bar_sync(2, kConsumerThreads + 32);       // the consumers have read their last slot
+            tc_fence_after_sync();
+            tmem_dealloc(c.tmem, 512);
+        }
+        return;
+    }
     if (is_producer) {
         setmaxnreg_dec<kProducerRegs>();
         // ---------------- producers: the weight / KV stream of every phase, in program order
@@ -1228,7 +1501,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
         for (prog_begin(p, g); g.kind != DONE; prog_next(p, g)) {
             set_step_rows(c, g.step);
             if (g.kind == ATTN) produce_attention(c, p.kvs[g.layer], g.step);
-            else if (g.kind != EMBED && g.kind != MERGE) produce_phase(c, g.kind, p.layers[g.layer]);
+            else if (g.kind != EMBED && g.kind != MERGE) produce_phase<TM>(c, g.kind, p.layers[g.layer]);
         }
         cp_async_wait_all();   // every copy this thread issued has landed before the CTA may exit
         PROF_FLUSH(c, 2, 4, c.warp == kConsumerWarps && c.lane == 0);
@@ -1236,7 +1509,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
     }
 
     // ---------------- consumers: one loop over the phase program; every phase ends in a grid barrier
-    setmaxnreg_inc<kConsumerRegs>();
+    setmaxnreg_inc<TM ? kTmConsumerRegs : kConsumerRegs>();
     bf16_t *s_hi = reinterpret_cast<bf16_t *>(c.scr);
     EpiCtx ex;
     ex.best = 0ull;
@@ -1300,7 +1573,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
             float pvc[kPartialRegs], pvd[kPartialRegs];
             const bool renorm = step > 0 && c.warp < R;
             if (renorm) {
-                const int col = src_row(p, c.warp, step);      // step 1 continues each sequence's last extend row
+                const int col = src_row(c, c.warp, step);      // step 1 continues each sequence's last extend row
                 load_partials(c, p.s.ssC, col, pvc);
                 load_partials(c, p.s.ssD, col, pvd);
             }
@@ -1315,7 +1588,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                 int tok;
                 if (step == 0) {
                     const int b = c.tid / p.M;         // a padding row's token is never looked at
-                    tok = (c.tid - b * p.M < seq_next(p, b)) ? p.tokens[c.tid] : 0;
+                    tok = (c.tid - b * p.M < seq_next(c, b)) ? p.tokens[c.tid] : 0;
                 } else {
                     if ((key >> 32) == 0ull) raise(c, kDevAllNan);
                     tok = (int)argmax_key_id(key);
@@ -1390,7 +1663,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
                 if (c.lane == 0) c.misc->scale0[c.warp] = sc;
             }
         }
-        if (kind == HEAD && c.tid < R) c.misc->outrow[c.tid] = out_row(p, c.tid, step);
+        if (kind == HEAD && c.tid < R) c.misc->outrow[c.tid] = out_row(c, c.tid, step);
         bar_sync(1, kConsumerThreads);
         if (kind == HEAD && p.out_h) {   // every CTA writes its slice of the post-final-norm hidden state
             int r0 = (int)(((long long)c.cta * p.d) / c.grid), r1 = (int)(((long long)(c.cta + 1) * p.d) / c.grid);
@@ -1406,7 +1679,7 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
         PROF(c, kind * 8 + 1);
 
         // ============ ... stream the weights ...
-        consume_tiles<TWO>(c, kind, act, ex);
+        consume_tiles<TWO, TM>(c, kind, act, ex);
 
         // ============ ... and publish what the next phase needs besides the vector
         if (kind == PROJ) flush_sq(c, ex.sq, p.s.ssA, nullptr);
@@ -1433,6 +1706,10 @@ __global__ void __launch_bounds__(kThreads, 1) mega_kernel(const __grid_constant
         grid_barrier(c);
     }
     PROF(c, DONE * 8);
+    if (TM) {                                  // lets the mover's warp free the tensor memory
+        tc_fence_before_sync();
+        bar_arrive(2, kConsumerThreads + 32);
+    }
 
     PROF_FLUSH(c, 0, 2, c.tid == 0);
     PROF_FLUSH(c, 4, 5, c.tid == 0);
@@ -1477,6 +1754,7 @@ size_t mega_smem_bytes(const MegaParams &p) {
     size_t off = (sizeof(Misc) + 127) & ~size_t(127);
     off += ((size_t)2 * kConsumerWarps * kTileRows * p.R * sizeof(float) + 127) & ~size_t(127);
     off += (size_t)p.scratch_smem;
+    if (p.use_tmem) off = ((off + 1023) & ~size_t(1023)) + 1024;      // the ring starts on a 1024-byte boundary, wherever the base lies
     off += (size_t)p.n_stages * p.stage_bytes;
     return off;
 }
@@ -1488,21 +1766,25 @@ size_t mega_fixed_smem(int R) {
 }
 
 namespace {
-const void *kernel_for(int R, int dh) {
-    if (dh == 128) return R > 4 ? (const void *)mega_kernel<true, 128> : (const void *)mega_kernel<false, 128>;
-    return R > 4 ? (const void *)mega_kernel<true, 64> : (const void *)mega_kernel<false, 64>;
+const void *kernel_for(int R, int dh, int tm) {
+    if (tm) return dh == 128 ? (const void *)mega_kernel<false, 128, true> : (const void *)mega_kernel<false, 64, true>;
+    if (dh == 128) return R > 4 ? (const void *)mega_kernel<true, 128, false> : (const void *)mega_kernel<false, 128, false>;
+    return R > 4 ? (const void *)mega_kernel<true, 64, false> : (const void *)mega_kernel<false, 64, false>;
 }
 }  // namespace
 
-int mega_kernel_index(const MegaParams &p) { return (p.dh == 128 ? 2 : 0) + (p.R > 4 ? 1 : 0); }
+int mega_kernel_index(const MegaParams &p) {
+    if (p.use_tmem) return 4 + (p.dh == 128 ? 1 : 0);
+    return (p.dh == 128 ? 2 : 0) + (p.R > 4 ? 1 : 0);
+}
 
 int mega_max_grid(const MegaParams &p, size_t smem_bytes, int *err) {
     int dev = 0, sms = 0, per_sm = 0;
-    const void *fn = kernel_for(p.R, p.dh);
+    const void *fn = kernel_for(p.R, p.dh, p.use_tmem);
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, smem_bytes);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, p.use_tmem ? kTmThreads : kThreads, smem_bytes);
     if (err) *err = (int)e;
     if (e != cudaSuccess) return 0;
     return sms * (per_sm > 0 ? 1 : 0);
@@ -1510,9 +1792,9 @@ int mega_max_grid(const MegaParams &p, size_t smem_bytes, int *err) {
 
 int mega_launch(const MegaParams &p, int grid, cudaStream_t stream) {
     size_t smem = mega_smem_bytes(p);
-    const void *fn = kernel_for(p.R, p.dh);
+    const void *fn = kernel_for(p.R, p.dh, p.use_tmem);
     void *args[] = {const_cast<MegaParams *>(&p)};
-    return (int)cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kThreads), args, smem, stream);
+    return (int)cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(p.use_tmem ? kTmThreads : kThreads), args, smem, stream);
 }
 
 }  // namespace fmtp

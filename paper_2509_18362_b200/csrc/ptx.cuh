@@ -138,6 +138,11 @@ __device__ __forceinline__ void bar_sync(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
+// Arrival without waiting: the threads that call bar_sync on the same barrier wait for these too.
+__device__ __forceinline__ void bar_arrive(int id, int nthreads) {
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
 // Order-preserving map float -> uint32 (larger float => larger key); NaN maps to 0.
 __device__ __forceinline__ uint32_t float_order_key(float v) {
     if (v != v) return 0u;
