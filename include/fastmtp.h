@@ -136,6 +136,10 @@ const char *fmtp_strerror(int status);
 int fmtp_last_cuda_error(const fmtp_ctx *ctx);
 /* Number of kernel launches this context has enqueued so far. */
 long long fmtp_launch_count(const fmtp_ctx *ctx);
+/* Of those, launches of the persistent kernel that staged weights through tensor memory (opt-in: environment
+ * variable FMTP_TMEM=1 when the context is created; used only for shapes whose contraction lengths are all
+ * multiples of 512 and calls of at most four activation rows). */
+long long fmtp_tmem_launch_count(const fmtp_ctx *ctx);
 
 /* Diagnostic (no counterpart in the paper): runs a one-warp kernel that waits, with the library's
  * bounded wait loop and a limit of `limit_ms` milliseconds (1..1000), for an event that never comes.

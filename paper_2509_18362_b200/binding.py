@@ -24,7 +24,7 @@ FMTP_OK = 0
 DEV_BAD_TOKEN, DEV_BAD_PAGE, DEV_BAD_POS, DEV_TIMEOUT, DEV_ALL_NAN = 1, 2, 4, 8, 16
 
 EXPORTS = ["fmtp_create", "fmtp_destroy", "fmtp_workspace_bytes", "fmtp_set_workspace", "fmtp_strerror",
-           "fmtp_last_cuda_error", "fmtp_launch_count", "fmtp_selftest_wait_timeout", "fmtp_selftest_inject_wait_timeout",
+           "fmtp_last_cuda_error", "fmtp_launch_count", "fmtp_tmem_launch_count", "fmtp_selftest_wait_timeout", "fmtp_selftest_inject_wait_timeout",
            "fastmtp_draft", "fastmtp_draft_host",
            "fastmtp_verify_accept", "fastmtp_verify_accept_host", "fastmtp_verify_accept_static", "fastmtp_accept_ids",
            "fastmtp_target_step"]
@@ -71,6 +71,8 @@ lib.fmtp_last_cuda_error.argtypes = [_p]
 lib.fmtp_last_cuda_error.restype = C.c_int
 lib.fmtp_launch_count.argtypes = [_p]
 lib.fmtp_launch_count.restype = C.c_longlong
+lib.fmtp_tmem_launch_count.argtypes = [_p]
+lib.fmtp_tmem_launch_count.restype = C.c_longlong
 lib.fmtp_selftest_wait_timeout.argtypes = [_p, C.c_int, _p, _p]
 lib.fmtp_selftest_wait_timeout.restype = C.c_int
 lib.fmtp_selftest_inject_wait_timeout.argtypes = [_p, C.c_int, C.c_int]
@@ -196,6 +198,10 @@ class Context:
     @property
     def launch_count(self) -> int:
         return int(lib.fmtp_launch_count(self.handle))
+
+    @property
+    def tmem_launch_count(self) -> int:
+        return int(lib.fmtp_tmem_launch_count(self.handle))
 
     # -- entry points (same names and argument order as the C ABI)
     def fastmtp_draft(self, w: fmtp_mtp_w, h_last, tok_last, mtp_kv: fmtp_kv, B, K, vocab_subset, out_drafts,

@@ -41,6 +41,7 @@ struct fmtp_ctx {
     BatchedShape bsh;
     BatchedWs bws;
     int batched_min;           // calls with at least this many sequences take the batched path (env FMTP_BATCHED_MIN)
+    long long tmem_launches;
     int tmem_staging;          // the persistent kernel stages weights through tensor memory where the shape allows (env FMTP_TMEM=1)
     // answers that depend on the geometry only, kept so that the hot calls make no CUDA attribute / occupancy query:
     struct { size_t smem; int grid; } mega_cfg[6];                 // per kernel instantiation: footprint its limit was raised to
@@ -215,6 +216,7 @@ int launch_mega(fmtp_ctx *c, MegaParams &p, cudaStream_t st) {
     err = mega_launch(p, cfg.grid, st);
     if (err) return cuda_fail(c, (cudaError_t)err);
     c->launches++;
+    if (p.use_tmem) c->tmem_launches++;
     return FMTP_OK;
 }
 
@@ -337,6 +339,7 @@ int fmtp_destroy(fmtp_ctx *c) {
 size_t fmtp_workspace_bytes(const fmtp_ctx *c) { return c ? c->ws_need : 0; }
 int fmtp_last_cuda_error(const fmtp_ctx *c) { return c ? c->last_cuda : 0; }
 long long fmtp_launch_count(const fmtp_ctx *c) { return c ? c->launches : 0; }
+long long fmtp_tmem_launch_count(const fmtp_ctx *c) { return c ? c->tmem_launches : 0; }
 
 int fmtp_set_workspace(fmtp_ctx *c, void *dev, size_t bytes) {
     if (!c || !dev) return FMTP_EINVAL;

@@ -50,6 +50,7 @@ def run_draft_case(shape, seed, B, L, K, N, subset="uniform", want_logits=True, 
         "k_pages": Bd.bf16_bits(dkv["k_pages"]),
         "v_pages": Bd.bf16_bits(dkv["v_pages"]),
         "launches": ctx.launch_count,
+        "tmem_launches": ctx.tmem_launch_count,
     }
     ctx.close()
 
@@ -79,6 +80,29 @@ def test_tiny_config_batch1():
     for k in range(3):
         lg = O.head_logits(ref["h_out"][0, k], ref["W"]["lm_head"], ref["ids"])
         close(got["logits"][0, k], lg, f"tiny logits step {k}")
+
+
+@pytest.mark.parametrize("B,L,K,N", [
+    (1, [70], 3, 1500),           # ragged last head tile
+    (2, [5, 130], 2, None),       # full vocabulary, context crossing an attention chunk
+    (4, [0, 63, 64, 200], 2, 640),
+])
+def test_tensor_memory_staging_matches_oracle(B, L, K, N, monkeypatch):
+    """The persistent kernel's optional second staging level (FMTP_TMEM=1, read when the context is created): a shape
+    whose contraction lengths are all multiples of the 512-wide stage (d=2048, 8/2 heads of 128, ffn 1536), so that
+    every phase runs its first eight stages through tensor memory and the rest from the shared-memory stages in the
+    slot layout; also against the same call without it."""
+    shape = I.Shape(d=2048, n_q_heads=8, n_kv_heads=2, head_dim=128, ffn=1536, vocab=4096, n_layers=1, rms_eps=1e-6,
+                    rope_theta=1e4, page_size=16)
+    monkeypatch.setenv("FMTP_TMEM", "1")
+    got, ref = run_draft_case(shape, 4100 + B, B, L, K, N)
+    check_draft(got, ref, f"tmem B={B} K={K} N={N}")
+    assert got["launches"] == 1 and got["tmem_launches"] == 1
+    monkeypatch.setenv("FMTP_TMEM", "0")
+    plain, _ = run_draft_case(shape, 4100 + B, B, L, K, N)
+    assert plain["tmem_launches"] == 0
+    assert np.array_equal(plain["drafts"], got["drafts"])
+    close(plain["logits"], got["logits"], "tmem vs plain logits")
 
 
 @pytest.mark.parametrize("B,L,K,N", [
