@@ -52,13 +52,6 @@ __device__ __forceinline__ void cp_async_arrive(uint64_t *bar) {
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
-// One contiguous block global -> shared by the copy engine (both addresses 16-byte aligned, size a multiple of 16);
-// its bytes count on `bar` (armed with mbar_arrive_expect_tx for the same number of bytes). `policy`: an L2 policy.
-__device__ __forceinline__ void bulk_g2s_hint(void *dst_smem, const void *src_gmem, uint32_t bytes, uint64_t *bar, uint64_t policy) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-                 ::"r"(smem_u32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
-}
-
 // Orders generic-proxy shared-memory writes before later async-proxy (bulk copy) writes.
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
