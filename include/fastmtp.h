@@ -70,7 +70,9 @@ typedef enum {
  *     stream that read every weight once per group (tensor-core GEMMs).
  * Within a path a sequence's results do not depend on the batch it is in; between the two paths
  * results agree within the documented tolerances, not bit for bit (different summation order).
- * The environment variable FMTP_BATCHED_MIN (read at fmtp_create) overrides the switch point. */
+ * The environment variable FMTP_BATCHED_MIN (read at fmtp_create) overrides the switch point; FMTP_TMEM=1 (also read
+ * at fmtp_create) lets the persistent kernel stage weights through tensor memory where the shape allows (results agree
+ * with the default within the tolerances of the tests, not bit for bit: the k chunks are dealt to the warps differently). */
 typedef struct {
     int32_t d, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
     int32_t n_layers;      /* target decoder depth (fastmtp_target_step); the MTP head has 1 */

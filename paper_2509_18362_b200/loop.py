@@ -16,32 +16,43 @@ from . import binding as Bd
 
 class Target:
     """Device copies of a target model's weights and per-layer paged caches (dicts of torch tensors as
-    produced by binding.to_device), stepped through fastmtp_target_step."""
+    produced by binding.to_device), stepped through fastmtp_target_step.
+
+    All layers hold the same sequence lengths, so they share layer 0's seq_lens tensor: advancing the
+    sequence is one device-side add, whose amount may itself be a device tensor (no host round trip)."""
 
     def __init__(self, ctx, shape, dev_weights, dev_kvs):
         self.ctx, self.shape = ctx, shape
         self.dW = dev_weights
         self.w, self._keep = Bd.target_w(dev_weights)
         self.dkvs = dev_kvs
+        self.seq_lens = dev_kvs[0]["seq_lens"]
+        for k in dev_kvs[1:]:
+            k["seq_lens"] = self.seq_lens
+        self._kvs = [Bd.kv(k) for k in dev_kvs]          # the structs hold addresses only: built once
         self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
         self.calls = 0
 
     def step(self, tokens, want_logits=False):
-        """tokens: [B, M] ids. Returns (hidden states [B, M, d] bf16, logits [B, M, V] bf16 or None,
-        greedy token per row [B, M] int32), all on the device."""
+        """tokens: [B, M] ids (host list / array, or an int32 device tensor, which is used as it is).
+        Returns (hidden states [B, M, d] bf16, logits [B, M, V] bf16 or None, greedy token per row
+        [B, M] int32), all on the device."""
         s = self.shape
-        t = torch.as_tensor(np.asarray(tokens, dtype=np.int32)).cuda()
+        if isinstance(tokens, torch.Tensor) and tokens.is_cuda:
+            t = tokens.contiguous()
+        else:
+            t = torch.as_tensor(np.asarray(tokens, dtype=np.int32)).cuda()
         B, M = t.shape
         out_h = torch.empty((B, M, s.d), dtype=torch.bfloat16, device="cuda")
         out_l = torch.empty((B, M, s.vocab), dtype=torch.bfloat16, device="cuda") if want_logits else None
         out_a = torch.full((B, M), -1, dtype=torch.int32, device="cuda")
-        self.ctx.fastmtp_target_step(self.w, t, [Bd.kv(k) for k in self.dkvs], B, M, out_h, out_l, out_a, self.status)
+        self.ctx.fastmtp_target_step(self.w, t, self._kvs, B, M, out_h, out_l, out_a, self.status)
         self.calls += 1
         return out_h, out_l, out_a
 
     def advance(self, n):
-        for k in self.dkvs:
-            k["seq_lens"] += int(n)
+        """n: a host integer or an int32 device tensor broadcastable to [B]."""
+        self.seq_lens += n
 
 
 def prefill(tgt: Target, prompt, chunk=8):
@@ -58,14 +69,15 @@ def prefill(tgt: Target, prompt, chunk=8):
 
 
 def greedy_decode(tgt: Target, prompt, n_new, chunk=8):
-    """Vanilla autoregressive greedy decoding: the sequence the speculative loop must reproduce."""
+    """Vanilla autoregressive greedy decoding: the sequence the speculative loop must reproduce. The greedy token
+    of a step is fed to the next step on the device; the host reads all of them once at the end."""
     _, first = prefill(tgt, prompt, chunk)
-    out = [first]
-    while len(out) < n_new:
-        _, _, a = tgt.step([[out[-1]]])
+    toks = [torch.tensor([[first]], dtype=torch.int32, device="cuda")]
+    while len(toks) < n_new:
+        _, _, a = tgt.step(toks[-1])
         tgt.advance(1)
-        out.append(int(a[0, 0].item()))
-    return out
+        toks.append(a)
+    return [int(t) for t in torch.cat(toks, dim=1)[0].tolist()]
 
 
 def speculative_decode(tgt: Target, mtp_w, mtp_kv, subset, prompt, n_new, K, inject=None, chunk=8, ext_chunk=64,
@@ -91,32 +103,37 @@ def speculative_decode(tgt: Target, mtp_w, mtp_kv, subset, prompt, n_new, K, inj
     out = [first]
     drafts_d = torch.zeros((1, K), dtype=torch.int32, device="cuda")
     scratch_d = torch.zeros((1, 1), dtype=torch.int32, device="cuda")
+    last_d = torch.zeros((1, 1), dtype=torch.int32, device="cuda")
     acc = torch.zeros(1, dtype=torch.int32, device="cuda")
     bon = torch.zeros(1, dtype=torch.int32, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     accepted, rnd = [], 0
     calls0 = tgt.calls
+    mkv_c = Bd.kv(mtp_kv)                                  # addresses only; seq_lens is advanced in place
     while len(out) < n_new:
         n, pos = len(pend_t), 0
         tok_all = torch.tensor(pend_t, dtype=torch.int32, device="cuda")
         while n - pos > max_ext:                           # a backlog (the prompt): whole chunks first, their draft dropped
             m = min(ext_chunk, n - pos - 1)
-            ctx.fastmtp_draft(mtp_w, pend_h[pos:pos + m].contiguous(), tok_all[pos:pos + m].contiguous(), Bd.kv(mtp_kv), 1, 1,
+            ctx.fastmtp_draft(mtp_w, pend_h[pos:pos + m].contiguous(), tok_all[pos:pos + m].contiguous(), mkv_c, 1, 1,
                               subset, scratch_d, None, None, status, max_ext=m)
             mtp_kv["seq_lens"] += m
             pos += m
         m = n - pos
-        ctx.fastmtp_draft(mtp_w, pend_h[pos:].contiguous(), tok_all[pos:].contiguous(), Bd.kv(mtp_kv), 1, K, subset, drafts_d,
+        ctx.fastmtp_draft(mtp_w, pend_h[pos:].contiguous(), tok_all[pos:].contiguous(), mkv_c, 1, K, subset, drafts_d,
                           None, None, status, max_ext=m)
         mtp_kv["seq_lens"] += m
-        drafts = [int(t) for t in drafts_d[0].tolist()]
         if inject is not None:
             forced = inject(rnd, K, len(out))
             if forced is not None:
-                drafts = [int(t) for t in forced]
-        h, _, a = tgt.step([[out[-1]] + drafts])
-        ctx.fastmtp_accept_ids(a, torch.tensor([drafts], dtype=torch.int32, device="cuda"), 1, K, acc, bon)
-        na, bonus = int(acc.item()), int(bon.item())
+                drafts_d.copy_(torch.tensor([[int(t) for t in forced]], dtype=torch.int32), non_blocking=True)
+        # the target scores [last token, drafts]; both stay on the device, and the round's one read-back brings the
+        # drafts, the accepted length and the bonus token together
+        last_d[0, 0] = out[-1]
+        h, _, a = tgt.step(torch.cat([last_d, drafts_d], dim=1))
+        ctx.fastmtp_accept_ids(a, drafts_d, 1, K, acc, bon)
+        rec = torch.cat([drafts_d[0], acc, bon]).tolist()
+        drafts, na, bonus = [int(t) for t in rec[:K]], int(rec[K]), int(rec[K + 1])
         tgt.advance(na + 1)
         new = drafts[:na] + [bonus]
         out.extend(new)
