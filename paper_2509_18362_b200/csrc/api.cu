@@ -155,7 +155,9 @@ int configure(fmtp_ctx *c, MegaParams &p, int mode, int B, int M) {
     p.wait_limit_ns = kDefaultWaitNs;
     p.mode = mode; p.B = B; p.M = M; p.R = B * M;
     const int R = p.R, Gq = p.Hq / p.Hkv;
-    size_t attn = (size_t)M * Gq * p.dh * 4;
+    // attention scratch: the rows' query vectors, then one (o, m, l) buffer per working warp group (the rows of a call
+    // are dealt to two groups): [4 warps][8 heads][dh + 2] + 64 words
+    size_t attn = (size_t)M * Gq * p.dh * 4 + (size_t)(M > 1 ? 2 : 1) * (4 * 8 * (p.dh + 2) + 64) * 4;
     size_t mrg = ((size_t)2 * c->max_chunks + (size_t)kConsumerThreads + 64) * 4;      // chunk-merge scratch
     if (mrg > attn) attn = mrg;
     size_t actd = (size_t)2 * R * act_stride(mode == 0 ? 2 * p.d : (p.d > p.qdim ? p.d : p.qdim)) * 2;

@@ -18,8 +18,9 @@
 //   * RMSNorm is folded: the producing phase stores x*g (split hi/lo) plus per-CTA partial sums of
 //     x^2; the consuming phase multiplies its accumulators by rsqrt(mean(x^2)+eps).
 //   * Attention splits the context into fixed 64-token chunks (work items over sequence x KV head
-//     x chunk) whose committed K/V the producers stream through the same ring, fp32 softmax per
-//     chunk; after a grid barrier a merge phase, spread over all CTAs, combines a head's chunk
+//     x chunk) whose committed K/V the producers stream through the same ring; scores and the weighted sum
+//     run on mma.sync with the query heads (and the probabilities) split into bf16 high and low parts, fp32 softmax
+//     per chunk; after a grid barrier a merge phase, spread over all CTAs, combines a head's chunk
 //     partials in ascending order -- no float atomics anywhere, results are reproducible.
 //   * Producers and consumers each walk the phase program from ONE loop with a runtime phase
 //     kind: the code is much larger than the instruction cache, and straight-line code that runs
@@ -969,135 +970,150 @@ __device__ __forceinline__ void flush_sq(const Cta &c, const SqAcc &q, float *tb
 // the 64 K rows. The consumers add the positions this launch produced (earlier draft steps from
 // the pages, this call's rows from the QKV scratch, rotated and rounded to bf16 exactly as they
 // are stored) into the same stage buffer and then work from shared memory only.
-// Scratch: qs[M*Gq][dh] rotated, pre-scaled queries of one KV head. The per-warp partials
-// wp[8 warps][Gq][dh + 2] (o, m, l) reuse the stage buffer once K and V are in registers.
+// Scratch: qs[M*Gq][dh] rotated, pre-scaled queries of one KV head, then the per-warp partials (o, m, l) of the
+// working warp groups.
 
-// One chunk of one KV head from shared memory, for every row of the call: each warp takes 8 tokens.
-// Scores: lane = (quarter of the head dimension, token); the four quarters are added with two
-// shuffles. Softmax statistics are per warp (merged across warps, then across chunks, in fixed
-// order). P*V: lane owns DH/32 output elements, probabilities are broadcast by shuffle.
-// The loop over query heads is a real loop (not unrolled) to keep this once-per-step code small.
+// One chunk of one KV head on the tensor cores, for every row of the call. K and V stay in the stage (16-byte piece w
+// of token row t stored at piece w ^ (t & 7), so that ldmatrix reads without bank conflicts). The consumer warps
+// form two groups of four; group g takes the rows m = g, g + 2, ..., so a row's arithmetic does not depend on how
+// many rows the call carries. Within a group warp wi owns tokens 16*wi .. 16*wi+15 of the chunk. Scores: the query
+// heads are the A operand (rows 0-7 the bf16 high parts of up to eight heads, rows 8-15 the low parts: products with
+// the bf16 keys are exact), K fragments by ldmatrix; softmax statistics per warp; P*V with the probabilities split
+// the same way, V fragments by transposing ldmatrix. The four warps' (o, m, l) are merged in warp order, then the
+// chunks in ascending order by the merge phase.
 template <int DH>
-__device__ __forceinline__ void attn_rows(Cta &c, bf16_t *sk, const bf16_t *sv, const float *qs,
-                                          int b, int kvh, int chunk, int base, int max_tokens, int rows) {
+__device__ __forceinline__ void attn_rows_mma(Cta &c, const bf16_t *sk, const bf16_t *sv, const float *qs, float *part,
+                                              int b, int kvh, int chunk, int base, int max_tokens, int rows) {
     const MegaParams &p = *c.p;
-    constexpr int SEG = DH / 4, EPL = DH / 32, wstride = DH + 2;
+    constexpr int wstride = DH + 2;
     const int Gq = p.Hq / p.Hkv, M = c.M;
     const int c0 = chunk * kAttnChunk;
-    const int tl = c.warp * 8;                       // first token (within the chunk) of this warp
-    // lanes of a quarter-warp share `part`, so a 128-bit query load is one broadcast per quarter
-    // (with part = lane & 3 the four parts of a quarter hit the same banks: 4x the wavefronts)
-    const int tkk = c.lane & 7, part = c.lane >> 3;
-    const int e0 = c.lane * EPL;
-    const uint32_t qs_u32 = smem_u32(qs);
-    // this warp's K slice (token tkk, quarter `part`) and V rows (8 tokens x EPL elements) in registers
-    float kf[SEG], vf[8][EPL];
-    {
-        const uint4 *kr = reinterpret_cast<const uint4 *>(sk + (size_t)(tl + tkk) * DH + part * SEG);
-#pragma unroll
-        for (int i = 0; i < SEG / 8; ++i) {
-            uint4 w = kr[i];
-            kf[8 * i + 0] = bf16lo_f32(w.x); kf[8 * i + 1] = bf16hi_f32(w.x);
-            kf[8 * i + 2] = bf16lo_f32(w.y); kf[8 * i + 3] = bf16hi_f32(w.y);
-            kf[8 * i + 4] = bf16lo_f32(w.z); kf[8 * i + 5] = bf16hi_f32(w.z);
-            kf[8 * i + 6] = bf16lo_f32(w.w); kf[8 * i + 7] = bf16hi_f32(w.w);
-        }
-#pragma unroll
-        for (int tk = 0; tk < 8; ++tk) {
-            const bf16_t *vr = sv + (size_t)(tl + tk) * DH + e0;
-            if (EPL == 4) {
-                uint2 w = *reinterpret_cast<const uint2 *>(vr);
-                vf[tk][0] = bf16lo_f32(w.x); vf[tk][1] = bf16hi_f32(w.x); vf[tk][EPL - 2] = bf16lo_f32(w.y); vf[tk][EPL - 1] = bf16hi_f32(w.y);
-            } else {
-                uint32_t w = *reinterpret_cast<const uint32_t *>(vr);
-                vf[tk][0] = bf16lo_f32(w); vf[tk][1] = bf16hi_f32(w);
-            }
-        }
-    }
-    // K and V now live in registers: the stage buffer is reused for the per-warp partials
-    // wp[8 warps][Gq][DH + 2] (o, m, l) and the merge weights behind them
-    bar_sync(1, kConsumerThreads);
-    float *wp = reinterpret_cast<float *>(sk);
-    PROF(c, ATTN * 8 + 6);
+    const int grp = c.warp >> 2, wi = c.warp & 3;
+    const int hrow = c.lane >> 2, kq = (c.lane & 3) * 2;
+    const int tw = wi * 16;                                  // first token (within the chunk) of this warp
+    float *wp = part + (size_t)grp * (4 * 8 * wstride + 64);  // this group's [4 warps][8 heads][DH + 2], then 32 weights, 8 x (m, l)
+    float *fw = wp + 4 * 8 * wstride;
+    const uint32_t sk_u = smem_u32(sk), sv_u = smem_u32(sv);
+    // ldmatrix row addresses (see the batched attention kernel): K: matrices (tokens 0-7, dims 0-7), (0-7, 8-15),
+    // (8-15, 0-7), (8-15, 8-15) of a 16-dim slice; V (transposed): (tokens 0-7, dims 0-7), (8-15, 0-7), (0-7, 8-15), (8-15, 8-15)
+    const int ktok = tw + (c.lane & 7) + ((c.lane >> 4) << 3), kpc = (c.lane >> 3) & 1;
+    const int vtok = tw + (c.lane & 7) + (((c.lane >> 3) & 1) << 3), vpc = c.lane >> 4;
+    const uint32_t krow = sk_u + (uint32_t)ktok * (DH * 2), vrow = sv_u + (uint32_t)vtok * (DH * 2);
+    const uint32_t ksw = (uint32_t)(ktok & 7), vsw = (uint32_t)(vtok & 7);
 #pragma unroll 1
-    for (int m = 0; m < M; ++m) {
+    for (int m = grp; m < M; m += 2) {
         const int npos = min(base + min(m, rows - 1), max_tokens - 1);   // last visible position of this row
-        const int nvis = min(8, npos - (c0 + tl) + 1);    // visible tokens of this warp (may be <= 0)
 #pragma unroll 1
-        for (int h = 0; h < Gq; ++h) {
-            // all query loads first (explicit shared-memory loads), then four independent partial sums
-            const uint32_t qa = qs_u32 + (uint32_t)(((m * Gq + h) * DH + part * SEG) * 4);
-            uint4 qw[SEG / 4];
+        for (int h0 = 0; h0 < Gq; h0 += 8) {                             // eight query heads per pass
+            const int nh = min(8, Gq - h0);
+            // query fragments from the fp32 vectors: hi parts in rows 0-7, lo parts in rows 8-15
+            uint32_t qa[DH / 16][4];
+            {
+                const float *qh = qs + ((size_t)(m * Gq + h0 + hrow)) * DH;
 #pragma unroll
-            for (int i = 0; i < SEG / 4; ++i) qw[i] = lds128_u32(qa + 16 * i);
-            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-            for (int i = 0; i < SEG / 4; ++i) {
-                s0 += __uint_as_float(qw[i].x) * kf[4 * i];
-                s1 += __uint_as_float(qw[i].y) * kf[4 * i + 1];
-                s2 += __uint_as_float(qw[i].z) * kf[4 * i + 2];
-                s3 += __uint_as_float(qw[i].w) * kf[4 * i + 3];
-            }
-            float s = (s0 + s1) + (s2 + s3);
-            s += __shfl_xor_sync(0xffffffffu, s, 8);
-            s += __shfl_xor_sync(0xffffffffu, s, 16);
-            if (tkk >= nvis) s = -INFINITY;
-            float mx = s;
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-            const float pe = (s == -INFINITY) ? 0.f : expf(s - mx);
-            float sm = pe;
-            sm += __shfl_xor_sync(0xffffffffu, sm, 1);
-            sm += __shfl_xor_sync(0xffffffffu, sm, 2);
-            sm += __shfl_xor_sync(0xffffffffu, sm, 4);
-            // o[e] = sum over the warp's tokens (ascending) of p * V
-            float o[EPL];
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) o[e] = 0.f;
-#pragma unroll
-            for (int tk = 0; tk < 8; ++tk) {
-                const float pr = __shfl_sync(0xffffffffu, pe, tk);
-                if (tk < nvis) {
-#pragma unroll
-                    for (int e = 0; e < EPL; ++e) o[e] += pr * vf[tk][e];
+                for (int ks = 0; ks < DH / 16; ++ks) {
+                    float2 x0 = make_float2(0.f, 0.f), x1 = make_float2(0.f, 0.f);
+                    if (hrow < nh) {
+                        x0 = *reinterpret_cast<const float2 *>(qh + ks * 16 + kq);
+                        x1 = *reinterpret_cast<const float2 *>(qh + ks * 16 + kq + 8);
+                    }
+                    uint16_t h0a, l0a, h0b, l0b, h1a, l1a, h1b, l1b;
+                    split_bf16(x0.x, h0a, l0a); split_bf16(x0.y, h0b, l0b);
+                    split_bf16(x1.x, h1a, l1a); split_bf16(x1.y, h1b, l1b);
+                    qa[ks][0] = (uint32_t)h0a | ((uint32_t)h0b << 16);
+                    qa[ks][1] = (uint32_t)l0a | ((uint32_t)l0b << 16);
+                    qa[ks][2] = (uint32_t)h1a | ((uint32_t)h1b << 16);
+                    qa[ks][3] = (uint32_t)l1a | ((uint32_t)l1b << 16);
                 }
             }
-            float *w = wp + ((size_t)c.warp * Gq + h) * wstride;
+            // scores of this warp's 16 tokens (two n-tiles of 8)
+            float s[2][4];
+            s[0][0] = s[0][1] = s[0][2] = s[0][3] = 0.f;
+            s[1][0] = s[1][1] = s[1][2] = s[1][3] = 0.f;
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) w[e0 + e] = o[e];
-            if (c.lane == 0) { w[DH] = mx; w[DH + 1] = sm; }
-        }
-        bar_sync(1, kConsumerThreads);
-        // ---- merge the 8 warps (fixed order) -> chunk partial in global memory.
-        // weight of warp w for head h: thread (h, w) computes it once
-        float *fw = wp + (size_t)kConsumerWarps * Gq * wstride;      // [Gq][8] weights, then [Gq][2] (m, l)
-        if (c.tid < Gq * kConsumerWarps) {
-            const int h = c.tid >> 3, w = c.tid & 7;
-            float mx = -INFINITY;
-#pragma unroll
-            for (int q = 0; q < kConsumerWarps; ++q) mx = fmaxf(mx, wp[((size_t)q * Gq + h) * wstride + DH]);
-            const float mw = wp[((size_t)w * Gq + h) * wstride + DH];
-            fw[h * kConsumerWarps + w] = (mw == -INFINITY) ? 0.f : expf(mw - mx);
-            if (w == 0) fw[Gq * kConsumerWarps + 2 * h] = mx;
-        }
-        bar_sync(1, kConsumerThreads);
-        for (int i = c.tid; i < Gq * DH; i += kConsumerThreads) {
-            const int h = i / DH, e = i - h * DH;
-            float ov = 0.f, l = 0.f;
-#pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) {
-                const float *pw = wp + ((size_t)w * Gq + h) * wstride;
-                const float f = fw[h * kConsumerWarps + w];
-                ov += f * pw[e];
-                l += f * pw[DH + 1];
+            for (int ks = 0; ks < DH / 16; ++ks) {
+                uint32_t b00, b01, b10, b11;
+                asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(b00), "=r"(b01), "=r"(b10), "=r"(b11) : "r"(krow + ((((uint32_t)(ks * 2 + kpc)) ^ ksw) << 4)));
+                mma_bf16(s[0], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b00, b01);
+                mma_bf16(s[1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b10, b11);
             }
-            const int r = b * M + m, hq = kvh * Gq + h;
-            float *dst = p.s.att_part + (((size_t)r * p.Hq + hq) * p.max_chunks + chunk) * wstride;
-            dst[e] = ov;
-            if (e == 0) { dst[DH] = fw[Gq * kConsumerWarps + 2 * h]; dst[DH + 1] = l; }
+            // thread: head hrow, tokens tw + nt*8 + kq + {0,1}; hi-part product in [0],[1], lo-part in [2],[3]
+            float sc[4], mx = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    float v = s[nt][j] + s[nt][j + 2];
+                    if (c0 + tw + nt * 8 + kq + j > npos) v = -INFINITY;
+                    sc[nt * 2 + j] = v;
+                    mx = fmaxf(mx, v);
+                }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            float psum = 0.f;
+            uint32_t pa[4];
+            {
+                float pr[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { pr[i] = (sc[i] == -INFINITY) ? 0.f : expf(sc[i] - mx); psum += pr[i]; }
+                uint16_t h0, l0, h1, l1, h2, l2, h3, l3;
+                split_bf16(pr[0], h0, l0); split_bf16(pr[1], h1, l1); split_bf16(pr[2], h2, l2); split_bf16(pr[3], h3, l3);
+                pa[0] = (uint32_t)h0 | ((uint32_t)h1 << 16);      // row hrow,     tokens kq, kq+1
+                pa[1] = (uint32_t)l0 | ((uint32_t)l1 << 16);      // row hrow + 8
+                pa[2] = (uint32_t)h2 | ((uint32_t)h3 << 16);      // row hrow,     tokens 8+kq, 8+kq+1
+                pa[3] = (uint32_t)l2 | ((uint32_t)l3 << 16);
+            }
+            psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+            psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+            // o[head][dim] = sum over the warp's tokens of p * V
+            float o[DH / 8][4];
+#pragma unroll
+            for (int nt = 0; nt < DH / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < DH / 8; nt += 2) {
+                uint32_t b00, b01, b10, b11;
+                asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(b00), "=r"(b01), "=r"(b10), "=r"(b11) : "r"(vrow + ((((uint32_t)(nt + vpc)) ^ vsw) << 4)));
+                mma_bf16(o[nt], pa[0], pa[1], pa[2], pa[3], b00, b01);
+                mma_bf16(o[nt + 1], pa[0], pa[1], pa[2], pa[3], b10, b11);
+            }
+            // ---- merge the group's four warps (fixed order) -> chunk partial in global memory
+            {
+                float *w = wp + ((size_t)wi * 8 + hrow) * wstride;
+#pragma unroll
+                for (int nt = 0; nt < DH / 8; ++nt) { w[nt * 8 + kq] = o[nt][0] + o[nt][2]; w[nt * 8 + kq + 1] = o[nt][1] + o[nt][3]; }
+                if ((c.lane & 3) == 0) { w[DH] = mx; w[DH + 1] = psum; }
+            }
+            bar_sync(3 + grp, 128);
+            const int gt = c.tid & 127;                      // thread within the group
+            if (gt < 32) {                                   // thread = (head gt >> 2, warp gt & 3): the warp's weight
+                const int h = gt >> 2, w = gt & 3;
+                float mm = -INFINITY;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) mm = fmaxf(mm, wp[((size_t)q * 8 + h) * wstride + DH]);
+                const float mw = wp[((size_t)w * 8 + h) * wstride + DH];
+                fw[w * 8 + h] = (mw == -INFINITY) ? 0.f : expf(mw - mm);
+                if (w == 0) fw[32 + 2 * h] = mm;
+            }
+            bar_sync(3 + grp, 128);
+            for (int i = gt; i < nh * DH; i += 128) {
+                const int h = i / DH, e = i - h * DH;
+                float ov = 0.f, l = 0.f;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    const float *pw = wp + ((size_t)w * 8 + h) * wstride;
+                    const float f = fw[w * 8 + h];
+                    ov += f * pw[e];
+                    l += f * pw[DH + 1];
+                }
+                const int r = b * M + m, hq = kvh * Gq + h0 + h;
+                float *dst = p.s.att_part + (((size_t)r * p.Hq + hq) * p.max_chunks + chunk) * wstride;
+                dst[e] = ov;
+                if (e == 0) { dst[DH] = fw[32 + 2 * h]; dst[DH + 1] = l; }
+            }
+            bar_sync(3 + grp, 128);                          // the group's buffer is free for its next pass
         }
-        bar_sync(1, kConsumerThreads);
     }
 }
 
@@ -1172,7 +1188,7 @@ __device__ __forceinline__ void produce_attention(Cta &c, const KvPtrs &kv, int 
                 int page = bt[j / p.page];
                 if ((unsigned)page >= (unsigned)kv.num_pages) { raise(c, kDevBadPage); page = 0; }
                 size_t off = ((((size_t)page * p.Hkv + it.kvh) * p.page + (j % p.page)) * p.dh) * 2 + (size_t)w * 16;
-                d[i] = dst0 + (uint32_t)(tok * p.dh * 2 + w * 16);
+                d[i] = dst0 + (uint32_t)(tok * p.dh * 2 + ((w ^ (tok & 7)) << 4));      // piece w of token row tok at w ^ (tok & 7)
                 qk[i] = reinterpret_cast<const unsigned char *>(kv.k_pages) + off;
                 qv[i] = reinterpret_cast<const unsigned char *>(kv.v_pages) + off;
             }
@@ -1248,8 +1264,9 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int st
                 int page = bt[j / p.page];
                 if ((unsigned)page >= (unsigned)kv.num_pages) { raise(c, kDevBadPage); page = 0; }
                 size_t off = (((size_t)page * p.Hkv + kvh) * p.page + (j % p.page)) * dh + (size_t)w * 8;
-                *reinterpret_cast<uint4 *>(sk + (size_t)(j - c0) * dh + w * 8) = ldcg128(kv.k_pages + off);
-                *reinterpret_cast<uint4 *>(sv + (size_t)(j - c0) * dh + w * 8) = ldcg128(kv.v_pages + off);
+                const int ws = w ^ ((j - c0) & 7);                       // the stage's piece order (see attn_rows_mma)
+                *reinterpret_cast<uint4 *>(sk + (size_t)(j - c0) * dh + ws * 8) = ldcg128(kv.k_pages + off);
+                *reinterpret_cast<uint4 *>(sv + (size_t)(j - c0) * dh + ws * 8) = ldcg128(kv.v_pages + off);
             }
         }
         // -- this call's rows: rotate, round to bf16, put into the stage and append to the cache
@@ -1266,7 +1283,9 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int st
             uint16_t k0 = f32_bf16bits(x * cs - y * sn), k1 = f32_bf16bits(y * cs + x * sn);
             uint16_t v0 = f32_bf16bits(ldcg_f32(vv + e)), v1 = f32_bf16bits(ldcg_f32(vv + e + half));
             bf16_t *dk = sk + (size_t)(pos - c0) * dh, *dv = sv + (size_t)(pos - c0) * dh;
-            dk[e] = k0; dk[e + half] = k1; dv[e] = v0; dv[e + half] = v1;
+            const int sw = (pos - c0) & 7;
+            const int ea = (((e >> 3) ^ sw) << 3) + (e & 7), eb = ((((e + half) >> 3) ^ sw) << 3) + ((e + half) & 7);
+            dk[ea] = k0; dk[eb] = k1; dv[ea] = v0; dv[eb] = v1;
             int page = bt[pos / p.page];
             if ((unsigned)page >= (unsigned)kv.num_pages) { raise(c, kDevBadPage); page = 0; }
             size_t o = (((size_t)page * p.Hkv + kvh) * p.page + (pos % p.page)) * dh;
@@ -1275,11 +1294,20 @@ __device__ __forceinline__ void attention_phase(Cta &c, const KvPtrs &kv, int st
             kv.v_pages[o + e] = v0;
             kv.v_pages[o + e + half] = v1;
         }
+        // -- value rows of the chunk's positions that nothing has written (beyond the last row of this call): zeros, so
+        // that a masked probability of 0 meets a finite number in the tensor-core product
+        {
+            const int last = min(base + rows - 1, max_tokens - 1);
+            const int nfill = max(0, min(kAttnChunk, last + 1 - c0));
+            for (int i = c.tid; i < (kAttnChunk - nfill) * upt; i += kConsumerThreads)
+                *reinterpret_cast<uint4 *>(sv + (size_t)nfill * dh + (size_t)i * 8) = make_uint4(0, 0, 0, 0);
+        }
         bar_sync(1, kConsumerThreads);
         PROF(c, ATTN * 8 + 5);
 
-        attn_rows<DH>(c, sk, sv, qs, b, kvh, chunk, base, max_tokens, rows);
-        // the stage is free again (all consumer warps passed the barrier at the end of attn_rows)
+        float *part = qs + (((size_t)M * Gq * dh + 3) & ~(size_t)3);
+        attn_rows_mma<DH>(c, sk, sv, qs, part, b, kvh, chunk, base, max_tokens, rows);
+        bar_sync(1, kConsumerThreads);   // every warp has read what it needs from the stage
         if (c.tid == 0) { volatile uint32_t *ud = &c.misc->use_done[slot]; *ud = *ud + 1; }   // see the mover of the tensor-memory path
         if (c.warp < kConsumerWarps / 2 && c.lane == 0) mbar_arrive(&c.misc->empty[slot]);
         next_stage(c);
