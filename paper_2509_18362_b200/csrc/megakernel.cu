@@ -907,16 +907,17 @@ __device__ __forceinline__ float reduce_partials(const float (&v)[kPartialRegs])
 // element offset `dst_off`.
 // With remap_step >= 1 row r is read from global row src_row(r, remap_step): the projection of draft step 1
 // continues each sequence's last extend row.
-__device__ __forceinline__ void stage_hilo(const Cta &c, const bf16_t *ghi, const bf16_t *glo, int gstride, int len, bf16_t *shi,
-                                           bf16_t *slo, int sstride, int dst_off, int remap_step = 0) {
+template <int U>
+__device__ __forceinline__ void stage_hilo_impl(const Cta &c, const bf16_t *ghi, const bf16_t *glo, int gstride, int len, bf16_t *shi,
+                                                bf16_t *slo, int sstride, int dst_off, int remap_step) {
     const int per_row = len / 8;
     const int total = c.R * per_row;
-    // four units per thread and round: eight loads in flight before the first store waits
+    // U units per thread and round: 2 U loads in flight before the first store waits
 #pragma unroll 1
-    for (int i0 = c.tid; i0 < total; i0 += 4 * kConsumerThreads) {
-        uint4 a[4], b[4];
+    for (int i0 = c.tid; i0 < total; i0 += U * kConsumerThreads) {
+        uint4 a[U], b[U];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < U; ++q) {
             int i = min(i0 + q * kConsumerThreads, total - 1);
             int r = i / per_row, k = (i - r * per_row) * 8;
             const int rs = remap_step > 0 ? src_row(c, r, remap_step) : r;
@@ -924,7 +925,7 @@ __device__ __forceinline__ void stage_hilo(const Cta &c, const bf16_t *ghi, cons
             b[q] = ldcg128(glo + (size_t)rs * gstride + k);
         }
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < U; ++q) {
             int i = i0 + q * kConsumerThreads;
             if (i < total) {
                 int r = i / per_row, k = (i - r * per_row) * 8;
@@ -933,6 +934,12 @@ __device__ __forceinline__ void stage_hilo(const Cta &c, const bf16_t *ghi, cons
             }
         }
     }
+}
+__device__ __forceinline__ void stage_hilo(const Cta &c, const bf16_t *ghi, const bf16_t *glo, int gstride, int len, bf16_t *shi,
+                                           bf16_t *slo, int sstride, int dst_off, int remap_step = 0) {
+    // several rows: twice as many loads per round, so that the copy stays at one or two L2 round trips
+    if (c.R * (len / 8) > 4 * kConsumerThreads) stage_hilo_impl<8>(c, ghi, glo, gstride, len, shi, slo, sstride, dst_off, remap_step);
+    else stage_hilo_impl<4>(c, ghi, glo, gstride, len, shi, slo, sstride, dst_off, remap_step);
 }
 
 __device__ __forceinline__ void flush_sq(const Cta &c, const SqAcc &q, float *tblA, float *tblB) {
