@@ -133,7 +133,7 @@ class ClockSampler:
 # DRAM traffic of one mega_kernel launch on the default workload, from the ncu capture summarised in
 # profiles/mega_kernel_7b_batch1_ncu.md (dram__bytes_read.sum + dram__bytes_write.sum). It is only
 # reported while the kernel sources are the ones the counters were taken from.
-NCU_TRAFFIC = {"bytes_per_launch": 2270611456 + 5941760, "sources_sha256": "710410f76df4f7b31c86753f4ce4c7b2a23e0b635b391ec48d4b028b368a91d1"}
+NCU_TRAFFIC = {"bytes_per_launch": 2261775616 + 4454656, "sources_sha256": "0da243f1dc023a98448c7c3b333abc2c2313b16b2c9368758d1d5de0b8b32421"}
 def kernel_sources_sha256():
     """Hash of every source the library is compiled from (all of csrc/ and the public header)."""
     import hashlib
