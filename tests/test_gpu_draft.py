@@ -175,6 +175,20 @@ def test_batched_path_odd_geometry():
     check_draft(got, ref, "odd geometry batched")
 
 
+@pytest.mark.parametrize("B,L,K", [
+    (1, [191], 3),                # last chunk one token short of full: the rows written in this call cross into a new chunk
+    (3, [0, 64, 130], 2),         # empty context, chunk-aligned context
+    (12, [0, 5, 63, 64, 65, 127, 128, 129, 200, 255, 256, 300], 2),   # the batched path's attention at the same geometry
+])
+def test_eight_query_heads_per_kv_head(B, L, K):
+    """The widest group the library takes (8 query heads on one KV head, head_dim 64): every row of the attention
+    operand carries a head, in the persistent kernel (1 and 3 sequences) and on the batched path (12)."""
+    shape = I.Shape(d=512, n_q_heads=8, n_kv_heads=1, head_dim=64, ffn=1024, vocab=2048, n_layers=1,
+                    rms_eps=1e-6, rope_theta=1e4, page_size=16)
+    got, ref = run_draft_case(shape, 8800 + B, B, L, K, 500)
+    check_draft(got, ref, f"8 heads per KV head B={B}")
+
+
 def test_batched_path_bit_reproducible_and_batch_invariant():
     """Two runs agree bit for bit, and a sequence's result is the same in a group of 12 and of 40."""
     L = [int(x) for x in I.context_lengths(40, 0, 300, 5)]
