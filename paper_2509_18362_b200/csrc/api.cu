@@ -144,10 +144,6 @@ int configure(fmtp_ctx *c, MegaParams &p, int mode, int B, int M) {
     {   // a stage also has to hold one 64-token K/V chunk of a KV head
         int kvb = 2 * kAttnChunk * p.dh * 2;
         if (kvb > p.stage_bytes) p.stage_bytes = kvb;
-        // ... and, once K/V sit in registers, the per-warp attention partials that reuse the buffer
-        const int gq = p.Hq / p.Hkv;
-        int wpb = (kConsumerWarps * gq * (p.dh + 2) + gq * (kConsumerWarps + 2)) * 4;
-        if (wpb > p.stage_bytes) p.stage_bytes = wpb;
         p.stage_bytes = (p.stage_bytes + 127) & ~127;
     }
     p.max_chunks = c->max_chunks;
@@ -304,7 +300,7 @@ int fmtp_create(const fmtp_shape *sh, fmtp_ctx **out) {
     // Which path a call takes depends on its number of sequences only (so a sequence scored with 1 or with K+1
     // rows takes the same path and gives the same bits). Small models: the persistent kernel as long as the
     // sequences fit one launch. Models that stream >= 256 MB of layer weights per step: the batched path from
-    // three sequences on (measured at the 7B shape: 185 us per step against 193 / 222 us at 3 / 4 sequences).
+    // three sequences on (measured at the 7B shape: 180 / 182 us per step against 181 / 208 us at 3 / 4 sequences).
     c->batched_min = g1 + 1;
     {
         const double qd = (double)sh->n_q_heads * sh->head_dim, kvd = (double)sh->n_kv_heads * sh->head_dim;
